@@ -1,0 +1,160 @@
+/*
+ * libapollo -- the APOLLO / APOLLO-Mini optimizer step on NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Every pointer argument is tagged HOST or DEVICE below.  Every function returns
+ * APOLLO_OK (0) or a negative APOLLO_ERR_* code; nothing is launched when validation
+ * fails; no exception crosses this boundary.  The library allocates no device memory: the
+ * caller owns the weights, the gradients and one workspace buffer and keeps them alive
+ * for the lifetime of the context.
+ *
+ * The method (Zhu et al., "APOLLO: SGD-like Memory, AdamW-level Performance",
+ * Algorithm 1).  For each 2-D weight W with gradient G, viewed as m x n with m <= n
+ * (m = the shorter stored side; on a tie the rows are the projected side):
+ *   1. P (r x m), entries N(0, 1/r), is regenerated from a counter-based Philox4x32-10
+ *      stream keyed by the seed, with counter (column quad, row, matrix index,
+ *      epoch = floor(t / T)); it is never stored (Algorithm 1, "P_t <- N_seed(0, 1/r)";
+ *      Section "Generating random projection matrix").
+ *   2. R = P G  (r x n)                                        (Algorithm 1, step 1).
+ *   3. M <- beta1 M + (1-beta1) R,  V <- beta2 V + (1-beta2) R^2,
+ *      R~ = M / (sqrt(V) + eps)                                (Algorithm 1, step 2).
+ *   4. channel mode: s_j = |R~[:,j]| / |R[:,j]|                (Eq. 5);
+ *      tensor mode (APOLLO-Mini): s = |R~|_F / |R|_F           (Section on APOLLO-Mini);
+ *      norm-growth limiter on the scaled gradient G diag(s)    (Eq. 4): if its
+ *      Frobenius norm exceeds gamma times the previous step's (limited) norm it is
+ *      rescaled by c = gamma * prev / norm.
+ *   5. W <- W - lr (alpha c s_j G_ij + wd W_ij)                (Algorithm 1, step 4;
+ *      G is the gradient of the loss, so the update subtracts).
+ */
+#ifndef APOLLO_H_
+#define APOLLO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define APOLLO_OK 0
+#define APOLLO_ERR_INVALID_ARG (-1) /* null pointer, non-finite scalar, bad enum, bad index */
+#define APOLLO_ERR_SHAPE (-2)       /* rows or cols < 1, or a side above 2^31 - 1 */
+#define APOLLO_ERR_RANK (-3)        /* rank < 1, rank > min(rows, cols) or rank > APOLLO_MAX_RANK */
+#define APOLLO_ERR_ALIGN (-4)       /* a device pointer is not 16-byte aligned */
+#define APOLLO_ERR_WORKSPACE (-5)   /* workspace smaller than apollo_workspace_bytes() */
+#define APOLLO_ERR_CUDA (-6)        /* a CUDA runtime or driver call failed */
+#define APOLLO_ERR_TIMEOUT (-7)     /* a bounded device-side wait expired (reported by apollo_status) */
+#define APOLLO_ERR_UNSUPPORTED (-8) /* the device is not an sm_100 part */
+
+#define APOLLO_MAX_RANK 512
+
+#define APOLLO_SCALE_CHANNEL 0 /* APOLLO: one scale per channel (Eq. 5) */
+#define APOLLO_SCALE_TENSOR 1  /* APOLLO-Mini: one scale per tensor (use with rank 1) */
+
+#define APOLLO_DT_F32 0  /* W and G are float */
+#define APOLLO_DT_BF16 1 /* W and G are bfloat16; W is stored with round-to-nearest-even */
+
+/* apollo_config.flags */
+#define APOLLO_FLAG_NO_TENSOR_CORES 1u /* run the projection on the CUDA cores (test and comparison aid) */
+
+typedef struct apollo_ctx apollo_ctx; /* opaque HOST object */
+
+typedef struct {
+    int64_t rows, cols; /* stored shape, row-major, contiguous (pitch = cols elements) */
+} apollo_shape;
+
+typedef struct {
+    int32_t rank;            /* r */
+    int32_t mode;            /* APOLLO_SCALE_* */
+    int32_t dtype;           /* APOLLO_DT_* of W and G; M, V, s and all reductions are fp32 */
+    int32_t T;               /* projection refresh period in steps, >= 1 (paper default 200) */
+    uint64_t seed;           /* Philox key */
+    float alpha;             /* gradient scale factor (1 for APOLLO, sqrt(128) for Mini) */
+    float gamma;             /* limiter threshold (paper default 1.01); <= 0 disables the limiter */
+    float beta1, beta2, eps; /* 0.9, 0.999, 1e-8 */
+    int32_t bias_correction; /* 0: moment equations as printed; 1: divide by 1-beta^t as Adam does */
+    uint32_t flags;          /* APOLLO_FLAG_* */
+} apollo_config;
+
+/*
+ * Bytes of DEVICE workspace a context over `shapes[0..n_matrices)` needs (moments, scales,
+ * partial sums, descriptor tables, tensor maps).  shapes, cfg, out: HOST.
+ */
+int apollo_workspace_bytes(const apollo_shape* shapes, int32_t n_matrices, const apollo_config* cfg,
+                           size_t* out_bytes);
+
+/*
+ * Create a context (Algorithm 1, "Initialize: t <- 0").  d_workspace: DEVICE, 256-byte
+ * aligned, workspace_bytes >= apollo_workspace_bytes(); owned by the caller, used
+ * exclusively by this context until apollo_destroy.  Launches nothing and touches no
+ * stream: the moments are zeroed (Appendix: "zero initialization") by the first
+ * apollo_step on that step's stream.  The matrix index in the list is the `matrix index`
+ * word of the Philox counter.  Must be called with the target device current.
+ */
+int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_matrices,
+                  const apollo_config* cfg, void* d_workspace, size_t workspace_bytes);
+
+/*
+ * One optimizer step over the whole parameter list (Algorithm 1, body of the loop).
+ * d_W, d_G: HOST arrays of n_matrices DEVICE pointers (16-byte aligned, dtype of the
+ * config, row-major rows x cols).  W is updated in place; G is read only.  lr and wd are
+ * the step size eta and the weight decay lambda.  Asynchronous on `cuda_stream`
+ * (a cudaStream_t; NULL = the legacy default stream); no host synchronisation; advances
+ * the step counter t.  Not thread-safe per context.
+ */
+int apollo_step(apollo_ctx* ctx, void* const* d_W, const void* const* d_G, float lr, float wd,
+                void* cuda_stream);
+
+int apollo_destroy(apollo_ctx* ctx);
+
+/* Number of steps taken so far (t of Algorithm 1).  out: HOST. */
+int apollo_step_count(const apollo_ctx* ctx, int64_t* out);
+
+/*
+ * Observability (used by the tests).  All copies are asynchronous on `cuda_stream`.
+ * apollo_get_scales:  d_out DEVICE, n floats: s_j of the last step (Eq. 5), n = max(rows, cols).
+ * apollo_get_limiter: d_out DEVICE, 4 floats: {norm after limiting (Eq. 4), factor c,
+ *                     norm before limiting, tensor-wise scale (tensor mode, else 0)}.
+ * apollo_get_state:   d_M, d_V DEVICE, r x n floats each, row-major (channel index contiguous).
+ */
+int apollo_get_scales(apollo_ctx* ctx, int32_t matrix, float* d_out, void* cuda_stream);
+int apollo_get_limiter(apollo_ctx* ctx, int32_t matrix, float* d_out, void* cuda_stream);
+int apollo_get_state(apollo_ctx* ctx, int32_t matrix, float* d_M, float* d_V, void* cuda_stream);
+
+/*
+ * Optional capture of the fp32 update dW = -lr (alpha c s_j G_ij + wd W_ij) before it is
+ * added to W and rounded (the quantity the parity bound is stated on).  d_dW: HOST array
+ * of n_matrices DEVICE pointers (rows x cols floats each), or NULL to switch capture off.
+ */
+int apollo_set_delta_out(apollo_ctx* ctx, float* const* d_dW);
+
+/*
+ * Synchronises `cuda_stream` and returns the device status word: APOLLO_OK, or
+ * APOLLO_ERR_TIMEOUT if a bounded wait inside a kernel expired since the last call.
+ */
+int apollo_status(apollo_ctx* ctx, void* cuda_stream);
+
+/*
+ * The generator by itself (Algorithm 1, "P_t <- N_seed(0, 1/r)"), for tests.
+ * apollo_philox_draws:  d_out DEVICE, r x ceil(m/4) x 4 uint32: the raw Philox4x32-10
+ *                       words for counter (q, k, matrix, epoch), key = seed.
+ * apollo_projection:    d_out DEVICE, r x m floats: the standard normals behind P after
+ *                       rounding to bfloat16 (P = d_out / sqrt(r)), exactly as the
+ *                       projection kernels materialise them.
+ */
+int apollo_philox_draws(uint64_t seed, uint32_t matrix, uint32_t epoch, int32_t r, int32_t m,
+                        uint32_t* d_out, void* cuda_stream);
+int apollo_projection(uint64_t seed, uint32_t matrix, uint32_t epoch, int32_t r, int32_t m,
+                      float* d_out, void* cuda_stream);
+
+/* Which projection kernel a matrix was assigned: 0 streaming (rank 1), 1 CUDA cores, 2 tensor cores. */
+int apollo_get_path(const apollo_ctx* ctx, int32_t matrix, int32_t* out);
+
+/* Kernel launches issued by the last apollo_step (HOST counter). */
+int apollo_last_launches(const apollo_ctx* ctx, int32_t* out);
+
+const char* apollo_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* APOLLO_H_ */
