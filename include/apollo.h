@@ -35,6 +35,12 @@
 extern "C" {
 #endif
 
+#if defined(__GNUC__)
+#define APOLLO_API __attribute__((visibility("default")))
+#else
+#define APOLLO_API
+#endif
+
 #define APOLLO_OK 0
 #define APOLLO_ERR_INVALID_ARG (-1) /* null pointer, non-finite scalar, bad enum, bad index */
 #define APOLLO_ERR_SHAPE (-2)       /* rows or cols < 1, or a side above 2^31 - 1 */
@@ -79,7 +85,7 @@ typedef struct {
  * Bytes of DEVICE workspace a context over `shapes[0..n_matrices)` needs (moments, scales,
  * partial sums, descriptor tables, tensor maps).  shapes, cfg, out: HOST.
  */
-int apollo_workspace_bytes(const apollo_shape* shapes, int32_t n_matrices, const apollo_config* cfg,
+APOLLO_API int apollo_workspace_bytes(const apollo_shape* shapes, int32_t n_matrices, const apollo_config* cfg,
                            size_t* out_bytes);
 
 /*
@@ -90,7 +96,7 @@ int apollo_workspace_bytes(const apollo_shape* shapes, int32_t n_matrices, const
  * apollo_step on that step's stream.  The matrix index in the list is the `matrix index`
  * word of the Philox counter.  Must be called with the target device current.
  */
-int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_matrices,
+APOLLO_API int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_matrices,
                   const apollo_config* cfg, void* d_workspace, size_t workspace_bytes);
 
 /*
@@ -101,13 +107,13 @@ int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_ma
  * (a cudaStream_t; NULL = the legacy default stream); no host synchronisation; advances
  * the step counter t.  Not thread-safe per context.
  */
-int apollo_step(apollo_ctx* ctx, void* const* d_W, const void* const* d_G, float lr, float wd,
+APOLLO_API int apollo_step(apollo_ctx* ctx, void* const* d_W, const void* const* d_G, float lr, float wd,
                 void* cuda_stream);
 
-int apollo_destroy(apollo_ctx* ctx);
+APOLLO_API int apollo_destroy(apollo_ctx* ctx);
 
 /* Number of steps taken so far (t of Algorithm 1).  out: HOST. */
-int apollo_step_count(const apollo_ctx* ctx, int64_t* out);
+APOLLO_API int apollo_step_count(const apollo_ctx* ctx, int64_t* out);
 
 /*
  * Observability (used by the tests).  All copies are asynchronous on `cuda_stream`.
@@ -116,22 +122,22 @@ int apollo_step_count(const apollo_ctx* ctx, int64_t* out);
  *                     norm before limiting, tensor-wise scale (tensor mode, else 0)}.
  * apollo_get_state:   d_M, d_V DEVICE, r x n floats each, row-major (channel index contiguous).
  */
-int apollo_get_scales(apollo_ctx* ctx, int32_t matrix, float* d_out, void* cuda_stream);
-int apollo_get_limiter(apollo_ctx* ctx, int32_t matrix, float* d_out, void* cuda_stream);
-int apollo_get_state(apollo_ctx* ctx, int32_t matrix, float* d_M, float* d_V, void* cuda_stream);
+APOLLO_API int apollo_get_scales(apollo_ctx* ctx, int32_t matrix, float* d_out, void* cuda_stream);
+APOLLO_API int apollo_get_limiter(apollo_ctx* ctx, int32_t matrix, float* d_out, void* cuda_stream);
+APOLLO_API int apollo_get_state(apollo_ctx* ctx, int32_t matrix, float* d_M, float* d_V, void* cuda_stream);
 
 /*
  * Optional capture of the fp32 update dW = -lr (alpha c s_j G_ij + wd W_ij) before it is
  * added to W and rounded (the quantity the parity bound is stated on).  d_dW: HOST array
  * of n_matrices DEVICE pointers (rows x cols floats each), or NULL to switch capture off.
  */
-int apollo_set_delta_out(apollo_ctx* ctx, float* const* d_dW);
+APOLLO_API int apollo_set_delta_out(apollo_ctx* ctx, float* const* d_dW);
 
 /*
  * Synchronises `cuda_stream` and returns the device status word: APOLLO_OK, or
  * APOLLO_ERR_TIMEOUT if a bounded wait inside a kernel expired since the last call.
  */
-int apollo_status(apollo_ctx* ctx, void* cuda_stream);
+APOLLO_API int apollo_status(apollo_ctx* ctx, void* cuda_stream);
 
 /*
  * The generator by itself (Algorithm 1, "P_t <- N_seed(0, 1/r)"), for tests.
@@ -141,18 +147,18 @@ int apollo_status(apollo_ctx* ctx, void* cuda_stream);
  *                       rounding to bfloat16 (P = d_out / sqrt(r)), exactly as the
  *                       projection kernels materialise them.
  */
-int apollo_philox_draws(uint64_t seed, uint32_t matrix, uint32_t epoch, int32_t r, int32_t m,
+APOLLO_API int apollo_philox_draws(uint64_t seed, uint32_t matrix, uint32_t epoch, int32_t r, int32_t m,
                         uint32_t* d_out, void* cuda_stream);
-int apollo_projection(uint64_t seed, uint32_t matrix, uint32_t epoch, int32_t r, int32_t m,
+APOLLO_API int apollo_projection(uint64_t seed, uint32_t matrix, uint32_t epoch, int32_t r, int32_t m,
                       float* d_out, void* cuda_stream);
 
 /* Which projection kernel a matrix was assigned: 0 streaming (rank 1), 1 CUDA cores, 2 tensor cores. */
-int apollo_get_path(const apollo_ctx* ctx, int32_t matrix, int32_t* out);
+APOLLO_API int apollo_get_path(const apollo_ctx* ctx, int32_t matrix, int32_t* out);
 
 /* Kernel launches issued by the last apollo_step (HOST counter). */
-int apollo_last_launches(const apollo_ctx* ctx, int32_t* out);
+APOLLO_API int apollo_last_launches(const apollo_ctx* ctx, int32_t* out);
 
-const char* apollo_strerror(int code);
+APOLLO_API const char* apollo_strerror(int code);
 
 #ifdef __cplusplus
 }

@@ -1,0 +1,421 @@
+// Host side of libapollo: validation, workspace planning, descriptor tables and the
+// launch sequence of one step (Algorithm 1): projection pass -> finalize -> update pass.
+#include "../../include/apollo.h"
+
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "apollo_internal.h"
+#include "kernels.h"
+
+using namespace apollo;
+
+namespace {
+
+constexpr size_t ALIGN = 256;
+inline size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
+
+struct MatPlan {
+    int32_t rows, cols, m, n, tall, path, slices, g2_slices, tiles_n, tiles_k;
+    int64_t proj_tiles, update_tiles;
+    size_t off_M, off_V, off_scal, off_s, off_part, off_g2, off_tmap;
+};
+
+struct Plan {
+    std::vector<MatPlan> mats;
+    size_t off_status, off_descs, off_prefix[4], off_tmaps, zero_begin, zero_end, total;
+    int64_t tiles[4];   // stream, simt, tensor, update
+};
+
+int validate_config(const apollo_config* cfg)
+{
+    if (!cfg) return APOLLO_ERR_INVALID_ARG;
+    if (cfg->rank < 1 || cfg->rank > APOLLO_MAX_RANK) return APOLLO_ERR_RANK;
+    if (cfg->mode != APOLLO_SCALE_CHANNEL && cfg->mode != APOLLO_SCALE_TENSOR) return APOLLO_ERR_INVALID_ARG;
+    if (cfg->dtype != APOLLO_DT_F32 && cfg->dtype != APOLLO_DT_BF16) return APOLLO_ERR_INVALID_ARG;
+    if (cfg->T < 1) return APOLLO_ERR_INVALID_ARG;
+    if (!std::isfinite(cfg->alpha) || !std::isfinite(cfg->gamma) || !std::isfinite(cfg->eps) || cfg->eps < 0.f)
+        return APOLLO_ERR_INVALID_ARG;
+    if (!(cfg->beta1 >= 0.f && cfg->beta1 <= 1.f) || !(cfg->beta2 >= 0.f && cfg->beta2 <= 1.f))
+        return APOLLO_ERR_INVALID_ARG;
+    if (cfg->bias_correction != 0 && cfg->bias_correction != 1) return APOLLO_ERR_INVALID_ARG;
+    if (cfg->bias_correction && (cfg->beta1 >= 1.f || cfg->beta2 >= 1.f)) return APOLLO_ERR_INVALID_ARG;
+    return APOLLO_OK;
+}
+
+int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cfg, Plan& plan)
+{
+    if (!shapes || n_mat < 1) return APOLLO_ERR_INVALID_ARG;
+    int rc = validate_config(cfg);
+    if (rc != APOLLO_OK) return rc;
+    plan.mats.resize(n_mat);
+    for (int t = 0; t < 4; ++t) plan.tiles[t] = 0;
+    const int r = cfg->rank;
+    for (int i = 0; i < n_mat; ++i) {
+        const int64_t rows = shapes[i].rows, cols = shapes[i].cols;
+        if (rows < 1 || cols < 1 || rows > INT32_MAX || cols > INT32_MAX) return APOLLO_ERR_SHAPE;
+        MatPlan& p = plan.mats[i];
+        p.rows = (int32_t)rows; p.cols = (int32_t)cols;
+        p.tall = rows > cols;
+        p.m = (int32_t)(p.tall ? cols : rows);
+        p.n = (int32_t)(p.tall ? rows : cols);
+        if (r > p.m) return APOLLO_ERR_RANK;
+        p.g2_slices = 0;
+        if (r == 1) {
+            p.path = PATH_STREAM;
+            if (!p.tall) {
+                p.tiles_n = (p.cols + STREAM_COLS - 1) / STREAM_COLS;
+                p.tiles_k = (p.rows + STREAM_ROWS - 1) / STREAM_ROWS;
+                p.slices = p.tiles_k;
+            } else {
+                p.tiles_n = (p.rows + STREAM_TALL_ROWS - 1) / STREAM_TALL_ROWS;
+                p.tiles_k = 1;
+                p.slices = 1;
+            }
+        } else if (tensor_path_supports(p.rows, p.cols, r, cfg->dtype) && !(cfg->flags & APOLLO_FLAG_NO_TENSOR_CORES)) {
+            p.path = PATH_TENSOR;
+            tensor_path_tiling(p.rows, p.cols, r, &p.tiles_n, &p.tiles_k);
+            p.slices = p.tiles_k;
+            p.g2_slices = 1;
+        } else {
+            p.path = PATH_SIMT;
+            p.tiles_n = (p.n + SIMT_BN - 1) / SIMT_BN;
+            p.tiles_k = (r + SIMT_BR - 1) / SIMT_BR;
+            p.slices = p.tiles_k;
+            p.g2_slices = 1;
+        }
+        p.proj_tiles = (int64_t)p.tiles_n * p.tiles_k;
+        p.update_tiles = (rows * cols + UPDATE_TILE - 1) / UPDATE_TILE;
+        plan.tiles[p.path] += p.proj_tiles;
+        plan.tiles[3] += p.update_tiles;
+    }
+    for (int t = 0; t < 4; ++t)
+        if (plan.tiles[t] > (int64_t)INT32_MAX - 1) return APOLLO_ERR_SHAPE;
+
+    size_t off = 0;
+    plan.off_status = off; off += ALIGN;
+    plan.off_descs = off; off = align_up(off + sizeof(MatDesc) * (size_t)n_mat);
+    for (int t = 0; t < 4; ++t) { plan.off_prefix[t] = off; off = align_up(off + sizeof(int) * ((size_t)n_mat + 1)); }
+    plan.off_tmaps = off; off = align_up(off + 128 * (size_t)n_mat);
+    plan.zero_begin = off;
+    for (int i = 0; i < n_mat; ++i) {
+        MatPlan& p = plan.mats[i];
+        const size_t state = sizeof(float) * (size_t)r * (size_t)p.n;
+        p.off_M = off; off = align_up(off + state);
+        p.off_V = off; off = align_up(off + state);
+        p.off_scal = off; off += ALIGN;     // scal[4] then prev at float index 8
+    }
+    plan.zero_end = off;
+    for (int i = 0; i < n_mat; ++i) {
+        MatPlan& p = plan.mats[i];
+        p.off_s = off; off = align_up(off + sizeof(float) * (size_t)p.n);
+        p.off_part = off; off = align_up(off + sizeof(float) * 2 * (size_t)p.slices * (size_t)p.n);
+        p.off_g2 = off; off = align_up(off + sizeof(float) * (size_t)(p.g2_slices > 0 ? p.g2_slices : 1) * (size_t)p.n);
+        p.off_tmap = plan.off_tmaps + 128 * (size_t)i;
+    }
+    plan.total = off;
+    return APOLLO_OK;
+}
+
+}  // namespace
+
+struct apollo_ctx {
+    apollo_config cfg;
+    int32_t n_mat;
+    Plan plan;
+    std::vector<MatDesc> h_descs;
+    std::vector<int> h_prefix[4];
+    char* ws;
+    MatDesc* d_descs;
+    int* d_prefix[4];
+    int32_t* d_status;
+    std::vector<float*> delta;
+    bool delta_on;
+    bool first;
+    bool descs_dirty;
+    int64_t t;
+    int device;
+    int sm_count;
+    int last_launches;
+};
+
+extern "C" {
+
+const char* apollo_strerror(int code)
+{
+    switch (code) {
+        case APOLLO_OK: return "ok";
+        case APOLLO_ERR_INVALID_ARG: return "invalid argument";
+        case APOLLO_ERR_SHAPE: return "unsupported shape";
+        case APOLLO_ERR_RANK: return "rank out of range for a matrix";
+        case APOLLO_ERR_ALIGN: return "device pointer not 16-byte aligned";
+        case APOLLO_ERR_WORKSPACE: return "workspace too small or misaligned";
+        case APOLLO_ERR_CUDA: return "CUDA call failed";
+        case APOLLO_ERR_TIMEOUT: return "bounded device-side wait expired";
+        case APOLLO_ERR_UNSUPPORTED: return "device is not an sm_100 GPU";
+        default: return "unknown error";
+    }
+}
+
+int apollo_workspace_bytes(const apollo_shape* shapes, int32_t n_matrices, const apollo_config* cfg,
+                           size_t* out_bytes)
+{
+    if (!out_bytes) return APOLLO_ERR_INVALID_ARG;
+    Plan plan;
+    const int rc = make_plan(shapes, n_matrices, cfg, plan);
+    if (rc != APOLLO_OK) return rc;
+    *out_bytes = plan.total;
+    return APOLLO_OK;
+}
+
+int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_matrices,
+                  const apollo_config* cfg, void* d_workspace, size_t workspace_bytes)
+{
+    if (!out_ctx) return APOLLO_ERR_INVALID_ARG;
+    *out_ctx = nullptr;
+    apollo_ctx* ctx = new (std::nothrow) apollo_ctx();
+    if (!ctx) return APOLLO_ERR_INVALID_ARG;
+    int rc = make_plan(shapes, n_matrices, cfg, ctx->plan);
+    if (rc != APOLLO_OK) { delete ctx; return rc; }
+    if (!d_workspace) { delete ctx; return APOLLO_ERR_INVALID_ARG; }
+    if (((uintptr_t)d_workspace % ALIGN) != 0 || workspace_bytes < ctx->plan.total) { delete ctx; return APOLLO_ERR_WORKSPACE; }
+
+    int device = 0, major = 0, sms = 0;
+    if (cudaGetDevice(&device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
+        cudaGetLastError();
+        delete ctx; return APOLLO_ERR_CUDA;
+    }
+    if (major != 10) { delete ctx; return APOLLO_ERR_UNSUPPORTED; }
+
+    ctx->cfg = *cfg;
+    ctx->n_mat = n_matrices;
+    ctx->ws = static_cast<char*>(d_workspace);
+    ctx->device = device;
+    ctx->sm_count = sms;
+    ctx->d_status = reinterpret_cast<int32_t*>(ctx->ws + ctx->plan.off_status);
+    ctx->d_descs = reinterpret_cast<MatDesc*>(ctx->ws + ctx->plan.off_descs);
+    ctx->h_descs.resize(n_matrices);
+    for (int t = 0; t < 4; ++t) {
+        ctx->d_prefix[t] = reinterpret_cast<int*>(ctx->ws + ctx->plan.off_prefix[t]);
+        ctx->h_prefix[t].assign(n_matrices + 1, 0);
+    }
+    for (int i = 0; i < n_matrices; ++i) {
+        const MatPlan& p = ctx->plan.mats[i];
+        MatDesc& d = ctx->h_descs[i];
+        std::memset(&d, 0, sizeof(d));
+        d.M = reinterpret_cast<float*>(ctx->ws + p.off_M);
+        d.V = reinterpret_cast<float*>(ctx->ws + p.off_V);
+        d.scal = reinterpret_cast<float*>(ctx->ws + p.off_scal);
+        d.prev = d.scal + 8;
+        d.s = reinterpret_cast<float*>(ctx->ws + p.off_s);
+        d.part = reinterpret_cast<float*>(ctx->ws + p.off_part);
+        d.g2 = reinterpret_cast<float*>(ctx->ws + p.off_g2);
+        d.rows = p.rows; d.cols = p.cols; d.m = p.m; d.n = p.n; d.tall = p.tall; d.path = p.path;
+        d.slices = p.slices; d.g2_slices = p.g2_slices; d.matrix_id = i;
+        d.tiles_n = p.tiles_n; d.tiles_k = p.tiles_k;
+        for (int t = 0; t < 3; ++t)
+            ctx->h_prefix[t][i + 1] = ctx->h_prefix[t][i] + (p.path == t ? (int)p.proj_tiles : 0);
+        ctx->h_prefix[3][i + 1] = ctx->h_prefix[3][i] + (int)p.update_tiles;
+    }
+    ctx->delta.assign(n_matrices, nullptr);
+    ctx->delta_on = false;
+    ctx->first = true;
+    ctx->descs_dirty = true;
+    ctx->t = 0;
+    ctx->last_launches = 0;
+    *out_ctx = ctx;
+    return APOLLO_OK;
+}
+
+int apollo_destroy(apollo_ctx* ctx)
+{
+    if (!ctx) return APOLLO_ERR_INVALID_ARG;
+    delete ctx;
+    return APOLLO_OK;
+}
+
+int apollo_step_count(const apollo_ctx* ctx, int64_t* out)
+{
+    if (!ctx || !out) return APOLLO_ERR_INVALID_ARG;
+    *out = ctx->t;
+    return APOLLO_OK;
+}
+
+int apollo_set_delta_out(apollo_ctx* ctx, float* const* d_dW)
+{
+    if (!ctx) return APOLLO_ERR_INVALID_ARG;
+    if (d_dW) {
+        for (int i = 0; i < ctx->n_mat; ++i) {
+            if (!d_dW[i]) return APOLLO_ERR_INVALID_ARG;
+            if ((uintptr_t)d_dW[i] % 16) return APOLLO_ERR_ALIGN;
+        }
+        for (int i = 0; i < ctx->n_mat; ++i) ctx->delta[i] = d_dW[i];
+        ctx->delta_on = true;
+    } else {
+        ctx->delta.assign(ctx->n_mat, nullptr);
+        ctx->delta_on = false;
+    }
+    ctx->descs_dirty = true;
+    return APOLLO_OK;
+}
+
+int apollo_step(apollo_ctx* ctx, void* const* d_W, const void* const* d_G, float lr, float wd,
+                void* cuda_stream)
+{
+    if (!ctx || !d_W || !d_G) return APOLLO_ERR_INVALID_ARG;
+    if (!std::isfinite(lr) || !std::isfinite(wd)) return APOLLO_ERR_INVALID_ARG;
+    for (int i = 0; i < ctx->n_mat; ++i) {
+        if (!d_W[i] || !d_G[i]) return APOLLO_ERR_INVALID_ARG;
+        if (((uintptr_t)d_W[i] % 16) || ((uintptr_t)d_G[i] % 16)) return APOLLO_ERR_ALIGN;
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const apollo_config& cfg = ctx->cfg;
+    const Plan& plan = ctx->plan;
+
+    if (ctx->first) {
+        if (cudaMemsetAsync(ctx->ws + plan.off_status, 0, ALIGN, stream) != cudaSuccess) return APOLLO_ERR_CUDA;
+        if (cudaMemsetAsync(ctx->ws + plan.zero_begin, 0, plan.zero_end - plan.zero_begin, stream) != cudaSuccess)
+            return APOLLO_ERR_CUDA;
+        for (int t = 0; t < 4; ++t)
+            if (cudaMemcpyAsync(ctx->d_prefix[t], ctx->h_prefix[t].data(), sizeof(int) * (ctx->n_mat + 1),
+                                cudaMemcpyHostToDevice, stream) != cudaSuccess)
+                return APOLLO_ERR_CUDA;
+    }
+    bool changed = ctx->descs_dirty;
+    for (int i = 0; i < ctx->n_mat; ++i) {
+        MatDesc& d = ctx->h_descs[i];
+        if (d.W != d_W[i] || d.G != d_G[i] || d.dW != ctx->delta[i]) {
+            d.W = d_W[i]; d.G = d_G[i]; d.dW = ctx->delta[i];
+            changed = true;
+        }
+    }
+    if (changed) {
+        const int rc = tensor_path_prepare(ctx->h_descs.data(), ctx->n_mat, cfg.rank,
+                                           ctx->ws + plan.off_tmaps, stream);
+        if (rc != APOLLO_OK) return rc;
+        if (cudaMemcpyAsync(ctx->d_descs, ctx->h_descs.data(), sizeof(MatDesc) * ctx->n_mat,
+                            cudaMemcpyHostToDevice, stream) != cudaSuccess)
+            return APOLLO_ERR_CUDA;
+        ctx->descs_dirty = false;
+    }
+
+    StepParams sp;
+    sp.key0 = (uint32_t)(cfg.seed & 0xFFFFFFFFull);
+    sp.key1 = (uint32_t)(cfg.seed >> 32);
+    sp.epoch = (uint32_t)(ctx->t / cfg.T);
+    sp.rank = cfg.rank; sp.mode = cfg.mode;
+    sp.inv_sqrt_r = (float)(1.0 / std::sqrt((double)cfg.rank));
+    sp.lr = lr; sp.wd = wd; sp.alpha = cfg.alpha; sp.gamma = cfg.gamma;
+    sp.beta1 = cfg.beta1; sp.beta2 = cfg.beta2; sp.eps = cfg.eps;
+    sp.inv_bc1 = 1.f; sp.inv_bc2 = 1.f;
+    if (cfg.bias_correction) {
+        sp.inv_bc1 = (float)(1.0 / (1.0 - std::pow((double)cfg.beta1, (double)(ctx->t + 1))));
+        sp.inv_bc2 = (float)(1.0 / (1.0 - std::pow((double)cfg.beta2, (double)(ctx->t + 1))));
+    }
+
+    int launches = 0;
+    if (plan.tiles[PATH_STREAM] > 0) {
+        launch_project_stream(cfg.dtype, ctx->d_descs, ctx->d_prefix[PATH_STREAM], ctx->n_mat,
+                              (int)plan.tiles[PATH_STREAM], sp, ctx->sm_count, stream);
+        ++launches;
+    }
+    if (plan.tiles[PATH_SIMT] > 0) {
+        launch_project_simt(cfg.dtype, ctx->d_descs, ctx->d_prefix[PATH_SIMT], ctx->n_mat,
+                            (int)plan.tiles[PATH_SIMT], sp, ctx->sm_count, stream);
+        ++launches;
+    }
+    if (plan.tiles[PATH_TENSOR] > 0) {
+        launches += launch_project_tensor(ctx->d_descs, ctx->d_prefix[PATH_TENSOR], ctx->n_mat,
+                                          (int)plan.tiles[PATH_TENSOR], sp, ctx->sm_count, ctx->d_status, stream);
+    }
+    launch_finalize(ctx->d_descs, ctx->n_mat, sp, stream);
+    ++launches;
+    launch_update(cfg.dtype, ctx->d_descs, ctx->d_prefix[3], ctx->n_mat, (int)plan.tiles[3], sp, ctx->sm_count, stream);
+    ++launches;
+    if (cudaGetLastError() != cudaSuccess) return APOLLO_ERR_CUDA;
+    ctx->first = false;
+    ctx->t += 1;
+    ctx->last_launches = launches;
+    return APOLLO_OK;
+}
+
+int apollo_get_scales(apollo_ctx* ctx, int32_t matrix, float* d_out, void* cuda_stream)
+{
+    if (!ctx || !d_out || matrix < 0 || matrix >= ctx->n_mat) return APOLLO_ERR_INVALID_ARG;
+    const MatDesc& d = ctx->h_descs[matrix];
+    return cudaMemcpyAsync(d_out, d.s, sizeof(float) * d.n, cudaMemcpyDeviceToDevice,
+                           static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? APOLLO_OK : APOLLO_ERR_CUDA;
+}
+
+int apollo_get_limiter(apollo_ctx* ctx, int32_t matrix, float* d_out, void* cuda_stream)
+{
+    if (!ctx || !d_out || matrix < 0 || matrix >= ctx->n_mat) return APOLLO_ERR_INVALID_ARG;
+    const MatDesc& d = ctx->h_descs[matrix];
+    return cudaMemcpyAsync(d_out, d.scal, sizeof(float) * 4, cudaMemcpyDeviceToDevice,
+                           static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? APOLLO_OK : APOLLO_ERR_CUDA;
+}
+
+int apollo_get_state(apollo_ctx* ctx, int32_t matrix, float* d_M, float* d_V, void* cuda_stream)
+{
+    if (!ctx || !d_M || !d_V || matrix < 0 || matrix >= ctx->n_mat) return APOLLO_ERR_INVALID_ARG;
+    const MatDesc& d = ctx->h_descs[matrix];
+    const size_t bytes = sizeof(float) * (size_t)ctx->cfg.rank * (size_t)d.n;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemcpyAsync(d_M, d.M, bytes, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) return APOLLO_ERR_CUDA;
+    if (cudaMemcpyAsync(d_V, d.V, bytes, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) return APOLLO_ERR_CUDA;
+    return APOLLO_OK;
+}
+
+int apollo_status(apollo_ctx* ctx, void* cuda_stream)
+{
+    if (!ctx) return APOLLO_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int32_t word = 0;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return APOLLO_ERR_CUDA;
+    if (ctx->first) return APOLLO_OK;   // nothing has run; the status word is not initialised yet
+    if (cudaMemcpy(&word, ctx->d_status, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return APOLLO_ERR_CUDA;
+    if (word != STATUS_OK) {
+        cudaMemset(ctx->d_status, 0, sizeof(word));
+        return APOLLO_ERR_TIMEOUT;
+    }
+    return APOLLO_OK;
+}
+
+int apollo_get_path(const apollo_ctx* ctx, int32_t matrix, int32_t* out)
+{
+    if (!ctx || !out || matrix < 0 || matrix >= ctx->n_mat) return APOLLO_ERR_INVALID_ARG;
+    *out = ctx->h_descs[matrix].path;
+    return APOLLO_OK;
+}
+
+int apollo_last_launches(const apollo_ctx* ctx, int32_t* out)
+{
+    if (!ctx || !out) return APOLLO_ERR_INVALID_ARG;
+    *out = ctx->last_launches;
+    return APOLLO_OK;
+}
+
+int apollo_philox_draws(uint64_t seed, uint32_t matrix, uint32_t epoch, int32_t r, int32_t m,
+                        uint32_t* d_out, void* cuda_stream)
+{
+    if (!d_out || r < 1 || m < 1) return APOLLO_ERR_INVALID_ARG;
+    if ((uintptr_t)d_out % 16) return APOLLO_ERR_ALIGN;
+    launch_philox_draws((uint32_t)(seed & 0xFFFFFFFFull), (uint32_t)(seed >> 32), matrix, epoch, r, m, d_out,
+                        static_cast<cudaStream_t>(cuda_stream));
+    return cudaGetLastError() == cudaSuccess ? APOLLO_OK : APOLLO_ERR_CUDA;
+}
+
+int apollo_projection(uint64_t seed, uint32_t matrix, uint32_t epoch, int32_t r, int32_t m,
+                      float* d_out, void* cuda_stream)
+{
+    if (!d_out || r < 1 || m < 1) return APOLLO_ERR_INVALID_ARG;
+    launch_projection((uint32_t)(seed & 0xFFFFFFFFull), (uint32_t)(seed >> 32), matrix, epoch, r, m, d_out,
+                      static_cast<cudaStream_t>(cuda_stream));
+    return cudaGetLastError() == cudaSuccess ? APOLLO_OK : APOLLO_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,62 @@
+// Structures shared by the host side of libapollo and its kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace apollo {
+
+// Which projection kernel serves a matrix.
+enum Path : int32_t {
+    PATH_STREAM = 0,  // rank 1: streaming matrix-vector pass, moments updated by the finalize kernel
+    PATH_SIMT = 1,    // any rank, any dtype, any pitch: CUDA-core tiles
+    PATH_TENSOR = 2,  // bf16, rank a multiple of 16, 16-byte row pitch: TMA + tcgen05 + TMEM
+};
+
+constexpr int STREAM_ROWS = 512;     // rows of a wide matrix one streaming tile covers
+constexpr int STREAM_COLS = 256;     // columns of a wide matrix one streaming tile covers
+constexpr int STREAM_TALL_ROWS = 64; // rows of a tall matrix one streaming tile covers
+constexpr int SIMT_BN = 64;          // channels per CUDA-core tile
+constexpr int SIMT_BR = 64;          // rows of R per CUDA-core tile
+constexpr int SIMT_BK = 32;          // contraction chunk of the CUDA-core tile
+constexpr int UPDATE_TILE = 16384;   // elements one tile of the update pass covers
+
+// Per-matrix record in device memory.  Pointers into the workspace are fixed at create
+// time; W, G and dW are refreshed whenever the caller passes different addresses.
+struct MatDesc {
+    void* W;
+    const void* G;
+    float* dW;        // optional fp32 capture of the update, or nullptr
+    float* M;         // r x n, row-major
+    float* V;         // r x n
+    float* s;         // n scales of the last step
+    float* part;      // projection partial sums, layout depends on the path (see kernels)
+    float* g2;        // squared column norms of G: g2_slices x n
+    float* scal;      // {norm after limiting, c, norm before limiting, tensor-wise s}
+    float* prev;      // previous limited norm (one float)
+    int32_t rows, cols;
+    int32_t m, n;     // m = min(rows, cols) = projected side; n = max = number of channels
+    int32_t tall;     // 1 if rows > cols: channels are the stored rows
+    int32_t path;
+    int32_t slices;   // number of partial slices in `part`
+    int32_t g2_slices;
+    int32_t matrix_id;
+    int32_t tiles_n;  // projection tiles along the channels
+    int32_t tiles_k;  // projection tiles along the other tiled axis (rows of G, or rows of R)
+    int32_t pad0;
+};
+
+struct StepParams {
+    uint32_t key0, key1;   // Philox key = seed
+    uint32_t epoch;        // floor(t / T)
+    int32_t rank, mode;
+    float inv_sqrt_r;
+    float lr, wd, alpha, gamma;
+    float beta1, beta2, eps;
+    float inv_bc1, inv_bc2;   // 1/(1-beta^t) with bias correction, else 1
+};
+
+// Device status word values.
+constexpr int32_t STATUS_OK = 0;
+constexpr int32_t STATUS_TIMEOUT = 1;
+
+}  // namespace apollo

@@ -1,0 +1,86 @@
+// Small device helpers shared by the kernels: tile lookup, typed 8-element loads and stores,
+// fixed-order block reductions.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "apollo_internal.h"
+
+namespace apollo {
+
+// prefix[i] = first tile of matrix i, prefix[n_mat] = total.  Returns the matrix that owns
+// `tile` (the last i with prefix[i] <= tile; matrices without tiles are skipped).
+__device__ __forceinline__ int find_matrix(const int* __restrict__ prefix, int n_mat, int tile)
+{
+    int lo = 0, hi = n_mat;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(prefix + mid) <= tile) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t bits16)
+{
+    return __uint_as_float(bits16 << 16);
+}
+
+__device__ __forceinline__ void unpack_bf16x8(const uint4& raw, float (&v)[8])
+{
+    v[0] = __uint_as_float(raw.x << 16); v[1] = __uint_as_float(raw.x & 0xFFFF0000u);
+    v[2] = __uint_as_float(raw.y << 16); v[3] = __uint_as_float(raw.y & 0xFFFF0000u);
+    v[4] = __uint_as_float(raw.z << 16); v[5] = __uint_as_float(raw.z & 0xFFFF0000u);
+    v[6] = __uint_as_float(raw.w << 16); v[7] = __uint_as_float(raw.w & 0xFFFF0000u);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    const __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&p);
+}
+
+__device__ __forceinline__ float load1(const float* p) { return __ldg(p); }
+__device__ __forceinline__ float load1(const __nv_bfloat16* p)
+{
+    return bf16_bits_to_float((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(p)));
+}
+
+// Eight consecutive elements starting at a 16-byte aligned address.
+__device__ __forceinline__ void load8_aligned(const float* p, float (&v)[8])
+{
+    const float4 a = __ldg(reinterpret_cast<const float4*>(p));
+    const float4 b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+__device__ __forceinline__ void load8_aligned(const __nv_bfloat16* p, float (&v)[8])
+{
+    const uint4 raw = __ldg(reinterpret_cast<const uint4*>(p));
+    unpack_bf16x8(raw, v);
+}
+
+// Up to eight consecutive elements with scalar loads; entries at or past `count` read as 0.
+template <typename T>
+__device__ __forceinline__ void load8_guarded(const T* p, int count, float (&v)[8])
+{
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[e] = e < count ? load1(p + e) : 0.0f;
+}
+
+// Sum of one double per thread over the block, in a fixed order (deterministic).
+// `scratch` holds at least 32 doubles; every thread gets the result.
+__device__ __forceinline__ double block_sum(double v, double* scratch)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int warps = (blockDim.x + 31) >> 5;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+    __syncthreads();
+    if (lane == 0) scratch[warp] = v;
+    __syncthreads();
+    double total = 0.0;
+    for (int w = 0; w < warps; ++w) total += scratch[w];
+    return total;
+}
+
+}  // namespace apollo

@@ -1,0 +1,30 @@
+// Host-callable launchers of the kernels (one grouped launch each over the parameter list).
+#pragma once
+#include "apollo_internal.h"
+
+namespace apollo {
+
+void launch_philox_draws(uint32_t key0, uint32_t key1, uint32_t matrix, uint32_t epoch, int r, int m,
+                         uint32_t* d_out, cudaStream_t stream);
+void launch_projection(uint32_t key0, uint32_t key1, uint32_t matrix, uint32_t epoch, int r, int m,
+                       float* d_out, cudaStream_t stream);
+void launch_project_stream(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int total_tiles,
+                           const StepParams& sp, int sm_count, cudaStream_t stream);
+void launch_project_simt(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int total_tiles,
+                         const StepParams& sp, int sm_count, cudaStream_t stream);
+void launch_finalize(const MatDesc* d_descs, int n_mat, const StepParams& sp, cudaStream_t stream);
+void launch_update(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int total_tiles,
+                   const StepParams& sp, int sm_count, cudaStream_t stream);
+
+
+// Tensor-core projection (TMA + tcgen05 + TMEM).
+bool tensor_path_supports(int rows, int cols, int rank, int dtype);
+void tensor_path_tiling(int rows, int cols, int rank, int32_t* tiles_n, int32_t* tiles_k);
+// Encodes the tensor maps of the matrices on the tensor path into the host copies and
+// queues their upload to `d_tmaps` (128 bytes per matrix).  Returns an APOLLO_* code.
+int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, void* d_tmaps, cudaStream_t stream);
+// Returns the number of launches issued.
+int launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_mat, int total_tiles,
+                          const StepParams& sp, int sm_count, int32_t* d_status, cudaStream_t stream);
+
+}  // namespace apollo
