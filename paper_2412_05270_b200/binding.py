@@ -1,0 +1,234 @@
+"""ctypes binding of libapollo.so: argument marshalling only.
+
+Every step of the optimizer runs inside the library's CUDA kernels; PyTorch supplies device
+memory and the stream.  There is no CPU fallback: if the shared library is missing the
+import of this module's symbols raises.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import torch
+
+_PKG = Path(__file__).resolve().parent
+LIB_PATH = _PKG / "libapollo.so"
+
+OK = 0
+ERR_INVALID_ARG, ERR_SHAPE, ERR_RANK, ERR_ALIGN, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED = (
+    -1, -2, -3, -4, -5, -6, -7, -8)
+SCALE_CHANNEL, SCALE_TENSOR = 0, 1
+DT_F32, DT_BF16 = 0, 1
+FLAG_NO_TENSOR_CORES = 1
+PATH_STREAM, PATH_SIMT, PATH_TENSOR = 0, 1, 2
+
+EXPORTS = [
+    "apollo_workspace_bytes", "apollo_create", "apollo_step", "apollo_destroy", "apollo_step_count",
+    "apollo_get_scales", "apollo_get_limiter", "apollo_get_state", "apollo_set_delta_out", "apollo_status",
+    "apollo_philox_draws", "apollo_projection", "apollo_get_path", "apollo_last_launches", "apollo_strerror",
+]
+
+
+class ApolloError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {strerror(code)} ({code})")
+        self.code = code
+
+
+class Shape(ctypes.Structure):
+    _fields_ = [("rows", ctypes.c_int64), ("cols", ctypes.c_int64)]
+
+
+class Config(ctypes.Structure):
+    _fields_ = [
+        ("rank", ctypes.c_int32), ("mode", ctypes.c_int32), ("dtype", ctypes.c_int32), ("T", ctypes.c_int32),
+        ("seed", ctypes.c_uint64),
+        ("alpha", ctypes.c_float), ("gamma", ctypes.c_float),
+        ("beta1", ctypes.c_float), ("beta2", ctypes.c_float), ("eps", ctypes.c_float),
+        ("bias_correction", ctypes.c_int32), ("flags", ctypes.c_uint32),
+    ]
+
+
+_lib = None
+
+
+def load():
+    """Load libapollo.so; raises if it has not been built (there is no fallback)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not LIB_PATH.exists():
+        raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2412_05270_b200.build` (nvcc, sm_100a)")
+    lib = ctypes.CDLL(str(LIB_PATH))
+    vp, i32, u32, u64, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint32, ctypes.c_uint64, ctypes.c_float
+    lib.apollo_workspace_bytes.argtypes = [ctypes.POINTER(Shape), i32, ctypes.POINTER(Config),
+                                           ctypes.POINTER(ctypes.c_size_t)]
+    lib.apollo_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(Shape), i32, ctypes.POINTER(Config), vp,
+                                  ctypes.c_size_t]
+    lib.apollo_step.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), f32, f32, vp]
+    lib.apollo_destroy.argtypes = [vp]
+    lib.apollo_step_count.argtypes = [vp, ctypes.POINTER(ctypes.c_int64)]
+    lib.apollo_get_scales.argtypes = [vp, i32, vp, vp]
+    lib.apollo_get_limiter.argtypes = [vp, i32, vp, vp]
+    lib.apollo_get_state.argtypes = [vp, i32, vp, vp, vp]
+    lib.apollo_set_delta_out.argtypes = [vp, ctypes.POINTER(vp)]
+    lib.apollo_status.argtypes = [vp, vp]
+    lib.apollo_philox_draws.argtypes = [u64, u32, u32, i32, i32, vp, vp]
+    lib.apollo_projection.argtypes = [u64, u32, u32, i32, i32, vp, vp]
+    lib.apollo_get_path.argtypes = [vp, i32, ctypes.POINTER(i32)]
+    lib.apollo_last_launches.argtypes = [vp, ctypes.POINTER(i32)]
+    lib.apollo_strerror.argtypes = [ctypes.c_int]
+    lib.apollo_strerror.restype = ctypes.c_char_p
+    for name in EXPORTS:
+        if name != "apollo_strerror":
+            getattr(lib, name).restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def strerror(code: int) -> str:
+    return load().apollo_strerror(code).decode()
+
+
+def _check(code: int, what: str):
+    if code != OK:
+        raise ApolloError(code, what)
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream
+
+
+def _shape_array(shapes):
+    arr = (Shape * len(shapes))()
+    for i, (r, c) in enumerate(shapes):
+        arr[i].rows, arr[i].cols = int(r), int(c)
+    return arr
+
+
+def make_config(rank, mode=SCALE_CHANNEL, dtype=DT_BF16, T=200, seed=0, alpha=1.0, gamma=1.01,
+                beta1=0.9, beta2=0.999, eps=1e-8, bias_correction=False, flags=0) -> Config:
+    return Config(int(rank), int(mode), int(dtype), int(T), int(seed), float(alpha), float(gamma),
+                  float(beta1), float(beta2), float(eps), int(bool(bias_correction)), int(flags))
+
+
+def workspace_bytes(shapes, cfg: Config) -> int:
+    out = ctypes.c_size_t(0)
+    _check(load().apollo_workspace_bytes(_shape_array(shapes), len(shapes), ctypes.byref(cfg), ctypes.byref(out)),
+           "apollo_workspace_bytes")
+    return out.value
+
+
+def philox_draws(seed: int, matrix: int, epoch: int, r: int, m: int, stream=None) -> torch.Tensor:
+    out = torch.empty((r, (m + 3) // 4, 4), dtype=torch.int32, device="cuda")
+    _check(load().apollo_philox_draws(seed, matrix, epoch, r, m, out.data_ptr(), _stream_ptr(stream)),
+           "apollo_philox_draws")
+    return out
+
+
+def projection(seed: int, matrix: int, epoch: int, r: int, m: int, stream=None) -> torch.Tensor:
+    out = torch.empty((r, m), dtype=torch.float32, device="cuda")
+    _check(load().apollo_projection(seed, matrix, epoch, r, m, out.data_ptr(), _stream_ptr(stream)),
+           "apollo_projection")
+    return out
+
+
+class Apollo:
+    """apollo_create / apollo_step over a list of CUDA tensors (same dtype, 2-D, contiguous)."""
+
+    def __init__(self, shapes, cfg: Config, device="cuda"):
+        self.lib = load()
+        self.shapes = [(int(r), int(c)) for r, c in shapes]
+        self.cfg = cfg
+        self.device = torch.device(device)
+        nbytes = workspace_bytes(self.shapes, cfg)
+        with torch.cuda.device(self.device):
+            self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+            base = self.workspace.data_ptr()
+            self._ws_ptr = (base + 255) // 256 * 256
+            ctx = ctypes.c_void_p()
+            _check(self.lib.apollo_create(ctypes.byref(ctx), _shape_array(self.shapes), len(self.shapes),
+                                          ctypes.byref(cfg), self._ws_ptr, nbytes), "apollo_create")
+        self.ctx = ctx
+        self._delta = None
+        self._w_arr = (ctypes.c_void_p * len(self.shapes))()
+        self._g_arr = (ctypes.c_void_p * len(self.shapes))()
+
+    def close(self):
+        if getattr(self, "ctx", None):
+            self.lib.apollo_destroy(self.ctx)
+            self.ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check_tensors(self, Ws, Gs):
+        want = torch.bfloat16 if self.cfg.dtype == DT_BF16 else torch.float32
+        if len(Ws) != len(self.shapes) or len(Gs) != len(self.shapes):
+            raise ValueError("parameter list length differs from the context's")
+        for w, g, shp in zip(Ws, Gs, self.shapes):
+            for x in (w, g):
+                if not x.is_cuda or x.dtype != want or tuple(x.shape) != shp or not x.is_contiguous():
+                    raise ValueError("tensors must be contiguous CUDA tensors of the context's dtype and shapes")
+
+    def step(self, Ws, Gs, lr: float, wd: float = 0.0, stream=None, check: bool = True):
+        if check:
+            self._check_tensors(Ws, Gs)
+        for i, (w, g) in enumerate(zip(Ws, Gs)):
+            self._w_arr[i] = w.data_ptr()
+            self._g_arr[i] = g.data_ptr()
+        _check(self.lib.apollo_step(self.ctx, self._w_arr, self._g_arr, lr, wd, _stream_ptr(stream)), "apollo_step")
+
+    def set_delta_out(self, deltas):
+        """deltas: list of float32 CUDA tensors shaped like the weights, or None."""
+        if deltas is None:
+            _check(self.lib.apollo_set_delta_out(self.ctx, None), "apollo_set_delta_out")
+            self._delta = None
+            return
+        arr = (ctypes.c_void_p * len(self.shapes))()
+        for i, d in enumerate(deltas):
+            assert d.is_cuda and d.dtype == torch.float32 and tuple(d.shape) == self.shapes[i] and d.is_contiguous()
+            arr[i] = d.data_ptr()
+        _check(self.lib.apollo_set_delta_out(self.ctx, arr), "apollo_set_delta_out")
+        self._delta = deltas
+
+    def scales(self, mat: int, stream=None) -> torch.Tensor:
+        out = torch.empty(max(self.shapes[mat]), dtype=torch.float32, device=self.device)
+        _check(self.lib.apollo_get_scales(self.ctx, mat, out.data_ptr(), _stream_ptr(stream)), "apollo_get_scales")
+        return out
+
+    def limiter(self, mat: int, stream=None) -> torch.Tensor:
+        out = torch.empty(4, dtype=torch.float32, device=self.device)
+        _check(self.lib.apollo_get_limiter(self.ctx, mat, out.data_ptr(), _stream_ptr(stream)), "apollo_get_limiter")
+        return out
+
+    def state(self, mat: int, stream=None):
+        n = max(self.shapes[mat])
+        M = torch.empty((self.cfg.rank, n), dtype=torch.float32, device=self.device)
+        V = torch.empty_like(M)
+        _check(self.lib.apollo_get_state(self.ctx, mat, M.data_ptr(), V.data_ptr(), _stream_ptr(stream)),
+               "apollo_get_state")
+        return M, V
+
+    def status(self, stream=None) -> int:
+        return self.lib.apollo_status(self.ctx, _stream_ptr(stream))
+
+    def path(self, mat: int) -> int:
+        out = ctypes.c_int32(-1)
+        _check(self.lib.apollo_get_path(self.ctx, mat, ctypes.byref(out)), "apollo_get_path")
+        return out.value
+
+    def step_count(self) -> int:
+        out = ctypes.c_int64(0)
+        _check(self.lib.apollo_step_count(self.ctx, ctypes.byref(out)), "apollo_step_count")
+        return out.value
+
+    def last_launches(self) -> int:
+        out = ctypes.c_int32(0)
+        _check(self.lib.apollo_last_launches(self.ctx, ctypes.byref(out)), "apollo_last_launches")
+        return out.value

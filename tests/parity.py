@@ -1,0 +1,86 @@
+"""Shared driver of the parity tests: runs the CUDA library and the CPU oracle on the same
+seeded inputs and compares them under the stated bounds.
+
+Bounds: Philox draws bit-exact; per element |dW_gpu - dW_oracle| <= 2e-3 max|dW_oracle| + 1e-6;
+scales within 1e-3 relative; stored W equal to round(W_old + dW_gpu) exactly.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2412_05270_b200 import binding as B
+from paper_2412_05270_b200 import workloads as WL
+
+DW_REL, DW_ABS, SCALE_REL = 2e-3, 1e-6, 1e-3
+
+
+def config_of(wl: WL.Workload, flags=0, bias_correction=False) -> B.Config:
+    return B.make_config(rank=wl.rank, mode=B.SCALE_TENSOR if wl.mode == "tensor" else B.SCALE_CHANNEL,
+                         dtype=B.DT_BF16 if wl.dtype == "bf16" else B.DT_F32, T=wl.T, seed=wl.seed,
+                         alpha=wl.alpha, gamma=wl.gamma, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps,
+                         bias_correction=bias_correction, flags=flags)
+
+
+def oracle_of(wl: WL.Workload, mats=None, bias_correction=False):
+    mats = range(len(wl.shapes)) if mats is None else mats
+    return {i: oracle.MatrixOracle(wl.shapes[i][0], wl.shapes[i][1], rank=wl.rank,
+                                   mode=oracle.MODE_TENSOR if wl.mode == "tensor" else oracle.MODE_CHANNEL,
+                                   dtype=oracle.DT_BF16 if wl.dtype == "bf16" else oracle.DT_F32,
+                                   seed=wl.seed, matrix_id=i, T=wl.T, alpha=wl.alpha, gamma=wl.gamma,
+                                   beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps, bias_correction=bias_correction,
+                                   p_round_bf16=True) for i in mats}
+
+
+def run_parity(wl: WL.Workload, steps=None, flags=0, bias_correction=False, check_mats=None, expect_path=None,
+               grad_fn=None):
+    """Steps the whole list on the GPU and the matrices in `check_mats` on the oracle."""
+    steps = wl.steps if steps is None else steps
+    n = len(wl.shapes)
+    check_mats = list(range(n)) if check_mats is None else list(check_mats)
+    dev = torch.device("cuda")
+    opt = B.Apollo(wl.shapes, config_of(wl, flags, bias_correction))
+    if expect_path is not None:
+        for i in check_mats:
+            assert opt.path(i) == expect_path, (i, opt.path(i))
+    Wc = [WL.make_weight(wl, i) for i in range(n)]
+    Wg = [w.to(dev) for w in Wc]
+    deltas = [torch.zeros(s, dtype=torch.float32, device=dev) for s in wl.shapes]
+    opt.set_delta_out(deltas)
+    orc = oracle_of(wl, check_mats, bias_correction)
+    Wo = {i: Wc[i].float().numpy() for i in check_mats}
+    worst = {"dw": 0.0, "s": 0.0}
+    for t in range(steps):
+        Gc = [(grad_fn or WL.make_grad)(wl, i, t) for i in range(n)]
+        Gg = [g.to(dev) for g in Gc]
+        W_before = {i: Wg[i].clone() for i in check_mats}
+        opt.step(Wg, Gg, wl.lr, wl.wd)
+        assert opt.status() == B.OK
+        for i in check_mats:
+            res = orc[i].step(Wo[i], Gc[i].float().numpy(), wl.lr, wl.wd)
+            dw_gpu = deltas[i].cpu().numpy().astype(np.float64)
+            bound = DW_REL * np.max(np.abs(res.dW)) + DW_ABS
+            err = np.max(np.abs(dw_gpu - res.dW))
+            assert err <= bound, f"step {t} matrix {i}: |dW error| {err:.3e} > {bound:.3e}"
+            worst["dw"] = max(worst["dw"], err / bound)
+            s_gpu = opt.scales(i).cpu().numpy().astype(np.float64)
+            ok = np.abs(s_gpu - res.s) <= SCALE_REL * np.abs(res.s) + 1e-30
+            assert ok.all(), f"step {t} matrix {i}: scale rel error {np.max(np.abs(s_gpu - res.s) / (np.abs(res.s) + 1e-30)):.3e}"
+            worst["s"] = max(worst["s"], float(np.max(np.abs(s_gpu - res.s) / (np.abs(res.s) + 1e-30))))
+            lim = opt.limiter(i).cpu().numpy()
+            assert abs(lim[0] - res.norm) <= 2e-3 * res.norm + 1e-30
+            assert abs(lim[1] - res.c) <= 2e-3
+            # the store is exactly round(W_old + dW_gpu) in the weight's dtype
+            want = (W_before[i].float() + deltas[i]).to(Wg[i].dtype)
+            assert torch.equal(want, Wg[i]), f"step {t} matrix {i}: stored W is not round(W_old + dW)"
+            # and agrees with the oracle's store up to one rounding step of the dtype
+            w_gpu = Wg[i].float().cpu().numpy()
+            tol = 2.0 ** -7 * np.abs(res.W) + 1e-6 if wl.dtype == "bf16" else 1e-6 * np.abs(res.W) + bound
+            assert np.all(np.abs(w_gpu - res.W) <= tol)
+            Wo[i] = res.W
+            # keep the two weight trajectories identical so that errors do not compound through wd
+            Wg[i].copy_(torch.from_numpy(res.W).to(Wg[i].dtype))
+    assert opt.step_count() == steps
+    opt.close()
+    return worst

@@ -1,0 +1,33 @@
+"""GPU generator against the oracle: Philox words bit-exact, normals equal after the
+bfloat16 rounding except where the fast logarithm / sine move a value across a rounding
+boundary."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2412_05270_b200 import binding as B
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("r,m", [(1, 4), (3, 10), (128, 512), (17, 4097)])
+def test_philox_words_bit_exact(r, m):
+    seed = 0xDEADBEEF12345678
+    got = B.philox_draws(seed, 7, 3, r, m).cpu().numpy().view(np.uint32)
+    want = oracle.philox_draws(seed, 7, 3, r, m)
+    assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("r,m", [(1, 5), (64, 1024), (256, 4096)])
+def test_projection_entries_match_the_oracle(r, m):
+    got = B.projection(42, 2, 1, r, m).cpu().numpy().astype(np.float64)
+    z = oracle.standard_normals(42, 2, 1, r, m)
+    want = np.vectorize(oracle.round_bf16)(z) if z.size < 5000 else \
+        torch.from_numpy(z).float().to(torch.bfloat16).double().numpy()
+    # every entry within the fast-math error of the unrounded normal plus half a bf16 step
+    assert np.all(np.abs(got - z) <= 2.0 ** -8 * np.abs(z) + 1e-3)
+    assert np.mean(got == want) > 0.995
+    # differing entries are one rounding step apart (or tiny values near zero radius)
+    diff = got != want
+    assert np.all(np.abs(got[diff] - want[diff]) <= 2.0 ** -7 * np.abs(want[diff]) + 1e-3)

@@ -1,0 +1,121 @@
+"""Parity of the CUDA step with the CPU oracle, element by element, through the C ABI."""
+import dataclasses
+import math
+
+import pytest
+import torch
+
+from paper_2412_05270_b200 import binding as B
+from paper_2412_05270_b200 import workloads as WL
+from parity import run_parity
+
+pytestmark = pytest.mark.gpu
+
+
+def _wl(shapes, rank, mode="channel", dtype="bf16", T=3, steps=6, **kw):
+    return WL.Workload("case", list(shapes), dtype, rank, mode, T=T, steps=steps, **kw)
+
+
+SMALL = [(5, 7), (7, 5), (33, 130), (130, 33), (64, 64), (100, 257), (257, 100), (1, 9), (9, 1)]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("mode", ["channel", "tensor"])
+def test_rank1_streaming_path_small_shapes(dtype, mode):
+    wl = _wl(SMALL, 1, mode=mode, dtype=dtype, alpha=math.sqrt(128.0) if mode == "tensor" else 1.0, wd=0.05)
+    run_parity(wl, expect_path=B.PATH_STREAM)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("rank,mode", [(2, "channel"), (5, "channel"), (5, "tensor")])
+def test_cuda_core_path_small_shapes(dtype, rank, mode):
+    shapes = [s for s in SMALL if min(s) >= rank]
+    wl = _wl(shapes, rank, mode=mode, dtype=dtype, wd=0.05)
+    run_parity(wl, flags=B.FLAG_NO_TENSOR_CORES, expect_path=B.PATH_SIMT)
+
+
+def test_cuda_core_path_rank_spanning_row_blocks_and_ragged_tiles():
+    wl = _wl([(200, 333), (333, 200), (130, 130)], 130, dtype="bf16", steps=4, T=2)
+    run_parity(wl, flags=B.FLAG_NO_TENSOR_CORES, expect_path=B.PATH_SIMT)
+
+
+def test_streaming_path_spanning_row_blocks_and_column_tiles():
+    # wide: > 512 rows and > 256 columns with ragged tails; tall: > 2048 columns of P per chunk
+    wl = _wl([(1100, 1300), (1300, 1100), (600, 2600), (70, 3000), (3000, 2100)], 1, mode="tensor", dtype="bf16",
+             steps=3, alpha=math.sqrt(128.0))
+    run_parity(wl, expect_path=B.PATH_STREAM)
+    wl = _wl([(1029, 1301), (1301, 1029)], 1, mode="channel", dtype="f32", steps=3)   # unaligned pitch
+    run_parity(wl, expect_path=B.PATH_STREAM)
+
+
+def test_bias_correction_variant():
+    wl = _wl([(33, 130), (130, 33)], 4, dtype="f32", steps=4)
+    run_parity(wl, flags=B.FLAG_NO_TENSOR_CORES, bias_correction=True)
+    wl = _wl([(33, 130), (130, 33)], 1, dtype="bf16", mode="tensor", steps=4)
+    run_parity(wl, bias_correction=True)
+
+
+def test_limiter_engages_on_growing_gradients():
+    wl = _wl([(40, 90), (90, 40)], 4, dtype="f32", steps=8, T=4)
+
+    def grad(w, i, t):
+        return WL.make_grad(w, i, t) * (1.5 ** t)
+    worst = run_parity(wl, flags=B.FLAG_NO_TENSOR_CORES, grad_fn=grad)
+    assert worst["dw"] <= 1.0
+
+
+def test_config_single_matrix_fp32_rank128():
+    run_parity(WL.workload("single"))
+
+
+def test_config_llama60m_mini_all_matrices():
+    wl = WL.workload("llama60m_mini")
+    run_parity(wl, steps=20, check_mats=[0, 3, 4, 6, 55], expect_path=B.PATH_STREAM)
+
+
+def test_zero_gradient_and_zero_lr():
+    dev = torch.device("cuda")
+    shapes = [(33, 130)]
+    opt = B.Apollo(shapes, B.make_config(rank=4, dtype=B.DT_F32, flags=B.FLAG_NO_TENSOR_CORES))
+    W = torch.randn(33, 130, device=dev) * 0.02
+    W0 = W.clone()
+    G = torch.zeros_like(W)
+    opt.step([W], [G], 0.1, 0.5)
+    torch.cuda.synchronize()
+    assert torch.all(opt.scales(0) == 0)
+    assert torch.allclose(W, W0 * 0.95, rtol=1e-6, atol=0)
+    G = torch.randn_like(W) * 1e-3
+    W1 = W.clone()
+    opt.step([W], [G], 0.0, 0.3)
+    torch.cuda.synchronize()
+    assert torch.equal(W, W1)
+    M, V = opt.state(0)
+    assert M.abs().sum() > 0 and V.abs().sum() > 0
+    opt.close()
+
+
+def test_runs_are_bitwise_reproducible():
+    wl = _wl([(200, 333), (333, 200)], 8, dtype="bf16", steps=3)
+    outs = []
+    for _ in range(2):
+        opt = B.Apollo(wl.shapes, B.make_config(rank=8, dtype=B.DT_BF16, T=2, seed=9))
+        Ws = [WL.make_weight(wl, i).cuda() for i in range(2)]
+        for t in range(3):
+            opt.step(Ws, [WL.make_grad(wl, i, t).cuda() for i in range(2)], 1e-2, 0.01)
+        torch.cuda.synchronize()
+        outs.append([w.clone() for w in Ws])
+        opt.close()
+    assert all(torch.equal(a, b) for a, b in zip(*outs))
+
+
+def test_misaligned_and_null_pointers_are_rejected_before_any_launch():
+    dev = torch.device("cuda")
+    opt = B.Apollo([(16, 32)], B.make_config(rank=2, dtype=B.DT_F32))
+    buf = torch.zeros(16 * 32 + 4, device=dev)
+    W = buf[1:1 + 512].view(16, 32)         # 4-byte offset: not 16-byte aligned
+    G = torch.zeros(16, 32, device=dev)
+    with pytest.raises(B.ApolloError) as e:
+        opt.step([W], [G], 0.1, check=False)
+    assert e.value.code == B.ERR_ALIGN
+    assert opt.step_count() == 0
+    opt.close()
