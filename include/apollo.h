@@ -143,9 +143,9 @@ APOLLO_API int apollo_status(apollo_ctx* ctx, void* cuda_stream);
  * The generator by itself (Algorithm 1, "P_t <- N_seed(0, 1/r)"), for tests.
  * apollo_philox_draws:  d_out DEVICE, r x ceil(m/4) x 4 uint32: the raw Philox4x32-10
  *                       words for counter (q, k, matrix, epoch), key = seed.
- * apollo_projection:    d_out DEVICE, r x m floats: the standard normals behind P after
- *                       rounding to bfloat16 (P = d_out / sqrt(r)), exactly as the
- *                       projection kernels materialise them.
+ * apollo_projection:    d_out DEVICE, r x m floats: the standard normals Z behind P
+ *                       (P = Z / sqrt(r)) in fp32, as the CUDA-core kernels use them; the
+ *                       tensor-core kernel rounds the same values to bfloat16 operands.
  */
 APOLLO_API int apollo_philox_draws(uint64_t seed, uint32_t matrix, uint32_t epoch, int32_t r, int32_t m,
                         uint32_t* d_out, void* cuda_stream);

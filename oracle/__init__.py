@@ -87,8 +87,8 @@ def standard_normals(seed: int, matrix_id: int, epoch: int, r: int, m: int) -> n
     return out
 
 
-def projection(seed: int, matrix_id: int, epoch: int, r: int, m: int, round_bf16: bool = True) -> np.ndarray:
-    """P (r x m), entries N(0, 1/r); bf16-rounded standard normals divided by sqrt(r)."""
+def projection(seed: int, matrix_id: int, epoch: int, r: int, m: int, round_bf16: bool = False) -> np.ndarray:
+    """P (r x m), entries N(0, 1/r): standard normals divided by sqrt(r) (optionally bf16-rounded first)."""
     out = np.zeros((r, m), dtype=np.float64)
     lib().oracle_projection(ctypes.c_uint64(seed), ctypes.c_uint32(matrix_id), ctypes.c_uint32(epoch),
                             ctypes.c_int32(r), ctypes.c_int32(m), ctypes.c_int32(int(round_bf16)),
@@ -125,7 +125,7 @@ class MatrixOracle:
     def __init__(self, rows: int, cols: int, rank: int, mode: int = MODE_CHANNEL, dtype: int = DT_F32,
                  seed: int = 0, matrix_id: int = 0, T: int = 200, alpha: float = 1.0, gamma: float = 1.01,
                  beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
-                 bias_correction: bool = False, p_round_bf16: bool = True):
+                 bias_correction: bool = False, p_round_bf16: bool = False):
         self.rows, self.cols = int(rows), int(cols)
         self.m, self.n = min(rows, cols), max(rows, cols)
         self.cfg = _Config(rank, mode, dtype, int(bias_correction), alpha, gamma, beta1, beta2, eps)

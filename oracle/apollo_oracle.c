@@ -127,7 +127,7 @@ void oracle_standard_normals(uint64_t seed, uint32_t matrix_id, uint32_t epoch,
 /*
  * P = Z / sqrt(r), entries N(0, 1/r) (Algorithm 1; Appendix notation "P_ij ~ N(0,1/r)").
  * With round_bf16 != 0 the standard normal is first rounded to bfloat16, which is the
- * precision the library keeps P in; the 1/sqrt(r) factor is applied after the rounding.
+ * precision the library keeps P in; the 1/sqrt(r) factor is applied after the rounding (the default is no rounding).
  */
 void oracle_projection(uint64_t seed, uint32_t matrix_id, uint32_t epoch,
                        int32_t r, int32_t m, int32_t round_bf16, double* P)

@@ -40,7 +40,7 @@ __global__ void projection_kernel(uint32_t key0, uint32_t key1, uint32_t matrix,
         const float zz[4] = { z.x, z.y, z.z, z.w };
         for (int e = 0; e < 4; ++e) {
             const int i = 4 * (int)q + e;
-            if (i < m) out[(int64_t)k * m + i] = round_to_bf16(zz[e]);
+            if (i < m) out[(int64_t)k * m + i] = zz[e];
         }
     }
 }
@@ -99,8 +99,8 @@ project_stream_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
             for (int q = tid; q < STREAM_ROWS / 4; q += STREAM_THREADS) {
                 const float4 z = normal_quad((uint32_t)(i0 / 4 + q), 0u, (uint32_t)d.matrix_id, sp.epoch,
                                              sp.key0, sp.key1);
-                Ps[4 * q + 0] = round_to_bf16(z.x); Ps[4 * q + 1] = round_to_bf16(z.y);
-                Ps[4 * q + 2] = round_to_bf16(z.z); Ps[4 * q + 3] = round_to_bf16(z.w);
+                Ps[4 * q + 0] = z.x; Ps[4 * q + 1] = z.y;
+                Ps[4 * q + 2] = z.z; Ps[4 * q + 3] = z.w;
             }
             __syncthreads();
             const int j0 = tn * STREAM_COLS + lane * 8;
@@ -141,8 +141,8 @@ project_stream_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                 for (int q = tid; q < STREAM_TALL_CHUNK / 4; q += STREAM_THREADS) {
                     const float4 z = normal_quad((uint32_t)(c0 / 4 + q), 0u, (uint32_t)d.matrix_id, sp.epoch,
                                                  sp.key0, sp.key1);
-                    Ps[4 * q + 0] = round_to_bf16(z.x); Ps[4 * q + 1] = round_to_bf16(z.y);
-                    Ps[4 * q + 2] = round_to_bf16(z.z); Ps[4 * q + 3] = round_to_bf16(z.w);
+                    Ps[4 * q + 0] = z.x; Ps[4 * q + 1] = z.y;
+                    Ps[4 * q + 2] = z.z; Ps[4 * q + 3] = z.w;
                 }
                 __syncthreads();
                 const int chunk = min(STREAM_TALL_CHUNK, cols - c0);
@@ -225,8 +225,8 @@ project_simt_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                 if (k0 + row < r)
                     z = normal_quad((uint32_t)(i0 / 4 + q), (uint32_t)(k0 + row), (uint32_t)d.matrix_id, sp.epoch,
                                     sp.key0, sp.key1);
-                Ps[4 * q + 0][row] = round_to_bf16(z.x); Ps[4 * q + 1][row] = round_to_bf16(z.y);
-                Ps[4 * q + 2][row] = round_to_bf16(z.z); Ps[4 * q + 3][row] = round_to_bf16(z.w);
+                Ps[4 * q + 0][row] = z.x; Ps[4 * q + 1][row] = z.y;
+                Ps[4 * q + 2][row] = z.z; Ps[4 * q + 3][row] = z.w;
             }
             // G chunk: Gs[kk][jj] = Gv[i0+kk][j0+jj], zero outside the matrix
             if (!d.tall) {

@@ -30,7 +30,7 @@ def oracle_of(wl: WL.Workload, mats=None, bias_correction=False):
                                    dtype=oracle.DT_BF16 if wl.dtype == "bf16" else oracle.DT_F32,
                                    seed=wl.seed, matrix_id=i, T=wl.T, alpha=wl.alpha, gamma=wl.gamma,
                                    beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps, bias_correction=bias_correction,
-                                   p_round_bf16=True) for i in mats}
+                                   p_round_bf16=False) for i in mats}
 
 
 def run_parity(wl: WL.Workload, steps=None, flags=0, bias_correction=False, check_mats=None, expect_path=None,

@@ -23,11 +23,8 @@ def test_philox_words_bit_exact(r, m):
 def test_projection_entries_match_the_oracle(r, m):
     got = B.projection(42, 2, 1, r, m).cpu().numpy().astype(np.float64)
     z = oracle.standard_normals(42, 2, 1, r, m)
-    want = np.vectorize(oracle.round_bf16)(z) if z.size < 5000 else \
-        torch.from_numpy(z).float().to(torch.bfloat16).double().numpy()
-    # every entry within the fast-math error of the unrounded normal plus half a bf16 step
-    assert np.all(np.abs(got - z) <= 2.0 ** -8 * np.abs(z) + 1e-3)
-    assert np.mean(got == want) > 0.995
-    # differing entries are one rounding step apart (or tiny values near zero radius)
-    diff = got != want
-    assert np.all(np.abs(got[diff] - want[diff]) <= 2.0 ** -7 * np.abs(want[diff]) + 1e-3)
+    err = np.abs(got - z)
+    # fast logarithm: absolute error 2^-22 in log2(u1), which only shows where the radius is tiny
+    assert err.max() <= 1e-3
+    assert np.mean(err <= 5e-6) > 0.995
+    assert np.mean(err <= 1e-4) > 0.9999
