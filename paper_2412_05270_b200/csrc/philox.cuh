@@ -46,9 +46,34 @@ __device__ __forceinline__ void box_muller(uint32_t xa, uint32_t xb, float& za, 
     zb = radius * sn;
 }
 
-// The four standard normals of quad q in row k.
+// Same transform with the full-precision logarithm, sine and cosine (a few ulp): used where
+// the generator is a negligible share of the work and P stays in fp32.
+__device__ __forceinline__ void box_muller_precise(uint32_t xa, uint32_t xb, float& za, float& zb)
+{
+    const float u1 = (float)((xa >> 8) + 1u) * 5.9604644775390625e-8f;
+    const float turn = (float)((int32_t)xb >> 8) * 5.9604644775390625e-8f;   // [-0.5, 0.5)
+    const float radius = sqrtf(-2.0f * logf(u1));
+    float sn, cs;
+    sincospif(2.0f * turn, &sn, &cs);
+    za = radius * cs;
+    zb = radius * sn;
+}
+
+// The four standard normals of quad q in row k (precise transform).
 __device__ __forceinline__ float4 normal_quad(uint32_t q, uint32_t k, uint32_t matrix, uint32_t epoch,
                                               uint32_t key0, uint32_t key1)
+{
+    const uint4 x = philox4x32_10(q, k, matrix, epoch, key0, key1);
+    float4 z;
+    box_muller_precise(x.x, x.y, z.x, z.y);
+    box_muller_precise(x.z, x.w, z.z, z.w);
+    return z;
+}
+
+// The same quad with the fast transform (special-function unit approximations), for the
+// tensor-core path, which rounds the result to bfloat16 anyway.
+__device__ __forceinline__ float4 normal_quad_fast(uint32_t q, uint32_t k, uint32_t matrix, uint32_t epoch,
+                                                   uint32_t key0, uint32_t key1)
 {
     const uint4 x = philox4x32_10(q, k, matrix, epoch, key0, key1);
     float4 z;

