@@ -1,0 +1,277 @@
+"""Benchmark of the APOLLO optimizer step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama7b] [--impl ours|reference]
+
+One "step" is one whole apollo_step (projection pass, finalize, update pass) over the
+LLaMA-7B-shaped list of 224 linear weights with rank 256 (bf16 W and G, fp32 states).
+Prints one JSON line.  With N > 1 (torchrun) every rank steps its own replica of the model;
+no collective runs inside the step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+import torch
+
+from paper_2412_05270_b200 import workloads as WL
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def measured_peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d} | {"source": "measured"}
+    return dict(FALLBACK_PEAKS) | {"source": "fallback"}
+
+
+def step_bytes(wl: WL.Workload):
+    """Algorithmic HBM bytes of one step: G read by both passes, W read and written,
+    fp32 M and V read and written (B_2p), and the single-read-of-G variant (B_min)."""
+    e = 2 if wl.dtype == "bf16" else 4
+    two_pass = minimal = flops = update = 0
+    for rows, cols in wl.shapes:
+        n = max(rows, cols)
+        two_pass += 4 * e * rows * cols + 16 * wl.rank * n
+        minimal += 3 * e * rows * cols + 16 * wl.rank * n
+        update += 3 * e * rows * cols
+        flops += 2 * wl.rank * rows * cols
+    return two_pass, minimal, update, flops
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def cpu_baseline(wl: WL.Workload, budget_s: float = 12.0):
+    """Times the oracle, as it stands, on the host cores over the leading matrices of the list."""
+    import oracle
+    sys.path.insert(0, str(ROOT / "tests"))
+    from parity import oracle_of
+    oracle.build()
+    cores = os.cpu_count() or 1
+    done_params, elapsed, used = 0, 0.0, []
+    for i in range(min(7, len(wl.shapes))):
+        mo = oracle_of(wl, [i])[i]
+        W = WL.make_weight(wl, i).float().numpy()
+        G = WL.make_grad(wl, i, 0).float().numpy()
+        t0 = time.perf_counter()
+        mo.step(W, G, wl.lr, wl.wd)
+        elapsed += time.perf_counter() - t0
+        done_params += W.size
+        used.append(f"{W.shape[0]}x{W.shape[1]}")
+        if elapsed > budget_s:
+            break
+    return {"value": done_params / elapsed, "unit": "params/s", "cores": cores, "kind": "oracle",
+            "sample": f"one step of matrices {', '.join(used)} of {wl.name} (rank {wl.rank}); {elapsed:.1f} s",
+            "seconds": elapsed, "params": done_params}
+
+
+def run_reference(args, wl, rank, world):
+    """The reference arm: the CPU oracle on a bounded sample of the workload."""
+    if rank != 0:
+        return
+    base = None
+    for _ in range(max(1, min(args.steps, 2))):
+        base = cpu_baseline(wl, budget_s=10.0)
+    line = {
+        "impl": "reference", "metric": "apollo_step_params_per_s", "value": base["value"], "unit": "params/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * base["seconds"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "rank": wl.rank, "mode": wl.mode, "sample": base["sample"]},
+        "cpu_baseline": {k: base[k] for k in ("value", "unit", "cores", "kind", "sample")},
+        "e2e": {"value": base["value"], "unit": "params/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, wl, rank, world, local_rank):
+    import torch.distributed as dist
+    from paper_2412_05270_b200 import binding as B
+    sys.path.insert(0, str(ROOT / "tests"))
+    from parity import config_of
+
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    n = len(wl.shapes)
+    Ws = [WL.make_weight(wl, i, device=dev) for i in range(n)]
+    Gs = [WL.make_grad(wl, i, 0, device=dev) for i in range(n)]
+    opt = B.Apollo(wl.shapes, config_of(wl), device=dev)
+    opt.set_timing(True)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        opt.step(Ws, Gs, wl.lr, wl.wd, check=False)
+    barrier()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local_rank) as clocks:
+        start.record(stream)
+        for _ in range(args.steps):
+            opt.step(Ws, Gs, wl.lr, wl.wd, check=False)
+        stop.record(stream)
+        barrier()
+    ms_total = start.elapsed_time(stop)
+    assert opt.status() == B.OK
+    launches = opt.last_launches() * args.steps
+    phases = [opt.timing(k) for k in range(min(args.steps, 64))]
+    proj_ms = sum(p[0] for p in phases) / len(phases)
+    fin_ms = sum(p[1] for p in phases) / len(phases)
+    upd_ms = sum(p[2] for p in phases) / len(phases)
+
+    # end to end: gradients arrive from pinned host memory every step, the limiter norms go back
+    e2e = None
+    if not args.no_e2e:
+        e2e_steps = max(1, min(args.steps, 3))
+        g_bytes = sum(g.numel() * g.element_size() for g in Gs)
+        host_G = [torch.empty(g.shape, dtype=g.dtype, pin_memory=True).copy_(g) for g in Gs]
+        norms_dev = torch.empty((n, 4), dtype=torch.float32, device=dev)
+        norms_host = torch.empty((n, 4), dtype=torch.float32, pin_memory=True)
+        barrier()
+        s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s2.record(stream)
+        for _ in range(e2e_steps):
+            for g, h in zip(Gs, host_G):
+                g.copy_(h, non_blocking=True)
+            opt.step(Ws, Gs, wl.lr, wl.wd, check=False)
+            for i in range(n):
+                B._check(opt.lib.apollo_get_limiter(opt.ctx, i, norms_dev[i].data_ptr(), stream.cuda_stream), "limiter")
+            norms_host.copy_(norms_dev, non_blocking=True)
+            stream.synchronize()
+        e2.record(stream)
+        barrier()
+        e2e_ms = s2.elapsed_time(e2) / e2e_steps
+        del host_G
+    times = torch.tensor([ms_total, e2e_ms if not args.no_e2e else 0.0], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms = times.tolist()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    ms_step = ms_total / args.steps
+    two_pass, minimal, update_bytes, flops = step_bytes(wl)
+    value = world * wl.params / (ms_step * 1e-3)
+    hbm, tc = peaks["hbm_gbs"] * 1e9, peaks["bf16_tflops_sustained"] * 1e12
+    t_roof = max(two_pass / hbm, flops / tc)
+    upd_gbs = update_bytes / (upd_ms * 1e-3) / 1e9
+    line = {
+        "metric": "apollo_step_params_per_s", "value": value, "unit": "params/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32",
+        "data": "synthetic",
+        "config": {"workload": wl.name, "matrices": n, "params": wl.params, "rank": wl.rank, "mode": wl.mode,
+                   "T": wl.T, "lr": wl.lr, "wd": wl.wd, "states": "f32", "replicas": world,
+                   "l2": "inputs (W, G: %.1f GB) exceed L2, no flush" % (2 * wl.params * 2 / 1e9)},
+        "roofline": {"bound": "hbm", "kernel": "update_kernel", "achieved": upd_gbs, "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": upd_gbs / peaks["hbm_gbs"], "traffic": None,
+                     "peak_source": peaks["source"], "bytes_per_launch": update_bytes, "ms_per_launch": upd_ms},
+        "step_roofline": {"bytes_two_pass": two_pass, "bytes_min": minimal, "gemm_flops": flops,
+                          "t_roofline_ms": 1e3 * t_roof, "frac": 1e3 * t_roof / ms_step,
+                          "frac_vs_8TBs": 1e3 * max(two_pass / 8e12, flops / tc) / ms_step,
+                          "phase_ms": {"projection": proj_ms, "finalize": fin_ms, "update": upd_ms}},
+        "clocks": clocks.summary(),
+        "gpu_launches": launches,
+    }
+    if not args.no_e2e:
+        line["e2e"] = {"value": world * wl.params / (e2e_ms * 1e-3), "unit": "params/s",
+                       "h2d_bytes_per_step": g_bytes, "d2h_bytes_per_step": n * 16, "ms_per_step": e2e_ms}
+    if world == 1 and not args.no_cpu:
+        base = cpu_baseline(wl)
+        line["cpu_baseline"] = {k: base[k] for k in ("value", "unit", "cores", "kind", "sample")}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="llama7b")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    wl = WL.workload(args.workload)
+    if args.impl == "reference":
+        run_reference(args, wl, rank, world)
+    else:
+        run_ours(args, wl, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

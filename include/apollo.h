@@ -155,6 +155,17 @@ APOLLO_API int apollo_projection(uint64_t seed, uint32_t matrix, uint32_t epoch,
 /* Which projection kernel a matrix was assigned: 0 streaming (rank 1), 1 CUDA cores, 2 tensor cores. */
 APOLLO_API int apollo_get_path(const apollo_ctx* ctx, int32_t matrix, int32_t* out);
 
+/*
+ * Per-phase device timing.  apollo_set_timing(ctx, 1) makes every later apollo_step record
+ * CUDA events on its stream around the three phases (projection, finalize, update); the
+ * last APOLLO_TIMING_SLOTS steps are kept.  apollo_get_timing waits for the chosen step
+ * (steps_back = 0 is the last one) and writes {projection, finalize, update, whole step}
+ * in milliseconds to h_ms (HOST, 4 floats).
+ */
+#define APOLLO_TIMING_SLOTS 64
+APOLLO_API int apollo_set_timing(apollo_ctx* ctx, int32_t on);
+APOLLO_API int apollo_get_timing(apollo_ctx* ctx, int32_t steps_back, float* h_ms);
+
 /* Kernel launches issued by the last apollo_step (HOST counter). */
 APOLLO_API int apollo_last_launches(const apollo_ctx* ctx, int32_t* out);
 

@@ -26,6 +26,7 @@ EXPORTS = [
     "apollo_workspace_bytes", "apollo_create", "apollo_step", "apollo_destroy", "apollo_step_count",
     "apollo_get_scales", "apollo_get_limiter", "apollo_get_state", "apollo_set_delta_out", "apollo_status",
     "apollo_philox_draws", "apollo_projection", "apollo_get_path", "apollo_last_launches", "apollo_strerror",
+    "apollo_set_timing", "apollo_get_timing",
 ]
 
 
@@ -77,6 +78,8 @@ def load():
     lib.apollo_projection.argtypes = [u64, u32, u32, i32, i32, vp, vp]
     lib.apollo_get_path.argtypes = [vp, i32, ctypes.POINTER(i32)]
     lib.apollo_last_launches.argtypes = [vp, ctypes.POINTER(i32)]
+    lib.apollo_set_timing.argtypes = [vp, i32]
+    lib.apollo_get_timing.argtypes = [vp, i32, ctypes.POINTER(f32)]
     lib.apollo_strerror.argtypes = [ctypes.c_int]
     lib.apollo_strerror.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -227,6 +230,15 @@ class Apollo:
         out = ctypes.c_int64(0)
         _check(self.lib.apollo_step_count(self.ctx, ctypes.byref(out)), "apollo_step_count")
         return out.value
+
+    def set_timing(self, on: bool):
+        _check(self.lib.apollo_set_timing(self.ctx, int(on)), "apollo_set_timing")
+
+    def timing(self, steps_back: int = 0):
+        """{projection, finalize, update, whole step} of a recent step, in milliseconds."""
+        out = (ctypes.c_float * 4)()
+        _check(self.lib.apollo_get_timing(self.ctx, steps_back, out), "apollo_get_timing")
+        return list(out)
 
     def last_launches(self) -> int:
         out = ctypes.c_int32(0)

@@ -139,6 +139,9 @@ struct apollo_ctx {
     int device;
     int sm_count;
     int last_launches;
+    bool timing_on;
+    bool timing_ready;
+    cudaEvent_t ev[APOLLO_TIMING_SLOTS][4];
 };
 
 extern "C" {
@@ -227,6 +230,8 @@ int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_ma
     ctx->descs_dirty = true;
     ctx->t = 0;
     ctx->last_launches = 0;
+    ctx->timing_on = false;
+    ctx->timing_ready = false;
     *out_ctx = ctx;
     return APOLLO_OK;
 }
@@ -234,6 +239,9 @@ int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_ma
 int apollo_destroy(apollo_ctx* ctx)
 {
     if (!ctx) return APOLLO_ERR_INVALID_ARG;
+    if (ctx->timing_ready)
+        for (int sl = 0; sl < APOLLO_TIMING_SLOTS; ++sl)
+            for (int e = 0; e < 4; ++e) cudaEventDestroy(ctx->ev[sl][e]);
     delete ctx;
     return APOLLO_OK;
 }
@@ -318,6 +326,8 @@ int apollo_step(apollo_ctx* ctx, void* const* d_W, const void* const* d_G, float
     }
 
     int launches = 0;
+    cudaEvent_t* ev = ctx->timing_on ? ctx->ev[ctx->t % APOLLO_TIMING_SLOTS] : nullptr;
+    if (ev) cudaEventRecord(ev[0], stream);
     if (plan.tiles[PATH_STREAM] > 0) {
         launch_project_stream(cfg.dtype, ctx->d_descs, ctx->d_prefix[PATH_STREAM], ctx->n_mat,
                               (int)plan.tiles[PATH_STREAM], sp, ctx->sm_count, stream);
@@ -332,10 +342,13 @@ int apollo_step(apollo_ctx* ctx, void* const* d_W, const void* const* d_G, float
         launches += launch_project_tensor(ctx->d_descs, ctx->d_prefix[PATH_TENSOR], ctx->n_mat,
                                           (int)plan.tiles[PATH_TENSOR], sp, ctx->sm_count, ctx->d_status, stream);
     }
+    if (ev) cudaEventRecord(ev[1], stream);
     launch_finalize(ctx->d_descs, ctx->n_mat, sp, stream);
     ++launches;
+    if (ev) cudaEventRecord(ev[2], stream);
     launch_update(cfg.dtype, ctx->d_descs, ctx->d_prefix[3], ctx->n_mat, (int)plan.tiles[3], sp, ctx->sm_count, stream);
     ++launches;
+    if (ev) cudaEventRecord(ev[3], stream);
     if (cudaGetLastError() != cudaSuccess) return APOLLO_ERR_CUDA;
     ctx->first = false;
     ctx->t += 1;
@@ -382,6 +395,32 @@ int apollo_status(apollo_ctx* ctx, void* cuda_stream)
         cudaMemset(ctx->d_status, 0, sizeof(word));
         return APOLLO_ERR_TIMEOUT;
     }
+    return APOLLO_OK;
+}
+
+int apollo_set_timing(apollo_ctx* ctx, int32_t on)
+{
+    if (!ctx) return APOLLO_ERR_INVALID_ARG;
+    if (on && !ctx->timing_ready) {
+        for (int sl = 0; sl < APOLLO_TIMING_SLOTS; ++sl)
+            for (int e = 0; e < 4; ++e)
+                if (cudaEventCreate(&ctx->ev[sl][e]) != cudaSuccess) return APOLLO_ERR_CUDA;
+        ctx->timing_ready = true;
+    }
+    ctx->timing_on = on != 0;
+    return APOLLO_OK;
+}
+
+int apollo_get_timing(apollo_ctx* ctx, int32_t steps_back, float* h_ms)
+{
+    if (!ctx || !h_ms || !ctx->timing_ready || steps_back < 0 || steps_back >= APOLLO_TIMING_SLOTS ||
+        steps_back >= ctx->t)
+        return APOLLO_ERR_INVALID_ARG;
+    cudaEvent_t* ev = ctx->ev[(ctx->t - 1 - steps_back) % APOLLO_TIMING_SLOTS];
+    if (cudaEventSynchronize(ev[3]) != cudaSuccess) return APOLLO_ERR_CUDA;
+    for (int e = 0; e < 3; ++e)
+        if (cudaEventElapsedTime(h_ms + e, ev[e], ev[e + 1]) != cudaSuccess) return APOLLO_ERR_CUDA;
+    if (cudaEventElapsedTime(h_ms + 3, ev[0], ev[3]) != cudaSuccess) return APOLLO_ERR_CUDA;
     return APOLLO_OK;
 }
 
