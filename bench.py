@@ -146,8 +146,6 @@ def run_reference(args, wl, rank, world):
 def run_ours(args, wl, rank, world, local_rank):
     import torch.distributed as dist
     from paper_2412_05270_b200 import binding as B
-    sys.path.insert(0, str(ROOT / "tests"))
-    from parity import config_of
 
     dev = torch.device("cuda", local_rank)
     torch.cuda.set_device(dev)
@@ -156,7 +154,7 @@ def run_ours(args, wl, rank, world, local_rank):
     n = len(wl.shapes)
     Ws = [WL.make_weight(wl, i, device=dev) for i in range(n)]
     Gs = [WL.make_grad(wl, i, 0, device=dev) for i in range(n)]
-    opt = B.Apollo(wl.shapes, config_of(wl), device=dev)
+    opt = B.Apollo(wl.shapes, B.config_for(wl), device=dev)
     opt.set_timing(True)
     stream = torch.cuda.current_stream()
 

@@ -117,6 +117,14 @@ def make_config(rank, mode=SCALE_CHANNEL, dtype=DT_BF16, T=200, seed=0, alpha=1.
                   float(beta1), float(beta2), float(eps), int(bool(bias_correction)), int(flags))
 
 
+def config_for(wl, flags=0, bias_correction=False) -> Config:
+    """The library configuration of a named workload (see workloads.py)."""
+    return make_config(rank=wl.rank, mode=SCALE_TENSOR if wl.mode == "tensor" else SCALE_CHANNEL,
+                       dtype=DT_BF16 if wl.dtype == "bf16" else DT_F32, T=wl.T, seed=wl.seed,
+                       alpha=wl.alpha, gamma=wl.gamma, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps,
+                       bias_correction=bias_correction, flags=flags)
+
+
 def workspace_bytes(shapes, cfg: Config) -> int:
     out = ctypes.c_size_t(0)
     _check(load().apollo_workspace_bytes(_shape_array(shapes), len(shapes), ctypes.byref(cfg), ctypes.byref(out)),

@@ -17,10 +17,7 @@ DW_REL, DW_ABS, SCALE_REL = 2e-3, 1e-6, 1e-3
 
 
 def config_of(wl: WL.Workload, flags=0, bias_correction=False) -> B.Config:
-    return B.make_config(rank=wl.rank, mode=B.SCALE_TENSOR if wl.mode == "tensor" else B.SCALE_CHANNEL,
-                         dtype=B.DT_BF16 if wl.dtype == "bf16" else B.DT_F32, T=wl.T, seed=wl.seed,
-                         alpha=wl.alpha, gamma=wl.gamma, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps,
-                         bias_correction=bias_correction, flags=flags)
+    return B.config_for(wl, flags, bias_correction)
 
 
 def oracle_of(wl: WL.Workload, mats=None, bias_correction=False):
