@@ -50,6 +50,7 @@ extern "C" {
 #define APOLLO_ERR_CUDA (-6)        /* a CUDA runtime or driver call failed */
 #define APOLLO_ERR_TIMEOUT (-7)     /* a bounded device-side wait expired (reported by apollo_status) */
 #define APOLLO_ERR_UNSUPPORTED (-8) /* the device is not an sm_100 part */
+#define APOLLO_ERR_TOO_LARGE (-9)   /* the matrix does not fit the built-in scratch of apollo_mini_step_static */
 
 #define APOLLO_MAX_RANK 512
 
@@ -165,6 +166,46 @@ APOLLO_API int apollo_get_path(const apollo_ctx* ctx, int32_t matrix, int32_t* o
 #define APOLLO_TIMING_SLOTS 64
 APOLLO_API int apollo_set_timing(apollo_ctx* ctx, int32_t on);
 APOLLO_API int apollo_get_timing(apollo_ctx* ctx, int32_t steps_back, float* h_ms);
+
+/*
+ * A rank-1 step for one matrix that allocates nothing and needs no workspace.  (The
+ * paper has no counterpart to this entry point; it computes exactly what apollo_step
+ * computes for a one-matrix list with rank 1.)
+ *
+ * Who it is for: code that is not allowed to obtain device memory at the point where it
+ * has to run the optimizer -- a plug-in running inside another runtime's memory plan, a
+ * real-time loop that must not hit the synchronisation a device allocation implies, a
+ * process whose memory pool is already handed out in full.  Such callers cannot provide
+ * apollo_create's workspace either.  Here the caller passes only the method's own inputs
+ * and outputs; the temporaries (descriptor, tile tables, partial sums of the projection,
+ * the n scales, limiter scalars) live in a fixed array of APOLLO_STATIC_SCRATCH_BYTES that
+ * is part of the library image: every GPU that loads the library holds it until exit.
+ *
+ *   d_W, d_G      DEVICE, rows x cols of cfg->dtype, 16-byte aligned; W updated in place.
+ *   d_M, d_V      DEVICE, n = max(rows, cols) floats each, 16-byte aligned: the rank-1
+ *                 moments, owned and kept by the caller between steps (zero them before
+ *                 the first step).
+ *   d_prev_norm   DEVICE, one float: the limiter's previous norm (Eq. 4), in and out;
+ *                 zero before the first step.
+ *   cfg           HOST; cfg->rank must be 1 (APOLLO_ERR_RANK otherwise); mode, dtype, T,
+ *                 seed, alpha, gamma, betas, eps, bias_correction as for apollo_create.
+ *   matrix, t     the matrix index word of the Philox counter and the number of steps
+ *                 already taken (the caller keeps t; epoch = t / T).
+ * Limits and rules: a matrix whose temporaries exceed the array -- 4 n + 8 n ceil(rows/512)
+ * bytes for a wide matrix, 12 n for a tall one, plus 1 KiB -- is rejected with
+ * APOLLO_ERR_TOO_LARGE and nothing is launched.  No cudaMalloc, cudaFree or other
+ * allocating call is made.  The first call on each device looks up the array's device
+ * address (with that device current); make that first call outside any stream capture.
+ * All calls on a device share the one array, which keeps whatever the previous call
+ * left; each call rewrites every entry it later reads, so no clearing is needed between
+ * calls, but two calls that overlap on the GPU (different streams, no ordering between
+ * them) race on it and give wrong results: order them.  Asynchronous on `cuda_stream`.
+ */
+#define APOLLO_STATIC_SCRATCH_BYTES (8u << 20)
+APOLLO_API int apollo_mini_step_static(void* d_W, const void* d_G, int64_t rows, int64_t cols,
+                                       float* d_M, float* d_V, float* d_prev_norm,
+                                       const apollo_config* cfg, uint32_t matrix, int64_t t,
+                                       float lr, float wd, void* cuda_stream);
 
 /* Kernel launches issued by the last apollo_step (HOST counter). */
 APOLLO_API int apollo_last_launches(const apollo_ctx* ctx, int32_t* out);

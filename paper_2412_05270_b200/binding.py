@@ -17,6 +17,8 @@ LIB_PATH = _PKG / "libapollo.so"
 OK = 0
 ERR_INVALID_ARG, ERR_SHAPE, ERR_RANK, ERR_ALIGN, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED = (
     -1, -2, -3, -4, -5, -6, -7, -8)
+ERR_TOO_LARGE = -9
+STATIC_SCRATCH_BYTES = 8 << 20
 SCALE_CHANNEL, SCALE_TENSOR = 0, 1
 DT_F32, DT_BF16 = 0, 1
 FLAG_NO_TENSOR_CORES = 1
@@ -26,7 +28,7 @@ EXPORTS = [
     "apollo_workspace_bytes", "apollo_create", "apollo_step", "apollo_destroy", "apollo_step_count",
     "apollo_get_scales", "apollo_get_limiter", "apollo_get_state", "apollo_set_delta_out", "apollo_status",
     "apollo_philox_draws", "apollo_projection", "apollo_get_path", "apollo_last_launches", "apollo_strerror",
-    "apollo_set_timing", "apollo_get_timing",
+    "apollo_set_timing", "apollo_get_timing", "apollo_mini_step_static",
 ]
 
 
@@ -80,6 +82,8 @@ def load():
     lib.apollo_last_launches.argtypes = [vp, ctypes.POINTER(i32)]
     lib.apollo_set_timing.argtypes = [vp, i32]
     lib.apollo_get_timing.argtypes = [vp, i32, ctypes.POINTER(f32)]
+    lib.apollo_mini_step_static.argtypes = [vp, vp, ctypes.c_int64, ctypes.c_int64, vp, vp, vp,
+                                            ctypes.POINTER(Config), u32, ctypes.c_int64, f32, f32, vp]
     lib.apollo_strerror.argtypes = [ctypes.c_int]
     lib.apollo_strerror.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -144,6 +148,21 @@ def projection(seed: int, matrix: int, epoch: int, r: int, m: int, stream=None) 
     _check(load().apollo_projection(seed, matrix, epoch, r, m, out.data_ptr(), _stream_ptr(stream)),
            "apollo_projection")
     return out
+
+
+def mini_step_static(W, G, M, V, prev_norm, cfg: Config, matrix: int, t: int, lr: float, wd: float = 0.0,
+                     stream=None):
+    """apollo_mini_step_static: a rank-1 step for one matrix that allocates nothing.
+
+    For callers that cannot get device memory when the optimizer has to run (see the
+    header): W, G are the weight and gradient, M, V (n floats) and prev_norm (1 float) the
+    state the caller keeps between steps; the temporaries live in a fixed array inside the
+    library, shared by all calls on the device, so calls must not overlap on the GPU.
+    """
+    rows, cols = W.shape
+    _check(load().apollo_mini_step_static(W.data_ptr(), G.data_ptr(), rows, cols, M.data_ptr(), V.data_ptr(),
+                                          prev_norm.data_ptr(), ctypes.byref(cfg), matrix, t, lr, wd,
+                                          _stream_ptr(stream)), "apollo_mini_step_static")
 
 
 class Apollo:

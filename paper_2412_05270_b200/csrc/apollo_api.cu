@@ -158,6 +158,7 @@ const char* apollo_strerror(int code)
         case APOLLO_ERR_CUDA: return "CUDA call failed";
         case APOLLO_ERR_TIMEOUT: return "bounded device-side wait expired";
         case APOLLO_ERR_UNSUPPORTED: return "device is not an sm_100 GPU";
+        case APOLLO_ERR_TOO_LARGE: return "matrix exceeds the built-in scratch of apollo_mini_step_static";
         default: return "unknown error";
     }
 }

@@ -27,7 +27,7 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_strerror_names_every_code():
-    for code in range(0, -9, -1):
+    for code in range(0, -10, -1):
         assert B.strerror(code) and "unknown" not in B.strerror(code)
     assert "unknown" in B.strerror(-99)
 
