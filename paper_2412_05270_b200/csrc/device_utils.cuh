@@ -59,6 +59,19 @@ __device__ __forceinline__ void load8_aligned(const __nv_bfloat16* p, float (&v)
     unpack_bf16x8(raw, v);
 }
 
+// The same for data that is read once: streaming loads that do not linger in L1.
+__device__ __forceinline__ void load8_stream(const float* p, float (&v)[8])
+{
+    const float4 a = __ldcs(reinterpret_cast<const float4*>(p));
+    const float4 b = __ldcs(reinterpret_cast<const float4*>(p) + 1);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+__device__ __forceinline__ void load8_stream(const __nv_bfloat16* p, float (&v)[8])
+{
+    const uint4 raw = __ldcs(reinterpret_cast<const uint4*>(p));
+    unpack_bf16x8(raw, v);
+}
+
 // Up to eight consecutive elements with scalar loads; entries at or past `count` read as 0.
 template <typename T>
 __device__ __forceinline__ void load8_guarded(const T* p, int count, float (&v)[8])

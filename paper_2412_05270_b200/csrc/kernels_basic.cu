@@ -404,37 +404,88 @@ update_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix,
         const float decay = sp.lr * sp.wd;
         const bool tall = d.tall != 0;
 
-#pragma unroll 2
-        for (int it = 0; it < UPDATE_TILE / (UPDATE_THREADS * 8); ++it) {
-            const uint32_t off = (uint32_t)(it * UPDATE_THREADS + threadIdx.x) * 8u;
-            const int64_t e = e0 + off;
-            if (e >= total) break;
-            const uint32_t cc = col0 + off;
-            const uint32_t radd = cc / cols;
-            uint32_t col = cc - radd * cols;
-            int64_t row = row0 + radd;
-            const int count = (int)min((int64_t)8, total - e);
-            float g[8], w[8], a[8];
-            if (count == 8) { load8_aligned(G + e, g); load8_aligned(W + e, w); }
-            else { load8_guarded(G + e, count, g); load8_guarded(W + e, count, w); }
+        constexpr int VECS = UPDATE_TILE / (UPDATE_THREADS * 8);   // vectors per thread per tile
+        constexpr int BATCH = 4;                                   // vectors whose loads are issued together
+        if (e0 + UPDATE_TILE <= total) {
+            // whole tile inside the matrix: every vector is full; issue a batch of loads first
+#pragma unroll 1
+            for (int b0 = 0; b0 < VECS; b0 += BATCH) {
+                float g[BATCH][8], w[BATCH][8];
 #pragma unroll
-            for (int x = 0; x < 8; ++x) {
-                a[x] = x < count ? __ldg(s + (tall ? (uint32_t)row : col)) : 0.f;
-                if (++col >= cols) { col = 0; ++row; }
-            }
-            float dw[8], wn[8];
+                for (int v = 0; v < BATCH; ++v) {
+                    const int64_t e = e0 + (uint32_t)((b0 + v) * UPDATE_THREADS + threadIdx.x) * 8u;
+                    load8_stream(G + e, g[v]);
+                    load8_stream(W + e, w[v]);
+                }
 #pragma unroll
-            for (int x = 0; x < 8; ++x) {
-                dw[x] = -__fmaf_rn(step * a[x], g[x], __fmul_rn(decay, w[x]));
-                wn[x] = __fadd_rn(w[x], dw[x]);
+                for (int v = 0; v < BATCH; ++v) {
+                    const uint32_t off = (uint32_t)((b0 + v) * UPDATE_THREADS + threadIdx.x) * 8u;
+                    const int64_t e = e0 + off;
+                    const uint32_t cc = col0 + off;
+                    const uint32_t radd = cc / cols;
+                    uint32_t col = cc - radd * cols;
+                    uint32_t row = (uint32_t)row0 + radd;
+                    float a[8];
+                    if (tall) {
+                        if (col + 8 <= cols) {
+                            const float sv = __ldg(s + row);
+#pragma unroll
+                            for (int x = 0; x < 8; ++x) a[x] = sv;
+                        } else {
+#pragma unroll
+                            for (int x = 0; x < 8; ++x) { a[x] = __ldg(s + row); if (++col >= cols) { col = 0; ++row; } }
+                        }
+                    } else if (col + 8 <= cols && (col & 3) == 0) {
+                        const float4 s0 = __ldg(reinterpret_cast<const float4*>(s + col));
+                        const float4 s1 = __ldg(reinterpret_cast<const float4*>(s + col + 4));
+                        a[0] = s0.x; a[1] = s0.y; a[2] = s0.z; a[3] = s0.w; a[4] = s1.x; a[5] = s1.y; a[6] = s1.z; a[7] = s1.w;
+                    } else {
+#pragma unroll
+                        for (int x = 0; x < 8; ++x) { a[x] = __ldg(s + col); if (++col >= cols) col = 0; }
+                    }
+                    float dw[8], wn[8];
+#pragma unroll
+                    for (int x = 0; x < 8; ++x) {
+                        dw[x] = -__fmaf_rn(step * a[x], g[v][x], __fmul_rn(decay, w[v][x]));
+                        wn[x] = __fadd_rn(w[v][x], dw[x]);
+                    }
+                    store8(W + e, wn);
+                    if (d.dW) store8(d.dW + e, dw);
+                }
             }
-            if (count == 8) {
-                store8(W + e, wn);
-                if (d.dW) store8(d.dW + e, dw);
-            } else {
-                for (int x = 0; x < count; ++x) {
-                    store1(W + e + x, wn[x]);
-                    if (d.dW) d.dW[e + x] = dw[x];
+        } else {
+            // last tile of a matrix: guarded vectors and a scalar tail
+            for (int it = 0; it < VECS; ++it) {
+                const uint32_t off = (uint32_t)(it * UPDATE_THREADS + threadIdx.x) * 8u;
+                const int64_t e = e0 + off;
+                if (e >= total) break;
+                const uint32_t cc = col0 + off;
+                const uint32_t radd = cc / cols;
+                uint32_t col = cc - radd * cols;
+                int64_t row = row0 + radd;
+                const int count = (int)min((int64_t)8, total - e);
+                float g[8], w[8], a[8];
+                if (count == 8) { load8_aligned(G + e, g); load8_aligned(W + e, w); }
+                else { load8_guarded(G + e, count, g); load8_guarded(W + e, count, w); }
+#pragma unroll
+                for (int x = 0; x < 8; ++x) {
+                    a[x] = x < count ? __ldg(s + (tall ? (uint32_t)row : col)) : 0.f;
+                    if (++col >= cols) { col = 0; ++row; }
+                }
+                float dw[8], wn[8];
+#pragma unroll
+                for (int x = 0; x < 8; ++x) {
+                    dw[x] = -__fmaf_rn(step * a[x], g[x], __fmul_rn(decay, w[x]));
+                    wn[x] = __fadd_rn(w[x], dw[x]);
+                }
+                if (count == 8) {
+                    store8(W + e, wn);
+                    if (d.dW) store8(d.dW + e, dw);
+                } else {
+                    for (int x = 0; x < count; ++x) {
+                        store1(W + e + x, wn[x]);
+                        if (d.dW) d.dW[e + x] = dw[x];
+                    }
                 }
             }
         }
