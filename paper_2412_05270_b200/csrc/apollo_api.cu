@@ -218,6 +218,7 @@ int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_ma
         d.s = reinterpret_cast<float*>(ctx->ws + p.off_s);
         d.part = reinterpret_cast<float*>(ctx->ws + p.off_part);
         d.g2 = reinterpret_cast<float*>(ctx->ws + p.off_g2);
+        d.tmap = ctx->ws + p.off_tmap;
         d.rows = p.rows; d.cols = p.cols; d.m = p.m; d.n = p.n; d.tall = p.tall; d.path = p.path;
         d.slices = p.slices; d.g2_slices = p.g2_slices; d.matrix_id = i;
         d.tiles_n = p.tiles_n; d.tiles_k = p.tiles_k;

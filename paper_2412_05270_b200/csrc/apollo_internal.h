@@ -33,6 +33,7 @@ struct MatDesc {
     float* g2;        // squared column norms of G: g2_slices x n
     float* scal;      // {norm after limiting, c, norm before limiting, tensor-wise s}
     float* prev;      // previous limited norm (one float)
+    const void* tmap; // 128-byte TMA tensor map of G in device memory (tensor path only)
     int32_t rows, cols;
     int32_t m, n;     // m = min(rows, cols) = projected side; n = max = number of channels
     int32_t tall;     // 1 if rows > cols: channels are the stored rows
@@ -53,6 +54,14 @@ struct StepParams {
     float lr, wd, alpha, gamma;
     float beta1, beta2, eps;
     float inv_bc1, inv_bc2;   // 1/(1-beta^t) with bias correction, else 1
+};
+
+// Tiling of the tensor-core projection (one choice per context, set by the rank).
+struct TcTiling {
+    int32_t r_slice;   // rows of R per tile = N of the MMA (multiple of 16, <= 256)
+    int32_t nblk;      // 128-channel blocks per tile (1, 2 or 4); nblk * r_slice <= 512 TMEM columns
+    int32_t stages;    // shared-memory pipeline depth
+    int32_t smem_bytes;
 };
 
 // Device status word values.

@@ -1,12 +1,425 @@
-// Tensor-core projection path (placeholder until the tcgen05 kernel lands: no matrix is
-// assigned to it).
+// Tensor-core projection: R = P G on tcgen05 with TMEM accumulators (Algorithm 1, step 1),
+// with P generated straight into shared memory (never stored) and the moment update and
+// per-channel norm sums fused into the epilogue (Algorithm 1, step 2; Eq. 5).
+//
+// Roles of the 14 warps of a CTA (one CTA per SM, persistent over tiles):
+//   warp 0      TMA producer: G tiles (128-byte swizzle) into a shared-memory ring
+//   warp 1      MMA issuer (one thread) and owner of the 512 TMEM columns
+//   warps 2-9   generators: Philox -> Box-Muller -> bf16 P tile in the UMMA K-major layout
+//   warps 10-13 column norms of G from the landed tiles
+//   warps 2-13  epilogue: tcgen05.ld of R, read-modify-write of M and V, partial sums
+//
+// Operand roles: D[128 channels x r_slice] = A[128 channels x 64] * B[r_slice x 64]^T, so
+// a TMEM lane is a channel and the reductions over r are per thread.  A = G tile: K-major
+// for a tall matrix (channels are stored rows), MN-major for a wide one.  B = P tile.
 #include "kernels.h"
+
+#include <cuda.h>
+#include <cstdlib>
+#include <cstring>
+#include <vector>
+
+#include "../../include/apollo.h"
+#include "device_utils.cuh"
+#include "philox.cuh"
+#include "tc_ptx.cuh"
 
 namespace apollo {
 
-bool tensor_path_supports(int, int, int, int) { return false; }
-void tensor_path_tiling(int, int, int, int32_t* tiles_n, int32_t* tiles_k) { *tiles_n = 0; *tiles_k = 0; }
-int tensor_path_prepare(MatDesc*, int, int, void*, cudaStream_t) { return 0; }
-int launch_project_tensor(const MatDesc*, const int*, int, int, const StepParams&, int, int32_t*, cudaStream_t) { return 0; }
+namespace {
+
+constexpr int TC_THREADS = 448;
+constexpr int TC_BK = 64;                 // contraction elements per stage (128 bytes of bf16)
+constexpr int TC_GEN_THREADS = 256;       // warps 2-9
+constexpr int TC_NORM_THREADS = 128;      // warps 10-13
+constexpr int TC_EPI_THREADS = 384;       // warps 2-13
+constexpr int TC_BLOCK_BYTES = 128 * TC_BK * 2;   // one 128-channel block of a G stage: 16 KiB
+constexpr int TC_MISC_BYTES = 256 + 3 * 512 * 8 + 8 * 512 * 4 + 1024;   // barriers, red, g2s, alignment slack
+constexpr int TC_MAX_SMEM = 227 * 1024;
+constexpr uint32_t TC_WAIT_CAP = 1u << 20;   // polls before a wait gives up (normal waits are far below 1 ms)
+
+TcTiling choose_tiling(int rank)
+{
+    TcTiling t;
+    t.r_slice = rank <= 256 ? rank : rank / 2;
+    if (const char* env = std::getenv("APOLLO_TC_RSLICE")) {
+        const int v = std::atoi(env);
+        if (v >= 16 && v <= 256 && v % 16 == 0 && rank % v == 0) t.r_slice = v;
+    }
+    const int fit = 512 / t.r_slice;
+    t.nblk = fit >= 4 ? 4 : (fit >= 2 ? 2 : 1);
+    if (const char* env = std::getenv("APOLLO_TC_NBLK")) {
+        const int v = std::atoi(env);
+        if ((v == 1 || v == 2 || v == 4) && v * t.r_slice <= 512) t.nblk = v;
+    }
+    const int stage = t.nblk * TC_BLOCK_BYTES + t.r_slice * 128;
+    t.stages = (TC_MAX_SMEM - TC_MISC_BYTES) / stage;
+    if (t.stages > 4) t.stages = 4;
+    t.smem_bytes = t.stages * stage + TC_MISC_BYTES;
+    return t;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+}  // namespace
+
+bool tensor_path_supports(int rows, int cols, int rank, int dtype)
+{
+    if (dtype != APOLLO_DT_BF16) return false;
+    if (rank < 16 || rank > 512 || rank % 16) return false;
+    if (rank > 256 && rank % 32) return false;
+    if (cols % 8) return false;                      // TMA needs a 16-byte row pitch
+    (void)rows;
+    return true;
+}
+
+void tensor_path_tiling(int rows, int cols, int rank, int32_t* tiles_n, int32_t* tiles_k)
+{
+    const TcTiling t = choose_tiling(rank);
+    const int n = rows > cols ? rows : cols;
+    *tiles_n = (n + t.nblk * 128 - 1) / (t.nblk * 128);
+    *tiles_k = rank / t.r_slice;
+}
+
+int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, void* d_tmaps, cudaStream_t stream)
+{
+    (void)rank;
+    bool any = false;
+    for (int i = 0; i < n_mat; ++i) any |= h_descs[i].path == PATH_TENSOR;
+    if (!any) return APOLLO_OK;
+    EncodeTiledFn encode = encode_fn();
+    if (!encode) return APOLLO_ERR_CUDA;
+    std::vector<CUtensorMap> maps(n_mat);
+    std::memset(maps.data(), 0, sizeof(CUtensorMap) * n_mat);
+    for (int i = 0; i < n_mat; ++i) {
+        const MatDesc& d = h_descs[i];
+        if (d.path != PATH_TENSOR) continue;
+        // dimension 0 is the contiguous one (the stored columns)
+        const cuuint64_t dims[2] = { (cuuint64_t)d.cols, (cuuint64_t)d.rows };
+        const cuuint64_t strides[1] = { (cuuint64_t)d.cols * 2 };
+        // wide: 64 channels x 64 rows of G; tall: 64 contraction elements x 128 channels
+        const cuuint32_t box[2] = { 64u, d.tall ? 128u : 64u };
+        const cuuint32_t elem[2] = { 1u, 1u };
+        const CUresult rc = encode(&maps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(d.G), dims,
+                                   strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (rc != CUDA_SUCCESS) return APOLLO_ERR_CUDA;
+    }
+    static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
+    if (cudaMemcpyAsync(d_tmaps, maps.data(), sizeof(CUtensorMap) * n_mat, cudaMemcpyHostToDevice, stream) !=
+        cudaSuccess)
+        return APOLLO_ERR_CUDA;
+    return APOLLO_OK;
+}
+
+namespace {
+
+// Bounded wait on an mbarrier phase.  On expiry the CTA-wide abort flag and the global
+// status word are set; later waits return at once, so the kernel always terminates.
+__device__ __forceinline__ void wait_phase(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status)
+{
+    if (*abort_flag) return;
+    for (uint32_t i = 0; i < TC_WAIT_CAP; ++i)
+        if (ptx::mbar_try_wait(bar, parity)) return;
+    *abort_flag = 1;
+    atomicExch(status, STATUS_TIMEOUT);
+}
+
+__device__ __forceinline__ float sum_sq_bf16x8(const uint4& v)
+{
+    float a = 0.f;
+    const uint32_t w[4] = { v.x, v.y, v.z, v.w };
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
+        a = fmaf(lo, lo, a);
+        a = fmaf(hi, hi, a);
+    }
+    return a;
+}
+
+__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, const uint4& v)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+__global__ void __launch_bounds__(TC_THREADS, 1)
+project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix, int n_mat, int total_tiles,
+                      StepParams sp, TcTiling tl, int32_t* __restrict__ status)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_addr(smem_raw));
+
+    const int r_slice = tl.r_slice, nblk = tl.nblk, stages = tl.stages;
+    const uint32_t stage_bytes = (uint32_t)(nblk * TC_BLOCK_BYTES + r_slice * 128);
+    const uint32_t p_off = (uint32_t)(nblk * TC_BLOCK_BYTES);
+    const uint32_t bars = smem_base + stages * stage_bytes;          // 8-byte mbarriers
+    const uint32_t bar_g_full = bars, bar_p_full = bars + 32, bar_empty = bars + 64, bar_acc = bars + 96;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + stages * stage_bytes + 104);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + stages * stage_bytes + 108);
+    float2* red = reinterpret_cast<float2*>(smem_gen + stages * stage_bytes + 256);          // [3][nblk*128]
+    float* g2s = reinterpret_cast<float*>(smem_gen + stages * stage_bytes + 256 + 3 * 512 * 8);   // [8][nblk*128]
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int chan_tile = nblk * 128;
+
+    if (tid == 0) {
+        for (int s = 0; s < stages; ++s) {
+            ptx::mbar_init(bar_g_full + 8 * s, 1);
+            ptx::mbar_init(bar_p_full + 8 * s, TC_GEN_THREADS / 32);
+            ptx::mbar_init(bar_empty + 8 * s, 1 + TC_NORM_THREADS / 32);
+        }
+        ptx::mbar_init(bar_acc, 1);
+        *abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_addr(tmem_slot), 512);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    uint32_t it = 0;          // k-block counter across tiles: stage = it % stages, phase = (it / stages) & 1
+    uint32_t tile_iter = 0;   // tiles done by this CTA: phase of the accumulator barrier
+
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tile_iter) {
+        const int mat = find_matrix(prefix, n_mat, tile);
+        const MatDesc& d = descs[mat];
+        const int local = tile - __ldg(prefix + mat);
+        const int tr = local % d.tiles_k, tn = local / d.tiles_k;   // row slices of one channel tile are neighbours
+        const int j0 = tn * chan_tile, r0 = tr * r_slice;
+        const int m = d.m, n = d.n;
+        const bool tall = d.tall != 0;
+        const int num_kb = (m + TC_BK - 1) / TC_BK;
+
+        if (warp == 0) {
+            // ---------------- TMA producer ----------------
+            if (lane == 0) {
+                ptx::fence_tensormap_acquire(d.tmap);
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const uint32_t s = it % stages, ph = (it / stages) & 1;
+                    wait_phase(bar_empty + 8 * s, ph ^ 1, abort_flag, status);
+                    const uint32_t g_s = smem_base + s * stage_bytes;
+                    ptx::mbar_arrive_expect_tx(bar_g_full + 8 * s, (uint32_t)(nblk * TC_BLOCK_BYTES));
+                    if (tall) {
+                        for (int b = 0; b < nblk; ++b)
+                            ptx::tma_load_2d(g_s + b * TC_BLOCK_BYTES, d.tmap, kb * TC_BK, j0 + b * 128, bar_g_full + 8 * s);
+                    } else {
+                        for (int b = 0; b < 2 * nblk; ++b)
+                            ptx::tma_load_2d(g_s + b * (TC_BLOCK_BYTES / 2), d.tmap, j0 + b * 64, kb * TC_BK, bar_g_full + 8 * s);
+                    }
+                }
+            } else {
+                it += num_kb;
+            }
+            it = __shfl_sync(0xFFFFFFFFu, it, 0);
+        } else if (warp == 1) {
+            // ---------------- MMA issuer ----------------
+            if (lane == 0) {
+                const uint32_t idesc = ptx::instr_desc_bf16((uint32_t)r_slice, !tall);
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const uint32_t s = it % stages, ph = (it / stages) & 1;
+                    wait_phase(bar_g_full + 8 * s, ph, abort_flag, status);
+                    wait_phase(bar_p_full + 8 * s, ph, abort_flag, status);
+                    ptx::tc_fence_after_sync();
+                    const uint32_t g_s = smem_base + s * stage_bytes, p_s = g_s + p_off;
+                    for (int b = 0; b < nblk; ++b) {
+#pragma unroll
+                        for (int kk = 0; kk < TC_BK / 16; ++kk) {
+                            const uint64_t a_desc = tall
+                                ? ptx::smem_desc_sw128(g_s + b * TC_BLOCK_BYTES + kk * 32, 16, 1024)
+                                : ptx::smem_desc_sw128(g_s + b * TC_BLOCK_BYTES + kk * 2048, TC_BLOCK_BYTES / 2, 1024);
+                            const uint64_t b_desc = ptx::smem_desc_sw128(p_s + kk * 32, 16, 1024);
+                            ptx::mma_bf16(tmem_base + (uint32_t)(b * r_slice), a_desc, b_desc, idesc,
+                                          (kb | kk) != 0 ? 1u : 0u);
+                        }
+                    }
+                    ptx::mma_commit(bar_empty + 8 * s);
+                }
+                ptx::mma_commit(bar_acc);
+            } else {
+                it += num_kb;
+            }
+            it = __shfl_sync(0xFFFFFFFFu, it, 0);
+        } else if (warp < 10) {
+            // ---------------- generators: P tile for every k-block ----------------
+            const int g = tid - 64;
+            for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                const uint32_t s = it % stages, ph = (it / stages) & 1;
+                wait_phase(bar_empty + 8 * s, ph ^ 1, abort_flag, status);
+                const uint32_t p_s = smem_base + s * stage_bytes + p_off;
+                for (int c = g; c < r_slice * 8; c += TC_GEN_THREADS) {
+                    const int row = c >> 3, chunk = c & 7;
+                    const uint32_t q0 = (uint32_t)(kb * (TC_BK / 4) + chunk * 2);
+                    const float4 za = normal_quad_fast(q0, (uint32_t)(r0 + row), (uint32_t)d.matrix_id, sp.epoch, sp.key0, sp.key1);
+                    const float4 zb = normal_quad_fast(q0 + 1, (uint32_t)(r0 + row), (uint32_t)d.matrix_id, sp.epoch, sp.key0, sp.key1);
+                    uint4 v;
+                    v.x = pack_bf16x2(za.x, za.y); v.y = pack_bf16x2(za.z, za.w);
+                    v.z = pack_bf16x2(zb.x, zb.y); v.w = pack_bf16x2(zb.z, zb.w);
+                    st_shared_v4(p_s + row * 128 + ((chunk ^ (row & 7)) << 4), v);
+                }
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(bar_p_full + 8 * s);
+            }
+        } else {
+            // ---------------- column norms of G from the landed tiles ----------------
+            const int t = tid - 320;
+            float acc[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+            const int ccols = 16 * nblk;                 // wide: 16-byte chunk columns per stage
+            const int parts = TC_NORM_THREADS / ccols;   // wide: threads sharing one chunk column
+            const int cc = t % ccols, part = t / ccols;
+            const int rows_pp = TC_BK / parts;
+            for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                const uint32_t s = it % stages, ph = (it / stages) & 1;
+                wait_phase(bar_g_full + 8 * s, ph, abort_flag, status);
+                const uint32_t g_s = smem_base + s * stage_bytes;
+                if (tall) {
+                    // block b, row t: 128 bytes = 8 chunks; the order of the chunks does not matter
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) {
+                        if (b < nblk) {
+                            const uint32_t row = g_s + b * TC_BLOCK_BYTES + t * 128;
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) acc[b] += sum_sq_bf16x8(ld_shared_v4(row + (((i + t) & 7) << 4)));
+                        }
+                    }
+                } else {
+                    const uint32_t colbase = g_s + (cc >> 3) * (TC_BLOCK_BYTES / 2);
+                    const int c = cc & 7;
+                    for (int k = part * rows_pp; k < (part + 1) * rows_pp; ++k) {
+                        const uint4 v = ld_shared_v4(colbase + k * 128 + ((c ^ (k & 7)) << 4));
+                        const uint32_t w[4] = { v.x, v.y, v.z, v.w };
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
+                            acc[2 * i] = fmaf(lo, lo, acc[2 * i]);
+                            acc[2 * i + 1] = fmaf(hi, hi, acc[2 * i + 1]);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(bar_empty + 8 * s);
+            }
+            if (tall) {
+#pragma unroll
+                for (int b = 0; b < 4; ++b) if (b < nblk) g2s[b * 128 + t] = acc[b];
+            } else {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) g2s[part * chan_tile + cc * 8 + e] = acc[e];
+            }
+        }
+
+        if (warp >= 2) {
+            // ---------------- epilogue: moments and per-channel sums ----------------
+            const int q = warp & 3, widx = (warp - 2) >> 2;
+            const int ch_in_blk = q * 32 + lane;
+            for (int b = 0; b < nblk; ++b) red[widx * chan_tile + b * 128 + ch_in_blk] = make_float2(0.f, 0.f);
+            wait_phase(bar_acc, tile_iter & 1, abort_flag, status);
+            ptx::tc_fence_after_sync();
+            const int chunks = r_slice / 16, items = nblk * chunks;
+            float num = 0.f, den = 0.f;
+            int cur_b = -1;
+            for (int item = widx; item < items; item += 3) {
+                const int b = item / chunks, cchunk = item % chunks;
+                if (b != cur_b) {
+                    if (cur_b >= 0) red[widx * chan_tile + cur_b * 128 + ch_in_blk] = make_float2(num, den);
+                    cur_b = b; num = 0.f; den = 0.f;
+                }
+                float rv[16];
+                ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * r_slice + cchunk * 16), rv);
+                const int j = j0 + b * 128 + ch_in_blk;
+                if (j < n) {
+                    float* Mp = d.M + (int64_t)(r0 + cchunk * 16) * n + j;
+                    float* Vp = d.V + (int64_t)(r0 + cchunk * 16) * n + j;
+                    float mv[16], vv[16];
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) { mv[k] = Mp[(int64_t)k * n]; vv[k] = Vp[(int64_t)k * n]; }
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) {
+                        const float r = rv[k] * sp.inv_sqrt_r;
+                        const float mn = sp.beta1 * mv[k] + (1.0f - sp.beta1) * r;
+                        const float vn = sp.beta2 * vv[k] + (1.0f - sp.beta2) * r * r;
+                        Mp[(int64_t)k * n] = mn; Vp[(int64_t)k * n] = vn;
+                        const float rt = (mn * sp.inv_bc1) / (sqrtf(vn * sp.inv_bc2) + sp.eps);
+                        num = fmaf(rt, rt, num);
+                        den = fmaf(r, r, den);
+                    }
+                }
+            }
+            if (cur_b >= 0) red[widx * chan_tile + cur_b * 128 + ch_in_blk] = make_float2(num, den);
+            ptx::tc_fence_before_sync();
+            ptx::named_barrier(1, TC_EPI_THREADS);
+            const int parts = tall ? 1 : TC_NORM_THREADS / (16 * nblk);
+            for (int ch = tid - 64; ch < chan_tile; ch += TC_EPI_THREADS) {
+                const int j = j0 + ch;
+                if (j < n) {
+                    const float2 a = red[ch], b2 = red[chan_tile + ch], c2 = red[2 * chan_tile + ch];
+                    reinterpret_cast<float2*>(d.part)[(int64_t)tr * n + j] = make_float2(a.x + b2.x + c2.x, a.y + b2.y + c2.y);
+                    if (tr == 0) {
+                        float g2 = 0.f;
+                        for (int p = 0; p < parts; ++p) g2 += g2s[p * chan_tile + ch];
+                        d.g2[j] = g2;
+                    }
+                }
+            }
+        }
+        // the accumulator is drained: the issuer may start the next tile
+        if (warp >= 1) {
+            ptx::tc_fence_before_sync();
+            ptx::named_barrier(2, TC_THREADS - 32);
+            ptx::tc_fence_after_sync();
+        }
+    }
+
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) ptx::tmem_dealloc(tmem_base, 512);
+}
+
+}  // namespace
+
+int launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_mat, int total_tiles,
+                          const StepParams& sp, int sm_count, int32_t* d_status, cudaStream_t stream)
+{
+    if (total_tiles <= 0) return 0;
+    const TcTiling tl = choose_tiling(sp.rank);
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(project_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
+        attr_set = true;
+    }
+    const int grid = total_tiles < sm_count ? total_tiles : sm_count;
+    project_tensor_kernel<<<grid, TC_THREADS, tl.smem_bytes, stream>>>(d_descs, d_prefix, n_mat, total_tiles, sp, tl,
+                                                                     d_status);
+    return 1;
+}
 
 }  // namespace apollo

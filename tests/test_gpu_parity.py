@@ -48,6 +48,24 @@ def test_streaming_path_spanning_row_blocks_and_column_tiles():
     run_parity(wl, expect_path=B.PATH_STREAM)
 
 
+@pytest.mark.parametrize("rank,shapes", [
+    (16, [(64, 72), (72, 64), (128, 128), (16, 520)]),
+    (64, [(200, 1000), (1000, 200), (520, 264)]),
+    (128, [(300, 1032), (1032, 304)]),
+    (256, [(512, 1376), (1376, 512), (512, 512)]),
+    (512, [(512, 1376), (1376, 512)]),
+    (48, [(96, 200), (200, 96)]),
+])
+def test_tensor_core_path(rank, shapes):
+    wl = _wl(shapes, rank, dtype="bf16", steps=4, T=2, wd=0.01)
+    run_parity(wl, expect_path=B.PATH_TENSOR)
+
+
+def test_tensor_core_path_tensor_mode_and_bias_correction():
+    wl = _wl([(256, 520), (520, 256)], 32, mode="tensor", dtype="bf16", steps=3, T=2)
+    run_parity(wl, expect_path=B.PATH_TENSOR, bias_correction=True)
+
+
 def test_bias_correction_variant():
     wl = _wl([(33, 130), (130, 33)], 4, dtype="f32", steps=4)
     run_parity(wl, flags=B.FLAG_NO_TENSOR_CORES, bias_correction=True)
