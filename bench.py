@@ -112,7 +112,7 @@ def cpu_baseline(wl: WL.Workload, budget_s: float = 12.0):
         W = WL.make_weight(wl, i).float().numpy()
         G = WL.make_grad(wl, i, 0).float().numpy()
         t0 = time.perf_counter()
-        mo.step(W, G, wl.lr, wl.wd)
+        mo.step(W, G, float(wl.lr), float(wl.wd))
         elapsed += time.perf_counter() - t0
         done_params += W.size
         used.append(f"{W.shape[0]}x{W.shape[1]}")

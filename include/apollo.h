@@ -13,7 +13,9 @@
  *   1. P (r x m), entries N(0, 1/r), is regenerated from a counter-based Philox4x32-10
  *      stream keyed by the seed, with counter (column quad, row, matrix index,
  *      epoch = floor(t / T)); it is never stored (Algorithm 1, "P_t <- N_seed(0, 1/r)";
- *      Section "Generating random projection matrix").
+ *      Section "Generating random projection matrix").  P has the precision of the
+ *      projection's operands: its standard normals are rounded to bfloat16 for bf16
+ *      gradients at rank > 1, and kept in fp32 for fp32 gradients and at rank 1.
  *   2. R = P G  (r x n)                                        (Algorithm 1, step 1).
  *   3. M <- beta1 M + (1-beta1) R,  V <- beta2 V + (1-beta2) R^2,
  *      R~ = M / (sqrt(V) + eps)                                (Algorithm 1, step 2).
@@ -145,8 +147,7 @@ APOLLO_API int apollo_status(apollo_ctx* ctx, void* cuda_stream);
  * apollo_philox_draws:  d_out DEVICE, r x ceil(m/4) x 4 uint32: the raw Philox4x32-10
  *                       words for counter (q, k, matrix, epoch), key = seed.
  * apollo_projection:    d_out DEVICE, r x m floats: the standard normals Z behind P
- *                       (P = Z / sqrt(r)) in fp32, as the CUDA-core kernels use them; the
- *                       tensor-core kernel rounds the same values to bfloat16 operands.
+ *                       (P = Z / sqrt(r)) in fp32, before any rounding to bfloat16.
  */
 APOLLO_API int apollo_philox_draws(uint64_t seed, uint32_t matrix, uint32_t epoch, int32_t r, int32_t m,
                         uint32_t* d_out, void* cuda_stream);

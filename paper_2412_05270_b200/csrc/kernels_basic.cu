@@ -225,6 +225,9 @@ project_simt_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                 if (k0 + row < r)
                     z = normal_quad((uint32_t)(i0 / 4 + q), (uint32_t)(k0 + row), (uint32_t)d.matrix_id, sp.epoch,
                                     sp.key0, sp.key1);
+                if (sizeof(T) == 2) {   // bf16 gradients: P has the precision of the GEMM operands
+                    z.x = round_to_bf16(z.x); z.y = round_to_bf16(z.y); z.z = round_to_bf16(z.z); z.w = round_to_bf16(z.w);
+                }
                 Ps[4 * q + 0][row] = z.x; Ps[4 * q + 1][row] = z.y;
                 Ps[4 * q + 2][row] = z.z; Ps[4 * q + 3][row] = z.w;
             }

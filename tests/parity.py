@@ -20,14 +20,22 @@ def config_of(wl: WL.Workload, flags=0, bias_correction=False) -> B.Config:
     return B.config_for(wl, flags, bias_correction)
 
 
+def _f32(x) -> float:
+    """The value the C ABI's float field holds: both sides get the same configuration."""
+    return float(np.float32(x))
+
+
 def oracle_of(wl: WL.Workload, mats=None, bias_correction=False):
     mats = range(len(wl.shapes)) if mats is None else mats
+    # P has the precision of the projection's operands: bfloat16 for bf16 gradients at rank > 1
+    # (tensor-core operands), fp32 for fp32 gradients and for the rank-1 matrix-vector pass.
+    p_bf16 = wl.dtype == "bf16" and wl.rank > 1
     return {i: oracle.MatrixOracle(wl.shapes[i][0], wl.shapes[i][1], rank=wl.rank,
                                    mode=oracle.MODE_TENSOR if wl.mode == "tensor" else oracle.MODE_CHANNEL,
                                    dtype=oracle.DT_BF16 if wl.dtype == "bf16" else oracle.DT_F32,
-                                   seed=wl.seed, matrix_id=i, T=wl.T, alpha=wl.alpha, gamma=wl.gamma,
-                                   beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps, bias_correction=bias_correction,
-                                   p_round_bf16=False) for i in mats}
+                                   seed=wl.seed, matrix_id=i, T=wl.T, alpha=_f32(wl.alpha), gamma=_f32(wl.gamma),
+                                   beta1=_f32(wl.beta1), beta2=_f32(wl.beta2), eps=_f32(wl.eps),
+                                   bias_correction=bias_correction, p_round_bf16=p_bf16) for i in mats}
 
 
 def run_parity(wl: WL.Workload, steps=None, flags=0, bias_correction=False, check_mats=None, expect_path=None,
@@ -55,7 +63,7 @@ def run_parity(wl: WL.Workload, steps=None, flags=0, bias_correction=False, chec
         opt.step(Wg, Gg, wl.lr, wl.wd)
         assert opt.status() == B.OK
         for i in check_mats:
-            res = orc[i].step(Wo[i], Gc[i].float().numpy(), wl.lr, wl.wd, want_R=True)
+            res = orc[i].step(Wo[i], Gc[i].float().numpy(), _f32(wl.lr), _f32(wl.wd), want_R=True)
             dw_gpu = deltas[i].cpu().numpy().astype(np.float64)
             bound = DW_REL * np.max(np.abs(res.dW)) + DW_ABS
             err = np.max(np.abs(dw_gpu - res.dW))
