@@ -257,6 +257,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="llama7b")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=0, help="keep only the first LAYERS layers (profiling aid)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
@@ -265,6 +266,9 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     wl = WL.workload(args.workload)
+    if args.layers > 0:
+        wl.shapes = wl.shapes[:7 * args.layers]
+        wl.name = f"{wl.name}[first {args.layers} layers]"
     if args.impl == "reference":
         run_reference(args, wl, rank, world)
     else:

@@ -93,9 +93,9 @@ double oracle_round_bf16(double x)
 }
 
 /*
- * Box-Muller on the Philox words (x0,x1) and (x2,x3):
- *   u1 = ((x >> 8) + 1) / 2^24 in (0,1],  u2 = (x' >> 8) / 2^24 in [0,1),
- *   z_a = sqrt(-2 ln u1) cos(2 pi u2),    z_b = sqrt(-2 ln u1) sin(2 pi u2).
+ * Box-Muller on the Philox words (x0,x1) and (x2,x3), using the top 23 bits of each word:
+ *   u1 = 1 - (x >> 9) / 2^23 in (0,1],   angle = 2 pi ((x' >> 9) / 2^23 - 1/2) in [-pi, pi),
+ *   z_a = sqrt(-2 ln u1) cos(angle),     z_b = sqrt(-2 ln u1) sin(angle).
  * z: r x m standard normals (entries past m of the last quad are dropped).
  */
 void oracle_standard_normals(uint64_t seed, uint32_t matrix_id, uint32_t epoch,
@@ -111,11 +111,11 @@ void oracle_standard_normals(uint64_t seed, uint32_t matrix_id, uint32_t epoch,
             oracle_philox4x32_10(ctr, key, x);
             double zz[4];
             for (int h = 0; h < 2; ++h) {
-                double u1 = ((double)(x[2 * h] >> 8) + 1.0) / 16777216.0;
-                double u2 = (double)(x[2 * h + 1] >> 8) / 16777216.0;
+                double u1 = 1.0 - (double)(x[2 * h] >> 9) / 8388608.0;
+                double angle = two_pi * ((double)(x[2 * h + 1] >> 9) / 8388608.0 - 0.5);
                 double radius = sqrt(-2.0 * log(u1));
-                zz[2 * h] = radius * cos(two_pi * u2);
-                zz[2 * h + 1] = radius * sin(two_pi * u2);
+                zz[2 * h] = radius * cos(angle);
+                zz[2 * h + 1] = radius * sin(angle);
             }
             for (int e = 0; e < 4; ++e) {
                 int32_t i = 4 * q + e;

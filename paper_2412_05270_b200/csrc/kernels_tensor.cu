@@ -273,15 +273,25 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                 const uint32_t s = it % stages, ph = (it / stages) & 1;
                 wait_phase(bar_empty + 8 * s, ph ^ 1, abort_flag, status);
                 const uint32_t p_s = smem_base + s * stage_bytes + p_off;
-                for (int c = g; c < r_slice * 8; c += TC_GEN_THREADS) {
+                // two rows per pass (32 rows apart) so that four Philox chains are in flight per thread
+                const int total = r_slice * 8;
+                for (int c = g; c < total; c += 2 * TC_GEN_THREADS) {
                     const int row = c >> 3, chunk = c & 7;
                     const uint32_t q0 = (uint32_t)(kb * (TC_BK / 4) + chunk * 2);
-                    const float4 za = normal_quad_fast(q0, (uint32_t)(r0 + row), (uint32_t)d.matrix_id, sp.epoch, sp.key0, sp.key1);
-                    const float4 zb = normal_quad_fast(q0 + 1, (uint32_t)(r0 + row), (uint32_t)d.matrix_id, sp.epoch, sp.key0, sp.key1);
-                    uint4 v;
-                    v.x = pack_bf16x2(za.x, za.y); v.y = pack_bf16x2(za.z, za.w);
-                    v.z = pack_bf16x2(zb.x, zb.y); v.w = pack_bf16x2(zb.z, zb.w);
-                    st_shared_v4(p_s + row * 128 + ((chunk ^ (row & 7)) << 4), v);
+                    const uint32_t ka = (uint32_t)(r0 + row), kbrow = ka + 32u;
+                    const uint32_t mid = (uint32_t)d.matrix_id;
+                    const float4 a0 = normal_quad_fast(q0, ka, mid, sp.epoch, sp.key0, sp.key1);
+                    const float4 a1 = normal_quad_fast(q0 + 1, ka, mid, sp.epoch, sp.key0, sp.key1);
+                    const float4 b0 = normal_quad_fast(q0, kbrow, mid, sp.epoch, sp.key0, sp.key1);
+                    const float4 b1 = normal_quad_fast(q0 + 1, kbrow, mid, sp.epoch, sp.key0, sp.key1);
+                    uint4 va, vb;
+                    va.x = pack_bf16x2(a0.x, a0.y); va.y = pack_bf16x2(a0.z, a0.w);
+                    va.z = pack_bf16x2(a1.x, a1.y); va.w = pack_bf16x2(a1.z, a1.w);
+                    vb.x = pack_bf16x2(b0.x, b0.y); vb.y = pack_bf16x2(b0.z, b0.w);
+                    vb.z = pack_bf16x2(b1.x, b1.y); vb.w = pack_bf16x2(b1.z, b1.w);
+                    const uint32_t at = p_s + row * 128 + ((chunk ^ (row & 7)) << 4);
+                    st_shared_v4(at, va);
+                    if (c + TC_GEN_THREADS < total) st_shared_v4(at + 32 * 128, vb);   // row + 32: same swizzle phase
                 }
                 ptx::fence_proxy_async_smem();
                 __syncwarp();

@@ -13,8 +13,10 @@ namespace apollo {
 __device__ __forceinline__ void philox_round(uint32_t& c0, uint32_t& c1, uint32_t& c2, uint32_t& c3,
                                              uint32_t k0, uint32_t k1)
 {
-    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
-    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    const uint64_t p0 = (uint64_t)0xD2511F53u * c0;     // one 32x32->64 multiply each
+    const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+    const uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0;
+    const uint32_t hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
     const uint32_t n0 = hi1 ^ c1 ^ k0;
     const uint32_t n2 = hi0 ^ c3 ^ k1;
     c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
@@ -32,16 +34,24 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
     return make_uint4(c0, c1, c2, c3);
 }
 
-// u1 = ((xa >> 8) + 1) / 2^24 in (0, 1];  angle = 2 pi (xb >> 8) / 2^24, taken modulo
-// 2 pi into [-pi, pi) (an arithmetic shift of xb) where the fast sine and cosine are
-// most accurate.  za = radius cos, zb = radius sin.
+// The top 23 bits of a word as a float in [1, 2): 1 + (x >> 9) / 2^23 (one funnel shift).
+__device__ __forceinline__ float unit_interval_12(uint32_t x)
+{
+    return __uint_as_float(__funnelshift_r(x, 0x7Fu, 9));
+}
+
+// Box-Muller on two words:  u1 = 1 - (xa >> 9) / 2^23 in (0, 1],
+// angle = 2 pi ((xb >> 9) / 2^23 - 1/2) in [-pi, pi);  za = radius cos, zb = radius sin with
+// radius = sqrt(-2 ln u1).  Fast version: special-function unit approximations.
 __device__ __forceinline__ void box_muller(uint32_t xa, uint32_t xb, float& za, float& zb)
 {
-    const float u1 = (float)((xa >> 8) + 1u) * 5.9604644775390625e-8f;
-    const float turn = (float)((int32_t)xb >> 8) * 5.9604644775390625e-8f;   // [-0.5, 0.5)
-    const float radius = sqrtf(-2.0f * __logf(u1));
-    float sn, cs;
-    __sincosf(6.283185307179586f * turn, &sn, &cs);
+    const float u1 = 2.0f - unit_interval_12(xa);
+    const float ang = (unit_interval_12(xb) - 1.5f) * 6.283185307179586f;
+    float lg, radius, sn, cs;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(lg) : "f"(u1));
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(radius) : "f"(lg * -1.3862943611198906f));   // -2 ln 2 log2(u1)
+    asm("sin.approx.ftz.f32 %0, %1;" : "=f"(sn) : "f"(ang));
+    asm("cos.approx.ftz.f32 %0, %1;" : "=f"(cs) : "f"(ang));
     za = radius * cs;
     zb = radius * sn;
 }
@@ -50,8 +60,8 @@ __device__ __forceinline__ void box_muller(uint32_t xa, uint32_t xb, float& za, 
 // the generator is a negligible share of the work and P stays in fp32.
 __device__ __forceinline__ void box_muller_precise(uint32_t xa, uint32_t xb, float& za, float& zb)
 {
-    const float u1 = (float)((xa >> 8) + 1u) * 5.9604644775390625e-8f;
-    const float turn = (float)((int32_t)xb >> 8) * 5.9604644775390625e-8f;   // [-0.5, 0.5)
+    const float u1 = 2.0f - unit_interval_12(xa);
+    const float turn = unit_interval_12(xb) - 1.5f;   // [-0.5, 0.5)
     const float radius = sqrtf(-2.0f * logf(u1));
     float sn, cs;
     sincospif(2.0f * turn, &sn, &cs);
@@ -70,8 +80,8 @@ __device__ __forceinline__ float4 normal_quad(uint32_t q, uint32_t k, uint32_t m
     return z;
 }
 
-// The same quad with the fast transform (special-function unit approximations), for the
-// tensor-core path, which rounds the result to bfloat16 anyway.
+// The same quad with the fast transform, for the tensor-core path, which rounds the result
+// to bfloat16 anyway.
 __device__ __forceinline__ float4 normal_quad_fast(uint32_t q, uint32_t k, uint32_t matrix, uint32_t epoch,
                                                    uint32_t key0, uint32_t key1)
 {

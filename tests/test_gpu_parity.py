@@ -44,7 +44,10 @@ def test_streaming_path_spanning_row_blocks_and_column_tiles():
     wl = _wl([(1100, 1300), (1300, 1100), (600, 2600), (70, 3000), (3000, 2100)], 1, mode="tensor", dtype="bf16",
              steps=3, alpha=math.sqrt(128.0))
     run_parity(wl, expect_path=B.PATH_STREAM)
-    wl = _wl([(1029, 1301), (1301, 1029)], 1, mode="channel", dtype="f32", steps=3)   # unaligned pitch
+    # unaligned pitch (scalar loads).  Tensor-wise scale: at rank 1 a channel-wise scale divides by
+    # one signed number per channel, which among a thousand channels cancels to ~1e-4 of its terms
+    # somewhere, and no fp32 path can then hold a relative bound.
+    wl = _wl([(1029, 1301), (1301, 1029)], 1, mode="tensor", dtype="f32", steps=3, alpha=math.sqrt(128.0))
     run_parity(wl, expect_path=B.PATH_STREAM)
 
 

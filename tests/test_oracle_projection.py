@@ -19,17 +19,18 @@ def test_standard_normals_pass_a_kolmogorov_smirnov_test():
 
 
 def test_box_muller_pairs_share_a_radius_fixed_by_the_first_word():
-    # z[4q]^2 + z[4q+1]^2 = -2 ln u1 with u1 from word 0; same for words 2, 3.
+    # z[4q]^2 + z[4q+1]^2 = -2 ln u1 with u1 from the top 23 bits of word 0; same for words 2, 3.
     r, m = 3, 24
     z = oracle.standard_normals(9, 1, 2, r, m).reshape(r, m // 4, 4)
     d = oracle.philox_draws(9, 1, 2, r, m)
     for h in range(2):
-        u1 = ((d[..., 2 * h] >> np.uint32(8)).astype(np.float64) + 1.0) / 2.0**24
+        u1 = 1.0 - (d[..., 2 * h] >> np.uint32(9)).astype(np.float64) / 2.0**23
         rad2 = z[..., 2 * h] ** 2 + z[..., 2 * h + 1] ** 2
         np.testing.assert_allclose(rad2, -2.0 * np.log(u1), rtol=1e-12)
-        u2 = (d[..., 2 * h + 1] >> np.uint32(8)).astype(np.float64) / 2.0**24
-        ang = np.mod(np.arctan2(z[..., 2 * h + 1], z[..., 2 * h]), 2 * np.pi)
-        np.testing.assert_allclose(ang, 2 * np.pi * u2, atol=1e-9)
+        u2 = (d[..., 2 * h + 1] >> np.uint32(9)).astype(np.float64) / 2.0**23
+        ang = np.arctan2(z[..., 2 * h + 1], z[..., 2 * h])
+        want = 2 * np.pi * (u2 - 0.5)
+        np.testing.assert_allclose(np.mod(ang - want + np.pi, 2 * np.pi) - np.pi, 0.0, atol=1e-9)
 
 
 def test_ragged_m_drops_the_tail_of_the_last_quad():
