@@ -213,6 +213,10 @@ APOLLO_API int apollo_last_launches(const apollo_ctx* ctx, int32_t* out);
 
 APOLLO_API const char* apollo_strerror(int code);
 
+/* Text of the last CUDA error this library saw on the calling thread ("no error" if none);
+ * the detail behind an APOLLO_ERR_CUDA return. */
+APOLLO_API const char* apollo_cuda_error_string(void);
+
 #ifdef __cplusplus
 }
 #endif

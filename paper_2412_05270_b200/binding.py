@@ -28,13 +28,14 @@ EXPORTS = [
     "apollo_workspace_bytes", "apollo_create", "apollo_step", "apollo_destroy", "apollo_step_count",
     "apollo_get_scales", "apollo_get_limiter", "apollo_get_state", "apollo_set_delta_out", "apollo_status",
     "apollo_philox_draws", "apollo_projection", "apollo_get_path", "apollo_last_launches", "apollo_strerror",
-    "apollo_set_timing", "apollo_get_timing", "apollo_mini_step_static",
+    "apollo_set_timing", "apollo_get_timing", "apollo_mini_step_static", "apollo_cuda_error_string",
 ]
 
 
 class ApolloError(RuntimeError):
     def __init__(self, code: int, what: str):
-        super().__init__(f"{what}: {strerror(code)} ({code})")
+        detail = f" [{load().apollo_cuda_error_string().decode()}]" if code == ERR_CUDA else ""
+        super().__init__(f"{what}: {strerror(code)} ({code}){detail}")
         self.code = code
 
 
@@ -86,8 +87,10 @@ def load():
                                             ctypes.POINTER(Config), u32, ctypes.c_int64, f32, f32, vp]
     lib.apollo_strerror.argtypes = [ctypes.c_int]
     lib.apollo_strerror.restype = ctypes.c_char_p
+    lib.apollo_cuda_error_string.argtypes = []
+    lib.apollo_cuda_error_string.restype = ctypes.c_char_p
     for name in EXPORTS:
-        if name != "apollo_strerror":
+        if name not in ("apollo_strerror", "apollo_cuda_error_string"):
             getattr(lib, name).restype = ctypes.c_int
     _lib = lib
     return lib

@@ -121,6 +121,15 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
 
 }  // namespace
 
+static thread_local cudaError_t g_last_cuda_error = cudaSuccess;
+
+// Records a failing CUDA status for apollo_cuda_error_string(); returns true on success.
+static bool cuda_ok(cudaError_t e)
+{
+    if (e != cudaSuccess) { g_last_cuda_error = e; cudaGetLastError(); return false; }
+    return true;
+}
+
 struct apollo_ctx {
     apollo_config cfg;
     int32_t n_mat;
@@ -145,6 +154,8 @@ struct apollo_ctx {
 };
 
 extern "C" {
+
+const char* apollo_cuda_error_string(void) { return cudaGetErrorString(g_last_cuda_error); }
 
 const char* apollo_strerror(int code)
 {
@@ -316,6 +327,7 @@ int apollo_step(apollo_ctx* ctx, void* const* d_W, const void* const* d_G, float
     StepParams sp;
     sp.key0 = (uint32_t)(cfg.seed & 0xFFFFFFFFull);
     sp.key1 = (uint32_t)(cfg.seed >> 32);
+    fill_round_keys(sp);
     sp.epoch = (uint32_t)(ctx->t / cfg.T);
     sp.rank = cfg.rank; sp.mode = cfg.mode;
     sp.inv_sqrt_r = (float)(1.0 / std::sqrt((double)cfg.rank));
@@ -351,7 +363,7 @@ int apollo_step(apollo_ctx* ctx, void* const* d_W, const void* const* d_G, float
     launch_update(cfg.dtype, ctx->d_descs, ctx->d_prefix[3], ctx->n_mat, (int)plan.tiles[3], sp, ctx->sm_count, stream);
     ++launches;
     if (ev) cudaEventRecord(ev[3], stream);
-    if (cudaGetLastError() != cudaSuccess) return APOLLO_ERR_CUDA;
+    if (!cuda_ok(cudaGetLastError())) return APOLLO_ERR_CUDA;
     ctx->first = false;
     ctx->t += 1;
     ctx->last_launches = launches;

@@ -54,7 +54,16 @@ struct StepParams {
     float lr, wd, alpha, gamma;
     float beta1, beta2, eps;
     float inv_bc1, inv_bc2;   // 1/(1-beta^t) with bias correction, else 1
+    uint32_t round_key[20];   // Philox key schedule: {key0 + i W0, key1 + i W1}, i = 0..9
 };
+
+inline void fill_round_keys(StepParams& sp)
+{
+    for (int i = 0; i < 10; ++i) {
+        sp.round_key[2 * i] = sp.key0 + (uint32_t)i * 0x9E3779B9u;
+        sp.round_key[2 * i + 1] = sp.key1 + (uint32_t)i * 0xBB67AE85u;
+    }
+}
 
 // Tiling of the tensor-core projection (one choice per context, set by the rank).
 struct TcTiling {

@@ -153,6 +153,13 @@ __device__ __forceinline__ float sum_sq_bf16x8(const uint4& v)
     return a;
 }
 
+__device__ __forceinline__ float fast_sqrt(float x)
+{
+    float y;
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 __device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr)
 {
     uint4 v;
@@ -164,6 +171,7 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, const uint4& v)
     asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
+// 14 warps are allocated as 16: 128 registers per thread is the ceiling
 __global__ void __launch_bounds__(TC_THREADS, 1)
 project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix, int n_mat, int total_tiles,
                       StepParams sp, TcTiling tl, int32_t* __restrict__ status)
@@ -209,18 +217,27 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
 
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tile_iter) {
         const int mat = find_matrix(prefix, n_mat, tile);
-        const MatDesc& d = descs[mat];
+        // copy what the roles need into registers: the descriptor lives in global memory and
+        // every shared-memory asm below is a compiler memory barrier
+        const MatDesc* dp = descs + mat;
+        const int tiles_k = __ldg(&dp->tiles_k);
+        const int m = __ldg(&dp->m), n = __ldg(&dp->n);
+        const bool tall = __ldg(&dp->tall) != 0;
+        const uint32_t matrix_id = (uint32_t)__ldg(&dp->matrix_id);
+        const void* tmap = dp->tmap;
+        float* const Mbase = dp->M;
+        float* const Vbase = dp->V;
+        float* const part = dp->part;
+        float* const g2out = dp->g2;
         const int local = tile - __ldg(prefix + mat);
-        const int tr = local % d.tiles_k, tn = local / d.tiles_k;   // row slices of one channel tile are neighbours
+        const int tr = local % tiles_k, tn = local / tiles_k;   // row slices of one channel tile are neighbours
         const int j0 = tn * chan_tile, r0 = tr * r_slice;
-        const int m = d.m, n = d.n;
-        const bool tall = d.tall != 0;
         const int num_kb = (m + TC_BK - 1) / TC_BK;
 
         if (warp == 0) {
             // ---------------- TMA producer ----------------
             if (lane == 0) {
-                ptx::fence_tensormap_acquire(d.tmap);
+                ptx::fence_tensormap_acquire(tmap);
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
                     const uint32_t s = it % stages, ph = (it / stages) & 1;
                     wait_phase(bar_empty + 8 * s, ph ^ 1, abort_flag, status);
@@ -228,10 +245,10 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                     ptx::mbar_arrive_expect_tx(bar_g_full + 8 * s, (uint32_t)(nblk * TC_BLOCK_BYTES));
                     if (tall) {
                         for (int b = 0; b < nblk; ++b)
-                            ptx::tma_load_2d(g_s + b * TC_BLOCK_BYTES, d.tmap, kb * TC_BK, j0 + b * 128, bar_g_full + 8 * s);
+                            ptx::tma_load_2d(g_s + b * TC_BLOCK_BYTES, tmap, kb * TC_BK, j0 + b * 128, bar_g_full + 8 * s);
                     } else {
                         for (int b = 0; b < 2 * nblk; ++b)
-                            ptx::tma_load_2d(g_s + b * (TC_BLOCK_BYTES / 2), d.tmap, j0 + b * 64, kb * TC_BK, bar_g_full + 8 * s);
+                            ptx::tma_load_2d(g_s + b * (TC_BLOCK_BYTES / 2), tmap, j0 + b * 64, kb * TC_BK, bar_g_full + 8 * s);
                     }
                 }
             } else {
@@ -279,11 +296,11 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                     const int row = c >> 3, chunk = c & 7;
                     const uint32_t q0 = (uint32_t)(kb * (TC_BK / 4) + chunk * 2);
                     const uint32_t ka = (uint32_t)(r0 + row), kbrow = ka + 32u;
-                    const uint32_t mid = (uint32_t)d.matrix_id;
-                    const float4 a0 = normal_quad_fast(q0, ka, mid, sp.epoch, sp.key0, sp.key1);
-                    const float4 a1 = normal_quad_fast(q0 + 1, ka, mid, sp.epoch, sp.key0, sp.key1);
-                    const float4 b0 = normal_quad_fast(q0, kbrow, mid, sp.epoch, sp.key0, sp.key1);
-                    const float4 b1 = normal_quad_fast(q0 + 1, kbrow, mid, sp.epoch, sp.key0, sp.key1);
+                    const uint32_t mid = matrix_id;
+                    const float4 a0 = normal_quad_fast(q0, ka, mid, sp.epoch, sp.round_key);
+                    const float4 a1 = normal_quad_fast(q0 + 1, ka, mid, sp.epoch, sp.round_key);
+                    const float4 b0 = normal_quad_fast(q0, kbrow, mid, sp.epoch, sp.round_key);
+                    const float4 b1 = normal_quad_fast(q0 + 1, kbrow, mid, sp.epoch, sp.round_key);
                     uint4 va, vb;
                     va.x = pack_bf16x2(a0.x, a0.y); va.y = pack_bf16x2(a0.z, a0.w);
                     va.z = pack_bf16x2(a1.x, a1.y); va.w = pack_bf16x2(a1.z, a1.w);
@@ -367,8 +384,8 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                 ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * r_slice + cchunk * 16), rv);
                 const int j = j0 + b * 128 + ch_in_blk;
                 if (j < n) {
-                    float* Mp = d.M + (int64_t)(r0 + cchunk * 16) * n + j;
-                    float* Vp = d.V + (int64_t)(r0 + cchunk * 16) * n + j;
+                    float* Mp = Mbase + (int64_t)(r0 + cchunk * 16) * n + j;
+                    float* Vp = Vbase + (int64_t)(r0 + cchunk * 16) * n + j;
                     float mv[16], vv[16];
 #pragma unroll
                     for (int k = 0; k < 16; ++k) { mv[k] = Mp[(int64_t)k * n]; vv[k] = Vp[(int64_t)k * n]; }
@@ -378,7 +395,7 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                         const float mn = sp.beta1 * mv[k] + (1.0f - sp.beta1) * r;
                         const float vn = sp.beta2 * vv[k] + (1.0f - sp.beta2) * r * r;
                         Mp[(int64_t)k * n] = mn; Vp[(int64_t)k * n] = vn;
-                        const float rt = (mn * sp.inv_bc1) / (sqrtf(vn * sp.inv_bc2) + sp.eps);
+                        const float rt = __fdividef(mn * sp.inv_bc1, fast_sqrt(vn * sp.inv_bc2) + sp.eps);
                         num = fmaf(rt, rt, num);
                         den = fmaf(r, r, den);
                     }
@@ -392,11 +409,11 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                 const int j = j0 + ch;
                 if (j < n) {
                     const float2 a = red[ch], b2 = red[chan_tile + ch], c2 = red[2 * chan_tile + ch];
-                    reinterpret_cast<float2*>(d.part)[(int64_t)tr * n + j] = make_float2(a.x + b2.x + c2.x, a.y + b2.y + c2.y);
+                    reinterpret_cast<float2*>(part)[(int64_t)tr * n + j] = make_float2(a.x + b2.x + c2.x, a.y + b2.y + c2.y);
                     if (tr == 0) {
                         float g2 = 0.f;
                         for (int p = 0; p < parts; ++p) g2 += g2s[p * chan_tile + ch];
-                        d.g2[j] = g2;
+                        g2out[j] = g2;
                     }
                 }
             }

@@ -34,6 +34,16 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
     return make_uint4(c0, c1, c2, c3);
 }
 
+// Same function with the ten round keys precomputed (kernel parameters: the additions of the
+// key schedule disappear and the keys are read as constant-bank operands).
+__device__ __forceinline__ uint4 philox4x32_10_keys(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                    const uint32_t (&rk)[20])
+{
+#pragma unroll
+    for (int round = 0; round < 10; ++round) philox_round(c0, c1, c2, c3, rk[2 * round], rk[2 * round + 1]);
+    return make_uint4(c0, c1, c2, c3);
+}
+
 // The top 23 bits of a word as a float in [1, 2): 1 + (x >> 9) / 2^23 (one funnel shift).
 __device__ __forceinline__ float unit_interval_12(uint32_t x)
 {
@@ -83,9 +93,9 @@ __device__ __forceinline__ float4 normal_quad(uint32_t q, uint32_t k, uint32_t m
 // The same quad with the fast transform, for the tensor-core path, which rounds the result
 // to bfloat16 anyway.
 __device__ __forceinline__ float4 normal_quad_fast(uint32_t q, uint32_t k, uint32_t matrix, uint32_t epoch,
-                                                   uint32_t key0, uint32_t key1)
+                                                   const uint32_t (&rk)[20])
 {
-    const uint4 x = philox4x32_10(q, k, matrix, epoch, key0, key1);
+    const uint4 x = philox4x32_10_keys(q, k, matrix, epoch, rk);
     float4 z;
     box_muller(x.x, x.y, z.x, z.y);
     box_muller(x.z, x.w, z.z, z.w);
