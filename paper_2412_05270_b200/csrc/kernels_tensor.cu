@@ -36,6 +36,7 @@ constexpr int TC_EPI_THREADS = 384;       // warps 2-13
 constexpr int TC_BLOCK_BYTES = 128 * TC_BK * 2;   // one 128-channel block of a G stage: 16 KiB
 constexpr int TC_MISC_BYTES = 256 + 3 * 512 * 8 + 8 * 512 * 4 + 1024;   // barriers, red, g2s, alignment slack
 constexpr int TC_MAX_SMEM = 227 * 1024;
+constexpr int TC_PREFETCH = 6;             // k-blocks of G requested into L2 ahead of their load
 constexpr uint32_t TC_WAIT_CAP = 1u << 20;   // polls before a wait gives up (normal waits are far below 1 ms)
 
 TcTiling choose_tiling(int rank)
@@ -238,7 +239,18 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
             // ---------------- TMA producer ----------------
             if (lane == 0) {
                 ptx::fence_tensormap_acquire(tmap);
+                // G tiles are pulled into L2 TC_PREFETCH k-blocks ahead of the load that needs them, so the
+                // load into shared memory sees L2 latency and a shallow ring suffices
+                auto prefetch = [&](int kb) {
+                    if (tall) {
+                        for (int b = 0; b < nblk; ++b) ptx::tma_prefetch_2d(tmap, kb * TC_BK, j0 + b * 128);
+                    } else {
+                        for (int b = 0; b < 2 * nblk; ++b) ptx::tma_prefetch_2d(tmap, j0 + b * 64, kb * TC_BK);
+                    }
+                };
+                for (int kb = 0; kb < TC_PREFETCH && kb < num_kb; ++kb) prefetch(kb);
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    if (kb + TC_PREFETCH < num_kb) prefetch(kb + TC_PREFETCH);
                     const uint32_t s = it % stages, ph = (it / stages) & 1;
                     wait_phase(bar_empty + 8 * s, ph ^ 1, abort_flag, status);
                     const uint32_t g_s = smem_base + s * stage_bytes;
