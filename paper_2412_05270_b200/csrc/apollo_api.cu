@@ -20,13 +20,18 @@ inline size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 struct MatPlan {
     int32_t rows, cols, m, n, tall, path, slices, g2_slices, tiles_n, tiles_k;
     int64_t proj_tiles, update_tiles;
-    size_t off_M, off_V, off_scal, off_s, off_part, off_g2, off_tmap;
+    size_t off_M, off_V, off_scal, off_s, off_part, off_g2, off_tmap, off_pstage;
+};
+
+struct StageGroup {   // matrices whose staged P share one filling of the staging buffer
+    int mat_begin, mat_end, tile_begin, tile_end;
 };
 
 struct Plan {
     std::vector<MatPlan> mats;
-    size_t off_status, off_descs, off_prefix[4], off_tmaps, zero_begin, zero_end, total;
+    size_t off_status, off_descs, off_prefix[4], off_tmaps, off_stage, stage_bytes, zero_begin, zero_end, total;
     int64_t tiles[4];   // stream, simt, tensor, update
+    std::vector<StageGroup> groups;
 };
 
 int validate_config(const apollo_config* cfg)
@@ -98,7 +103,34 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
     plan.off_status = off; off += ALIGN;
     plan.off_descs = off; off = align_up(off + sizeof(MatDesc) * (size_t)n_mat);
     for (int t = 0; t < 4; ++t) { plan.off_prefix[t] = off; off = align_up(off + sizeof(int) * ((size_t)n_mat + 1)); }
-    plan.off_tmaps = off; off = align_up(off + 128 * (size_t)n_mat);
+    plan.off_tmaps = off; off = align_up(off + 256 * (size_t)n_mat);
+    // staging groups: consecutive matrices whose P fit the staging budget together
+    plan.groups.clear();
+    plan.stage_bytes = 0;
+    {
+        const size_t budget = tensor_path_stage_budget();
+        StageGroup g = { 0, 0, 0, 0 };
+        size_t used = 0;
+        int tile_at = 0;
+        for (int i = 0; i < n_mat; ++i) {
+            MatPlan& p = plan.mats[i];
+            const bool tensor = p.path == PATH_TENSOR;
+            const size_t need = tensor && tensor_path_staged() ? align_up(tensor_path_stage_bytes(p.rows, p.cols, r)) : 0;
+            if (used > 0 && used + need > budget) {
+                g.mat_end = i; g.tile_end = tile_at;
+                plan.groups.push_back(g);
+                g.mat_begin = i; g.tile_begin = tile_at;
+                used = 0;
+            }
+            p.off_pstage = used;
+            used += need;
+            if (used > plan.stage_bytes) plan.stage_bytes = used;
+            if (tensor) tile_at += (int)p.proj_tiles;
+        }
+        g.mat_end = n_mat; g.tile_end = tile_at;
+        plan.groups.push_back(g);
+    }
+    plan.off_stage = off; off = align_up(off + plan.stage_bytes);
     plan.zero_begin = off;
     for (int i = 0; i < n_mat; ++i) {
         MatPlan& p = plan.mats[i];
@@ -113,7 +145,7 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
         p.off_s = off; off = align_up(off + sizeof(float) * (size_t)p.n);
         p.off_part = off; off = align_up(off + sizeof(float) * 2 * (size_t)p.slices * (size_t)p.n);
         p.off_g2 = off; off = align_up(off + sizeof(float) * (size_t)(p.g2_slices > 0 ? p.g2_slices : 1) * (size_t)p.n);
-        p.off_tmap = plan.off_tmaps + 128 * (size_t)i;
+        p.off_tmap = plan.off_tmaps + 256 * (size_t)i;
     }
     plan.total = off;
     return APOLLO_OK;
@@ -230,6 +262,9 @@ int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_ma
         d.part = reinterpret_cast<float*>(ctx->ws + p.off_part);
         d.g2 = reinterpret_cast<float*>(ctx->ws + p.off_g2);
         d.tmap = ctx->ws + p.off_tmap;
+        d.tmap_p = ctx->ws + p.off_tmap + 128;
+        d.pstage = ctx->ws + ctx->plan.off_stage + p.off_pstage;
+        d.m_pad = (p.m + 63) / 64 * 64;
         d.rows = p.rows; d.cols = p.cols; d.m = p.m; d.n = p.n; d.tall = p.tall; d.path = p.path;
         d.slices = p.slices; d.g2_slices = p.g2_slices; d.matrix_id = i;
         d.tiles_n = p.tiles_n; d.tiles_k = p.tiles_k;
@@ -353,8 +388,16 @@ int apollo_step(apollo_ctx* ctx, void* const* d_W, const void* const* d_G, float
         ++launches;
     }
     if (plan.tiles[PATH_TENSOR] > 0) {
-        launches += launch_project_tensor(ctx->d_descs, ctx->d_prefix[PATH_TENSOR], ctx->n_mat,
-                                          (int)plan.tiles[PATH_TENSOR], sp, ctx->sm_count, ctx->d_status, stream);
+        for (const StageGroup& g : plan.groups) {
+            if (g.tile_end <= g.tile_begin) continue;
+            if (tensor_path_staged()) {
+                launch_generate_p(ctx->d_descs, g.mat_begin, g.mat_end, sp, stream);
+                ++launches;
+            }
+            launch_project_tensor(ctx->d_descs, ctx->d_prefix[PATH_TENSOR], ctx->n_mat, g.tile_begin, g.tile_end, sp,
+                                  ctx->sm_count, ctx->d_status, stream);
+            ++launches;
+        }
     }
     if (ev) cudaEventRecord(ev[1], stream);
     launch_finalize(ctx->d_descs, ctx->n_mat, sp, stream);

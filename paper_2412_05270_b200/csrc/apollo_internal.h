@@ -34,6 +34,8 @@ struct MatDesc {
     float* scal;      // {norm after limiting, c, norm before limiting, tensor-wise s}
     float* prev;      // previous limited norm (one float)
     const void* tmap; // 128-byte TMA tensor map of G in device memory (tensor path only)
+    const void* tmap_p; // tensor map of the staged P (tensor path with L2 staging)
+    void* pstage;     // this matrix's r x m_pad bf16 standard normals in the staging buffer
     int32_t rows, cols;
     int32_t m, n;     // m = min(rows, cols) = projected side; n = max = number of channels
     int32_t tall;     // 1 if rows > cols: channels are the stored rows
@@ -43,7 +45,7 @@ struct MatDesc {
     int32_t matrix_id;
     int32_t tiles_n;  // projection tiles along the channels
     int32_t tiles_k;  // projection tiles along the other tiled axis (rows of G, or rows of R)
-    int32_t pad0;
+    int32_t m_pad;    // m rounded up to 64: row length of the staged P
 };
 
 struct StepParams {
@@ -71,6 +73,7 @@ struct TcTiling {
     int32_t nblk;      // 128-channel blocks per tile (1, 2 or 4); nblk * r_slice <= 512 TMEM columns
     int32_t stages;    // shared-memory pipeline depth
     int32_t smem_bytes;
+    int32_t staged;    // 1: P tiles come from the L2 staging buffer by TMA; 0: generated in shared memory
 };
 
 // Device status word values.

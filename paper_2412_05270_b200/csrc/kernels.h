@@ -20,11 +20,18 @@ void launch_update(int dtype, const MatDesc* d_descs, const int* d_prefix, int n
 // Tensor-core projection (TMA + tcgen05 + TMEM).
 bool tensor_path_supports(int rows, int cols, int rank, int dtype);
 void tensor_path_tiling(int rows, int cols, int rank, int32_t* tiles_n, int32_t* tiles_k);
-// Encodes the tensor maps of the matrices on the tensor path into the host copies and
-// queues their upload to `d_tmaps` (128 bytes per matrix).  Returns an APOLLO_* code.
+// L2 staging of P: whether it is on, the byte budget of the staging buffer, and the bytes
+// one matrix needs in it (rank x round_up(m, 64) bf16).
+bool tensor_path_staged();
+size_t tensor_path_stage_budget();
+size_t tensor_path_stage_bytes(int rows, int cols, int rank);
+// Encodes the tensor maps of the matrices on the tensor path (G at +0, staged P at +128 of
+// each 256-byte slot) and queues their upload to `d_tmaps`.  Returns an APOLLO_* code.
 int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, void* d_tmaps, cudaStream_t stream);
-// Returns the number of launches issued.
-int launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_mat, int total_tiles,
-                          const StepParams& sp, int sm_count, int32_t* d_status, cudaStream_t stream);
+// Fills the staging buffer with the standard normals of matrices [mat_begin, mat_end).
+void launch_generate_p(const MatDesc* d_descs, int mat_begin, int mat_end, const StepParams& sp, cudaStream_t stream);
+// Projection over tiles [tile_begin, tile_end) of the tensor-path prefix table.
+void launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_mat, int tile_begin, int tile_end,
+                           const StepParams& sp, int sm_count, int32_t* d_status, cudaStream_t stream);
 
 }  // namespace apollo

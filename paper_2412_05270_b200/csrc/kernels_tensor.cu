@@ -57,6 +57,7 @@ TcTiling choose_tiling(int rank)
     t.stages = (TC_MAX_SMEM - TC_MISC_BYTES) / stage;
     if (t.stages > 4) t.stages = 4;
     t.smem_bytes = t.stages * stage + TC_MISC_BYTES;
+    t.staged = tensor_path_staged() ? 1 : 0;
     return t;
 }
 
@@ -79,6 +80,30 @@ EncodeTiledFn encode_fn()
 
 }  // namespace
 
+// P tiles either come from a per-step staging buffer that stays in L2 (default) or are
+// generated in shared memory by every CTA that needs them (APOLLO_P_STAGING=0).
+bool tensor_path_staged()
+{
+    const char* env = std::getenv("APOLLO_P_STAGING");
+    return !(env && env[0] == '0');
+}
+
+size_t tensor_path_stage_budget()
+{
+    size_t mb = 512;
+    if (const char* env = std::getenv("APOLLO_P_STAGING_MB")) {
+        const long v = std::atol(env);
+        if (v >= 1 && v <= 65536) mb = (size_t)v;
+    }
+    return mb << 20;
+}
+
+size_t tensor_path_stage_bytes(int rows, int cols, int rank)
+{
+    const int m = rows > cols ? cols : rows;
+    return (size_t)rank * (size_t)((m + 63) / 64 * 64) * 2;
+}
+
 bool tensor_path_supports(int rows, int cols, int rank, int dtype)
 {
     if (dtype != APOLLO_DT_BF16) return false;
@@ -99,14 +124,14 @@ void tensor_path_tiling(int rows, int cols, int rank, int32_t* tiles_n, int32_t*
 
 int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, void* d_tmaps, cudaStream_t stream)
 {
-    (void)rank;
+    const TcTiling tl = choose_tiling(rank);
     bool any = false;
     for (int i = 0; i < n_mat; ++i) any |= h_descs[i].path == PATH_TENSOR;
     if (!any) return APOLLO_OK;
     EncodeTiledFn encode = encode_fn();
     if (!encode) return APOLLO_ERR_CUDA;
-    std::vector<CUtensorMap> maps(n_mat);
-    std::memset(maps.data(), 0, sizeof(CUtensorMap) * n_mat);
+    std::vector<CUtensorMap> maps(2 * (size_t)n_mat);
+    std::memset(maps.data(), 0, sizeof(CUtensorMap) * maps.size());
     for (int i = 0; i < n_mat; ++i) {
         const MatDesc& d = h_descs[i];
         if (d.path != PATH_TENSOR) continue;
@@ -116,13 +141,23 @@ int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, void* d_tmaps, cu
         // wide: 64 channels x 64 rows of G; tall: 64 contraction elements x 128 channels
         const cuuint32_t box[2] = { 64u, d.tall ? 128u : 64u };
         const cuuint32_t elem[2] = { 1u, 1u };
-        const CUresult rc = encode(&maps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(d.G), dims,
+        const CUresult rc = encode(&maps[2 * i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(d.G), dims,
                                    strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (rc != CUDA_SUCCESS) return APOLLO_ERR_CUDA;
+        if (tl.staged) {
+            // staged P: rank rows of m_pad bf16, loaded as 64 x r_slice boxes (K-major UMMA tiles)
+            const cuuint64_t pdims[2] = { (cuuint64_t)d.m_pad, (cuuint64_t)rank };
+            const cuuint64_t pstrides[1] = { (cuuint64_t)d.m_pad * 2 };
+            const cuuint32_t pbox[2] = { 64u, (cuuint32_t)tl.r_slice };
+            const CUresult rp = encode(&maps[2 * i + 1], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, d.pstage, pdims, pstrides,
+                                       pbox, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (rp != CUDA_SUCCESS) return APOLLO_ERR_CUDA;
+        }
     }
     static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
-    if (cudaMemcpyAsync(d_tmaps, maps.data(), sizeof(CUtensorMap) * n_mat, cudaMemcpyHostToDevice, stream) !=
+    if (cudaMemcpyAsync(d_tmaps, maps.data(), sizeof(CUtensorMap) * maps.size(), cudaMemcpyHostToDevice, stream) !=
         cudaSuccess)
         return APOLLO_ERR_CUDA;
     return APOLLO_OK;
@@ -174,14 +209,15 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, const uint4& v)
 
 // 14 warps are allocated as 16: 128 registers per thread is the ceiling
 __global__ void __launch_bounds__(TC_THREADS, 1)
-project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix, int n_mat, int total_tiles,
-                      StepParams sp, TcTiling tl, int32_t* __restrict__ status)
+project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix, int n_mat, int tile_begin,
+                      int tile_end, StepParams sp, TcTiling tl, int32_t* __restrict__ status)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_addr(smem_raw));
 
     const int r_slice = tl.r_slice, nblk = tl.nblk, stages = tl.stages;
+    const bool staged = tl.staged != 0;
     const uint32_t stage_bytes = (uint32_t)(nblk * TC_BLOCK_BYTES + r_slice * 128);
     const uint32_t p_off = (uint32_t)(nblk * TC_BLOCK_BYTES);
     const uint32_t bars = smem_base + stages * stage_bytes;          // 8-byte mbarriers
@@ -216,7 +252,7 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
     uint32_t it = 0;          // k-block counter across tiles: stage = it % stages, phase = (it / stages) & 1
     uint32_t tile_iter = 0;   // tiles done by this CTA: phase of the accumulator barrier
 
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tile_iter) {
+    for (int tile = tile_begin + blockIdx.x; tile < tile_end; tile += gridDim.x, ++tile_iter) {
         const int mat = find_matrix(prefix, n_mat, tile);
         // copy what the roles need into registers: the descriptor lives in global memory and
         // every shared-memory asm below is a compiler memory barrier
@@ -226,6 +262,7 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
         const bool tall = __ldg(&dp->tall) != 0;
         const uint32_t matrix_id = (uint32_t)__ldg(&dp->matrix_id);
         const void* tmap = dp->tmap;
+        const void* tmap_p = dp->tmap_p;
         float* const Mbase = dp->M;
         float* const Vbase = dp->V;
         float* const part = dp->part;
@@ -239,6 +276,7 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
             // ---------------- TMA producer ----------------
             if (lane == 0) {
                 ptx::fence_tensormap_acquire(tmap);
+                if (staged) ptx::fence_tensormap_acquire(tmap_p);
                 // G tiles are pulled into L2 TC_PREFETCH k-blocks ahead of the load that needs them, so the
                 // load into shared memory sees L2 latency and a shallow ring suffices
                 auto prefetch = [&](int kb) {
@@ -254,7 +292,9 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                     const uint32_t s = it % stages, ph = (it / stages) & 1;
                     wait_phase(bar_empty + 8 * s, ph ^ 1, abort_flag, status);
                     const uint32_t g_s = smem_base + s * stage_bytes;
-                    ptx::mbar_arrive_expect_tx(bar_g_full + 8 * s, (uint32_t)(nblk * TC_BLOCK_BYTES));
+                    ptx::mbar_arrive_expect_tx(bar_g_full + 8 * s,
+                                               (uint32_t)(nblk * TC_BLOCK_BYTES + (staged ? r_slice * 128 : 0)));
+                    if (staged) ptx::tma_load_2d(g_s + p_off, tmap_p, kb * TC_BK, r0, bar_g_full + 8 * s);
                     if (tall) {
                         for (int b = 0; b < nblk; ++b)
                             ptx::tma_load_2d(g_s + b * TC_BLOCK_BYTES, tmap, kb * TC_BK, j0 + b * 128, bar_g_full + 8 * s);
@@ -274,7 +314,7 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
                     const uint32_t s = it % stages, ph = (it / stages) & 1;
                     wait_phase(bar_g_full + 8 * s, ph, abort_flag, status);
-                    wait_phase(bar_p_full + 8 * s, ph, abort_flag, status);
+                    if (!staged) wait_phase(bar_p_full + 8 * s, ph, abort_flag, status);
                     ptx::tc_fence_after_sync();
                     const uint32_t g_s = smem_base + s * stage_bytes, p_s = g_s + p_off;
                     for (int b = 0; b < nblk; ++b) {
@@ -298,7 +338,8 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
         } else if (warp < 10) {
             // ---------------- generators: P tile for every k-block ----------------
             const int g = tid - 64;
-            for (int kb = 0; kb < num_kb; ++kb, ++it) {
+            if (staged) it += num_kb;     // P arrives by TMA from the staging buffer
+            for (int kb = 0; kb < num_kb && !staged; ++kb, ++it) {
                 const uint32_t s = it % stages, ph = (it / stages) & 1;
                 wait_phase(bar_empty + 8 * s, ph ^ 1, abort_flag, status);
                 const uint32_t p_s = smem_base + s * stage_bytes + p_off;
@@ -443,22 +484,50 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
     if (warp == 1) ptx::tmem_dealloc(tmem_base, 512);
 }
 
+// Standard normals of the staged P: one 16-byte store (8 bf16) per thread and pass.
+__global__ void generate_p_kernel(const MatDesc* __restrict__ descs, int mat_begin, StepParams sp)
+{
+    const MatDesc* dp = descs + mat_begin + blockIdx.y;
+    if (__ldg(&dp->path) != PATH_TENSOR) return;
+    const int m_pad = __ldg(&dp->m_pad);
+    const uint32_t matrix_id = (uint32_t)__ldg(&dp->matrix_id);
+    uint4* out = static_cast<uint4*>(dp->pstage);
+    const int chunks_per_row = m_pad / 8;
+    const int total = sp.rank * chunks_per_row;
+    for (int c = blockIdx.x * blockDim.x + threadIdx.x; c < total; c += gridDim.x * blockDim.x) {
+        const int row = c / chunks_per_row, ch = c - row * chunks_per_row;
+        const float4 a0 = normal_quad_fast((uint32_t)(2 * ch), (uint32_t)row, matrix_id, sp.epoch, sp.round_key);
+        const float4 a1 = normal_quad_fast((uint32_t)(2 * ch + 1), (uint32_t)row, matrix_id, sp.epoch, sp.round_key);
+        uint4 v;
+        v.x = pack_bf16x2(a0.x, a0.y); v.y = pack_bf16x2(a0.z, a0.w);
+        v.z = pack_bf16x2(a1.x, a1.y); v.w = pack_bf16x2(a1.z, a1.w);
+        out[c] = v;
+    }
+}
+
 }  // namespace
 
-int launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_mat, int total_tiles,
-                          const StepParams& sp, int sm_count, int32_t* d_status, cudaStream_t stream)
+void launch_generate_p(const MatDesc* d_descs, int mat_begin, int mat_end, const StepParams& sp, cudaStream_t stream)
 {
-    if (total_tiles <= 0) return 0;
+    if (mat_end <= mat_begin) return;
+    const dim3 grid(64, (unsigned)(mat_end - mat_begin));
+    generate_p_kernel<<<grid, 256, 0, stream>>>(d_descs, mat_begin, sp);
+}
+
+void launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_mat, int tile_begin, int tile_end,
+                           const StepParams& sp, int sm_count, int32_t* d_status, cudaStream_t stream)
+{
+    const int tiles = tile_end - tile_begin;
+    if (tiles <= 0) return;
     const TcTiling tl = choose_tiling(sp.rank);
     static bool attr_set = false;
     if (!attr_set) {
         cudaFuncSetAttribute(project_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
         attr_set = true;
     }
-    const int grid = total_tiles < sm_count ? total_tiles : sm_count;
-    project_tensor_kernel<<<grid, TC_THREADS, tl.smem_bytes, stream>>>(d_descs, d_prefix, n_mat, total_tiles, sp, tl,
-                                                                     d_status);
-    return 1;
+    const int grid = tiles < sm_count ? tiles : sm_count;
+    project_tensor_kernel<<<grid, TC_THREADS, tl.smem_bytes, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end, sp,
+                                                                     tl, d_status);
 }
 
 }  // namespace apollo
