@@ -132,7 +132,8 @@ APOLLO_API int apollo_get_state(apollo_ctx* ctx, int32_t matrix, float* d_M, flo
 /*
  * Optional capture of the fp32 update dW = -lr (alpha c s_j G_ij + wd W_ij) before it is
  * added to W and rounded (the quantity the parity bound is stated on).  d_dW: HOST array
- * of n_matrices DEVICE pointers (rows x cols floats each), or NULL to switch capture off.
+ * of n_matrices DEVICE pointers (rows x cols floats each; a null entry leaves that matrix
+ * uncaptured), or NULL to switch capture off.
  */
 APOLLO_API int apollo_set_delta_out(apollo_ctx* ctx, float* const* d_dW);
 

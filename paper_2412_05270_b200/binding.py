@@ -218,13 +218,16 @@ class Apollo:
         _check(self.lib.apollo_step(self.ctx, self._w_arr, self._g_arr, lr, wd, _stream_ptr(stream)), "apollo_step")
 
     def set_delta_out(self, deltas):
-        """deltas: list of float32 CUDA tensors shaped like the weights, or None."""
+        """deltas: list of float32 CUDA tensors shaped like the weights (None entries skip a matrix), or None."""
         if deltas is None:
             _check(self.lib.apollo_set_delta_out(self.ctx, None), "apollo_set_delta_out")
             self._delta = None
             return
         arr = (ctypes.c_void_p * len(self.shapes))()
         for i, d in enumerate(deltas):
+            if d is None:
+                arr[i] = None
+                continue
             assert d.is_cuda and d.dtype == torch.float32 and tuple(d.shape) == self.shapes[i] and d.is_contiguous()
             arr[i] = d.data_ptr()
         _check(self.lib.apollo_set_delta_out(self.ctx, arr), "apollo_set_delta_out")

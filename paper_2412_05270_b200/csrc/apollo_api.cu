@@ -305,10 +305,8 @@ int apollo_set_delta_out(apollo_ctx* ctx, float* const* d_dW)
 {
     if (!ctx) return APOLLO_ERR_INVALID_ARG;
     if (d_dW) {
-        for (int i = 0; i < ctx->n_mat; ++i) {
-            if (!d_dW[i]) return APOLLO_ERR_INVALID_ARG;
-            if ((uintptr_t)d_dW[i] % 16) return APOLLO_ERR_ALIGN;
-        }
+        for (int i = 0; i < ctx->n_mat; ++i)
+            if ((uintptr_t)d_dW[i] % 16) return APOLLO_ERR_ALIGN;   // a null entry skips that matrix
         for (int i = 0; i < ctx->n_mat; ++i) ctx->delta[i] = d_dW[i];
         ctx->delta_on = true;
     } else {

@@ -39,8 +39,11 @@ def oracle_of(wl: WL.Workload, mats=None, bias_correction=False):
 
 
 def run_parity(wl: WL.Workload, steps=None, flags=0, bias_correction=False, check_mats=None, expect_path=None,
-               grad_fn=None):
-    """Steps the whole list on the GPU and the matrices in `check_mats` on the oracle."""
+               grad_fn=None, gen_device="cpu"):
+    """Steps the whole list on the GPU and the matrices in `check_mats` on the oracle.
+
+    With gen_device="cuda" the inputs are drawn on the GPU (large lists) and only the checked
+    matrices are copied to the host for the oracle."""
     steps = wl.steps if steps is None else steps
     n = len(wl.shapes)
     check_mats = list(range(n)) if check_mats is None else list(check_mats)
@@ -49,21 +52,21 @@ def run_parity(wl: WL.Workload, steps=None, flags=0, bias_correction=False, chec
     if expect_path is not None:
         for i in check_mats:
             assert opt.path(i) == expect_path, (i, opt.path(i))
-    Wc = [WL.make_weight(wl, i) for i in range(n)]
-    Wg = [w.to(dev) for w in Wc]
-    deltas = [torch.zeros(s, dtype=torch.float32, device=dev) for s in wl.shapes]
+    Wg = [WL.make_weight(wl, i, device=gen_device).to(dev) for i in range(n)]
+    deltas = [torch.zeros(wl.shapes[i], dtype=torch.float32, device=dev) if i in check_mats else None
+              for i in range(n)]
     opt.set_delta_out(deltas)
     orc = oracle_of(wl, check_mats, bias_correction)
-    Wo = {i: Wc[i].float().numpy() for i in check_mats}
+    Wo = {i: Wg[i].float().cpu().numpy() for i in check_mats}
     worst = {"dw": 0.0, "s": 0.0}
     for t in range(steps):
-        Gc = [(grad_fn or WL.make_grad)(wl, i, t) for i in range(n)]
-        Gg = [g.to(dev) for g in Gc]
+        Gg = [(grad_fn(wl, i, t) if grad_fn else WL.make_grad(wl, i, t, device=gen_device)).to(dev)
+              for i in range(n)]
         W_before = {i: Wg[i].clone() for i in check_mats}
         opt.step(Wg, Gg, wl.lr, wl.wd)
         assert opt.status() == B.OK
         for i in check_mats:
-            res = orc[i].step(Wo[i], Gc[i].float().numpy(), _f32(wl.lr), _f32(wl.wd), want_R=True)
+            res = orc[i].step(Wo[i], Gg[i].float().cpu().numpy(), _f32(wl.lr), _f32(wl.wd), want_R=True)
             dw_gpu = deltas[i].cpu().numpy().astype(np.float64)
             bound = DW_REL * np.max(np.abs(res.dW)) + DW_ABS
             err = np.max(np.abs(dw_gpu - res.dW))
@@ -96,6 +99,7 @@ def run_parity(wl: WL.Workload, steps=None, flags=0, bias_correction=False, chec
             Wo[i] = res.W
             # keep the two weight trajectories identical so that errors do not compound through wd
             Wg[i].copy_(torch.from_numpy(res.W).to(Wg[i].dtype))
+        del Gg
     assert opt.step_count() == steps
     opt.close()
     return worst
