@@ -51,6 +51,25 @@ def step_bytes(wl: WL.Workload):
     return two_pass, minimal, update, flops
 
 
+def max_over_ranks(values, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_value(params_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Parameters per second over all replicas (every rank steps its own copy of the list)."""
+    return world * params_per_rank / (ms_per_step * 1e-3)
+
+
+# DRAM bytes per parameter of update_kernel<bf16> from its ncu capture (profiles/update_kernel_*.md);
+# set to None when the kernel changes until the counters are taken again.
+UPDATE_TRAFFIC_BYTES_PER_PARAM = 5.88
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
     QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -205,10 +224,7 @@ def run_ours(args, wl, rank, world, local_rank):
         barrier()
         e2e_ms = s2.elapsed_time(e2) / e2e_steps
         del host_G
-    times = torch.tensor([ms_total, e2e_ms if not args.no_e2e else 0.0], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_total, e2e_ms = times.tolist()
+    ms_total, e2e_ms = max_over_ranks([ms_total, e2e_ms if not args.no_e2e else 0.0], device=dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -217,7 +233,7 @@ def run_ours(args, wl, rank, world, local_rank):
     peaks = measured_peaks()
     ms_step = ms_total / args.steps
     two_pass, minimal, update_bytes, flops = step_bytes(wl)
-    value = world * wl.params / (ms_step * 1e-3)
+    value = whole_job_value(wl.params, world, ms_step)
     hbm, tc = peaks["hbm_gbs"] * 1e9, peaks["bf16_tflops_sustained"] * 1e12
     t_roof = max(two_pass / hbm, flops / tc)
     upd_gbs = update_bytes / (upd_ms * 1e-3) / 1e9
@@ -230,7 +246,9 @@ def run_ours(args, wl, rank, world, local_rank):
                    "T": wl.T, "lr": wl.lr, "wd": wl.wd, "states": "f32", "replicas": world,
                    "l2": "inputs (W, G: %.1f GB) exceed L2, no flush" % (2 * wl.params * 2 / 1e9)},
         "roofline": {"bound": "hbm", "kernel": "update_kernel", "achieved": upd_gbs, "peak": peaks["hbm_gbs"],
-                     "unit": "GB/s", "frac": upd_gbs / peaks["hbm_gbs"], "traffic": None,
+                     "unit": "GB/s", "frac": upd_gbs / peaks["hbm_gbs"],
+                     "traffic": (UPDATE_TRAFFIC_BYTES_PER_PARAM * wl.params
+                                 if UPDATE_TRAFFIC_BYTES_PER_PARAM and wl.dtype == "bf16" else None),
                      "peak_source": peaks["source"], "bytes_per_launch": update_bytes, "ms_per_launch": upd_ms},
         "step_roofline": {"bytes_two_pass": two_pass, "bytes_min": minimal, "gemm_flops": flops,
                           "t_roofline_ms": 1e3 * t_roof, "frac": 1e3 * t_roof / ms_step,
@@ -240,7 +258,7 @@ def run_ours(args, wl, rank, world, local_rank):
         "gpu_launches": launches,
     }
     if not args.no_e2e:
-        line["e2e"] = {"value": world * wl.params / (e2e_ms * 1e-3), "unit": "params/s",
+        line["e2e"] = {"value": whole_job_value(wl.params, world, e2e_ms), "unit": "params/s",
                        "h2d_bytes_per_step": g_bytes, "d2h_bytes_per_step": n * 16, "ms_per_step": e2e_ms}
     if world == 1 and not args.no_cpu:
         base = cpu_baseline(wl)
