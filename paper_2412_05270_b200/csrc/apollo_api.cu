@@ -20,7 +20,7 @@ inline size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 struct MatPlan {
     int32_t rows, cols, m, n, tall, path, slices, g2_slices, tiles_n, tiles_k;
     int64_t proj_tiles, update_tiles;
-    size_t off_M, off_V, off_scal, off_s, off_part, off_g2, off_tmap, off_pstage;
+    size_t off_M, off_V, off_scal, off_s, off_part, off_g2, off_tmap, off_pstage, off_gpad, gpad_bytes;
 };
 
 struct StageGroup {   // matrices whose staged P share one filling of the staging buffer
@@ -30,6 +30,7 @@ struct StageGroup {   // matrices whose staged P share one filling of the stagin
 struct Plan {
     std::vector<MatPlan> mats;
     size_t off_status, off_descs, off_prefix[4], off_tmaps, off_stage, stage_bytes, zero_begin, zero_end, total;
+    bool any_repitch;
     int64_t tiles[4];   // stream, simt, tensor, update
     std::vector<StageGroup> groups;
 };
@@ -131,6 +132,17 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
         plan.groups.push_back(g);
     }
     plan.off_stage = off; off = align_up(off + plan.stage_bytes);
+    // padded copies of the gradients whose row pitch TMA cannot take (cols not a multiple of 8)
+    plan.any_repitch = false;
+    for (int i = 0; i < n_mat; ++i) {
+        MatPlan& p = plan.mats[i];
+        p.gpad_bytes = 0;
+        if (p.path == PATH_TENSOR && (p.cols % 8) != 0) {
+            p.gpad_bytes = (size_t)p.rows * (size_t)((p.cols + 7) / 8 * 8) * 2;
+            plan.any_repitch = true;
+        }
+        p.off_gpad = off; off = align_up(off + p.gpad_bytes);
+    }
     plan.zero_begin = off;
     for (int i = 0; i < n_mat; ++i) {
         MatPlan& p = plan.mats[i];
@@ -265,6 +277,8 @@ int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_ma
         d.tmap_p = ctx->ws + p.off_tmap + 128;
         d.pstage = ctx->ws + ctx->plan.off_stage + p.off_pstage;
         d.m_pad = (p.m + 63) / 64 * 64;
+        d.gpad = p.gpad_bytes ? ctx->ws + p.off_gpad : nullptr;
+        d.g_pitch = p.gpad_bytes ? (p.cols + 7) / 8 * 8 : p.cols;
         d.rows = p.rows; d.cols = p.cols; d.m = p.m; d.n = p.n; d.tall = p.tall; d.path = p.path;
         d.slices = p.slices; d.g2_slices = p.g2_slices; d.matrix_id = i;
         d.tiles_n = p.tiles_n; d.tiles_k = p.tiles_k;
@@ -386,6 +400,10 @@ int apollo_step(apollo_ctx* ctx, void* const* d_W, const void* const* d_G, float
         ++launches;
     }
     if (plan.tiles[PATH_TENSOR] > 0) {
+        if (plan.any_repitch) {
+            launch_repitch(ctx->d_descs, ctx->n_mat, stream);
+            ++launches;
+        }
         for (const StageGroup& g : plan.groups) {
             if (g.tile_end <= g.tile_begin) continue;
             if (tensor_path_staged()) {

@@ -28,6 +28,8 @@ size_t tensor_path_stage_bytes(int rows, int cols, int rank);
 // Encodes the tensor maps of the matrices on the tensor path (G at +0, staged P at +128 of
 // each 256-byte slot) and queues their upload to `d_tmaps`.  Returns an APOLLO_* code.
 int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, void* d_tmaps, cudaStream_t stream);
+// Copies the gradients whose row pitch is not a multiple of 16 bytes into their padded buffers.
+void launch_repitch(const MatDesc* d_descs, int n_mat, cudaStream_t stream);
 // Fills the staging buffer with the standard normals of matrices [mat_begin, mat_end).
 void launch_generate_p(const MatDesc* d_descs, int mat_begin, int mat_end, const StepParams& sp, cudaStream_t stream);
 // Projection over tiles [tile_begin, tile_end) of the tensor-path prefix table.

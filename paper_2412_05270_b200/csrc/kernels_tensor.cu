@@ -125,8 +125,7 @@ bool tensor_path_supports(int rows, int cols, int rank, int dtype)
     if (dtype != APOLLO_DT_BF16) return false;
     if (rank < 16 || rank > 512 || rank % 16) return false;
     if (rank > 256 && rank % 32) return false;
-    if (cols % 8) return false;                      // TMA needs a 16-byte row pitch
-    (void)rows;
+    (void)rows; (void)cols;   // a row pitch that is not a multiple of 16 bytes goes through a padded copy
     return true;
 }
 
@@ -153,11 +152,12 @@ int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, void* d_tmaps, cu
         if (d.path != PATH_TENSOR) continue;
         // dimension 0 is the contiguous one (the stored columns)
         const cuuint64_t dims[2] = { (cuuint64_t)d.cols, (cuuint64_t)d.rows };
-        const cuuint64_t strides[1] = { (cuuint64_t)d.cols * 2 };
+        const cuuint64_t strides[1] = { (cuuint64_t)d.g_pitch * 2 };
         // wide: 64 channels x 64 rows of G; tall: 64 contraction elements x 128 channels
         const cuuint32_t box[2] = { 64u, d.tall ? 128u : 64u };
         const cuuint32_t elem[2] = { 1u, 1u };
-        const CUresult rc = encode(&maps[2 * i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(d.G), dims,
+        const CUresult rc = encode(&maps[2 * i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                                   d.gpad ? d.gpad : const_cast<void*>(d.G), dims,
                                    strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (rc != CUDA_SUCCESS) return APOLLO_ERR_CUDA;
@@ -1015,6 +1015,28 @@ __global__ void generate_p_kernel(const MatDesc* __restrict__ descs, int mat_beg
 }
 
 }  // namespace
+
+// G with an odd row pitch -> copy with the pitch rounded up to 8 elements (TMA needs 16-byte rows).
+__global__ void repitch_kernel(const MatDesc* __restrict__ descs)
+{
+    const MatDesc* dp = descs + blockIdx.y;
+    unsigned short* dst = static_cast<unsigned short*>(dp->gpad);
+    if (!dst) return;
+    const unsigned short* __restrict__ src = static_cast<const unsigned short*>(dp->G);
+    const int cols = __ldg(&dp->cols), pitch = __ldg(&dp->g_pitch);
+    const int64_t total = (int64_t)__ldg(&dp->rows) * cols;
+    for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = e / cols;
+        dst[row * pitch + (e - row * cols)] = __ldg(src + e);
+    }
+}
+
+void launch_repitch(const MatDesc* d_descs, int n_mat, cudaStream_t stream)
+{
+    if (n_mat <= 0) return;
+    const dim3 grid(128, (unsigned)n_mat);
+    repitch_kernel<<<grid, 256, 0, stream>>>(d_descs);
+}
 
 void launch_generate_p(const MatDesc* d_descs, int mat_begin, int mat_end, const StepParams& sp, cudaStream_t stream)
 {

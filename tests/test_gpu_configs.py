@@ -34,7 +34,7 @@ def test_llama1b_rank512_with_the_unaligned_intermediate_size():
     wl.T = 2
     opt_paths = B.Apollo(wl.shapes, B.config_for(wl))
     assert opt_paths.path(0) == B.PATH_TENSOR and opt_paths.path(6) == B.PATH_TENSOR
-    assert opt_paths.path(4) == B.PATH_SIMT    # 5461 columns: the row pitch is not a multiple of 16 bytes
+    assert opt_paths.path(4) == B.PATH_TENSOR  # 5461 columns: read through a copy with a 16-byte row pitch
     opt_paths.close()
     worst = run_parity(wl, steps=4, check_mats=[0, 4, 6], gen_device="cuda")
     assert worst["dw"] <= 1.0

@@ -58,6 +58,7 @@ def test_streaming_path_spanning_row_blocks_and_column_tiles():
     (256, [(512, 1376), (1376, 512), (512, 512)]),
     (512, [(512, 1376), (1376, 512)]),
     (48, [(96, 200), (200, 96)]),
+    (32, [(200, 333), (336, 203), (64, 77)]),      # row pitch not a multiple of 16 bytes: padded copy
 ])
 def test_tensor_core_path(rank, shapes):
     wl = _wl(shapes, rank, dtype="bf16", steps=4, T=2, wd=0.01)
