@@ -72,6 +72,30 @@ __device__ __forceinline__ void load8_stream(const __nv_bfloat16* p, float (&v)[
     unpack_bf16x8(raw, v);
 }
 
+// Eight elements as loaded (16 bytes of bf16 / 32 bytes of fp32), unpacked only when used, so that
+// many loads can be in flight per thread without holding eight floats each.
+template <typename T> struct Raw8;
+template <> struct Raw8<float> { float4 a, b; };
+template <> struct Raw8<__nv_bfloat16> { uint4 v; };
+__device__ __forceinline__ Raw8<float> load_raw8_stream(const float* p)
+{
+    Raw8<float> r;
+    r.a = __ldcs(reinterpret_cast<const float4*>(p));
+    r.b = __ldcs(reinterpret_cast<const float4*>(p) + 1);
+    return r;
+}
+__device__ __forceinline__ Raw8<__nv_bfloat16> load_raw8_stream(const __nv_bfloat16* p)
+{
+    Raw8<__nv_bfloat16> r;
+    r.v = __ldcs(reinterpret_cast<const uint4*>(p));
+    return r;
+}
+__device__ __forceinline__ void unpack_raw8(const Raw8<float>& r, float (&v)[8])
+{
+    v[0] = r.a.x; v[1] = r.a.y; v[2] = r.a.z; v[3] = r.a.w; v[4] = r.b.x; v[5] = r.b.y; v[6] = r.b.z; v[7] = r.b.w;
+}
+__device__ __forceinline__ void unpack_raw8(const Raw8<__nv_bfloat16>& r, float (&v)[8]) { unpack_bf16x8(r.v, v); }
+
 // Up to eight consecutive elements with scalar loads; entries at or past `count` read as 0.
 template <typename T>
 __device__ __forceinline__ void load8_guarded(const T* p, int count, float (&v)[8])

@@ -109,8 +109,24 @@ project_stream_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
 #pragma unroll
             for (int e = 0; e < 8; ++e) { accR[e] = 0.0f; accG[e] = 0.0f; }
             if (count > 0) {
-#pragma unroll 4
-                for (int ii = warp; ii < rows_here; ii += 8) {
+                int ii = warp;
+                if (vec_ok) {
+                    // eight rows per pass: all eight 16-byte loads are issued before the first use
+                    for (; ii + 56 < rows_here; ii += 64) {
+                        Raw8<T> raw[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) raw[u] = load_raw8_stream(G + (int64_t)(i0 + ii + 8 * u) * cols + j0);
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            float g[8];
+                            unpack_raw8(raw[u], g);
+                            const float p = Ps[ii + 8 * u];
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) { accR[e] = fmaf(p, g[e], accR[e]); accG[e] = fmaf(g[e], g[e], accG[e]); }
+                        }
+                    }
+                }
+                for (; ii < rows_here; ii += 8) {
                     float g[8];
                     const T* src = G + (int64_t)(i0 + ii) * cols + j0;
                     if (vec_ok) load8_aligned(src, g); else load8_guarded(src, count, g);
@@ -508,7 +524,7 @@ void launch_project_stream(int dtype, const MatDesc* d_descs, const int* d_prefi
                            const StepParams& sp, int sm_count, cudaStream_t stream)
 {
     if (total_tiles <= 0) return;
-    const int grid = grid_for(total_tiles, 4, sm_count);
+    const int grid = grid_for(total_tiles, 6, sm_count);
     if (dtype == 0)
         project_stream_kernel<float><<<grid, STREAM_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, total_tiles, sp);
     else
