@@ -176,3 +176,22 @@ class ModelOracle:
 
     def step(self, Ws, Gs, lr: float, wd: float):
         return [mo.step(W, G, lr, wd) for mo, W, G in zip(self.mats, Ws, Gs)]
+
+
+def adamw_step(p, g, m, v, t, lr, beta1=0.9, beta2=0.999, eps=1e-8, wd=0.0, dtype=DT_F32, bias_correction=True):
+    """One AdamW step (Eq. 1 with decoupled weight decay) on flat arrays; m, v (float64) are updated.
+
+    Returns (p_new as float32 holding values of the stored dtype, update before the final rounding)."""
+    p = np.ascontiguousarray(p, dtype=np.float32).reshape(-1)
+    g = np.ascontiguousarray(g, dtype=np.float32).reshape(-1)
+    assert m.dtype == np.float64 and v.dtype == np.float64 and m.size == p.size and v.size == p.size
+    out = np.empty_like(p)
+    dp = np.empty(p.size, dtype=np.float64)
+    rc = lib().oracle_adamw_step(_ptr(p, ctypes.c_float), _ptr(g, ctypes.c_float), ctypes.c_int64(p.size),
+                                 ctypes.c_int32(dtype), ctypes.c_int32(int(bias_correction)), ctypes.c_double(lr),
+                                 ctypes.c_double(beta1), ctypes.c_double(beta2), ctypes.c_double(eps),
+                                 ctypes.c_double(wd), ctypes.c_int64(t), _ptr(m, ctypes.c_double),
+                                 _ptr(v, ctypes.c_double), _ptr(out, ctypes.c_float), _ptr(dp, ctypes.c_double))
+    if rc != 0:
+        raise ValueError(f"oracle adamw step failed with code {rc}")
+    return out, dp

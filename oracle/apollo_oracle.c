@@ -291,3 +291,34 @@ int oracle_apollo_step(const oracle_config* cfg, uint64_t seed, uint32_t matrix_
     free(P);
     return rc;
 }
+
+/*
+ * AdamW for the parameters APOLLO does not project (embeddings, norms, output head): the
+ * paper applies its method to 2-D weight matrices and leaves the rest to the base optimizer
+ * (Eq. 1 with decoupled weight decay; bias-corrected moments as in Loshchilov & Hutter's
+ * AdamW, which is what `bias_correction = 1` selects; 0 gives Eq. 1 exactly as printed).
+ *   m <- b1 m + (1-b1) g;  v <- b2 v + (1-b2) g^2;
+ *   p <- p - lr ( (m / c1) / (sqrt(v / c2) + eps) + wd p ),  c_i = 1 - b_i^(t+1) or 1.
+ * p, g: float arrays holding values of the stored dtype; m, v: double state.
+ */
+int oracle_adamw_step(const float* p, const float* g, int64_t numel, int32_t dtype, int32_t bias_correction,
+                      double lr, double beta1, double beta2, double eps, double wd, int64_t t,
+                      double* m, double* v, float* p_out, double* dp)
+{
+    if (!p || !g || !m || !v || !p_out || numel < 0) return ORACLE_ERR_ARG;
+    double c1 = 1.0, c2 = 1.0;
+    if (bias_correction) {
+        c1 = 1.0 - pow(beta1, (double)(t + 1));
+        c2 = 1.0 - pow(beta2, (double)(t + 1));
+    }
+    for (int64_t i = 0; i < numel; ++i) {
+        const double gi = (double)g[i], pi = (double)p[i];
+        m[i] = beta1 * m[i] + (1.0 - beta1) * gi;
+        v[i] = beta2 * v[i] + (1.0 - beta2) * gi * gi;
+        const double delta = -lr * ((m[i] / c1) / (sqrt(v[i] / c2) + eps) + wd * pi);
+        if (dp) dp[i] = delta;
+        const double pn = pi + delta;
+        p_out[i] = (float)(dtype == 1 ? oracle_round_bf16(pn) : pn);
+    }
+    return ORACLE_OK;
+}
