@@ -260,6 +260,27 @@ def run_ours(args, wl, rank, world, local_rank):
     if not args.no_e2e:
         line["e2e"] = {"value": whole_job_value(wl.params, world, e2e_ms), "unit": "params/s",
                        "h2d_bytes_per_step": g_bytes, "d2h_bytes_per_step": n * 16, "ms_per_step": e2e_ms}
+    if args.adamw:
+        # the non-projected parameters of the same model (embedding and head 32000 x hidden, norms):
+        # 22 bytes per bf16 parameter (read g, p, m, v; write p, m, v)
+        hidden = wl.shapes[0][0]
+        sizes = [32000 * hidden, 32000 * hidden] + [hidden] * 65
+        Pn = [torch.zeros(k, dtype=torch.bfloat16, device=dev) for k in sizes]
+        Gn = [torch.full((k,), 1e-3, dtype=torch.bfloat16, device=dev) for k in sizes]
+        Mn = [torch.zeros(k, dtype=torch.float32, device=dev) for k in sizes]
+        Vn = [torch.zeros(k, dtype=torch.float32, device=dev) for k in sizes]
+        for t in range(3):
+            B.adamw_step(Pn, Gn, Mn, Vn, t, 1e-3, wd=0.01)
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record(stream)
+        for t in range(10):
+            B.adamw_step(Pn, Gn, Mn, Vn, 3 + t, 1e-3, wd=0.01)
+        a1.record(stream)
+        torch.cuda.synchronize()
+        ms = a0.elapsed_time(a1) / 10
+        nbytes = 22 * sum(sizes)
+        line["adamw"] = {"params": sum(sizes), "ms_per_step": ms, "achieved": nbytes / (ms * 1e-3) / 1e9,
+                         "unit": "GB/s", "frac": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "bytes_per_param": 22}
     if world == 1 and not args.no_cpu:
         base = cpu_baseline(wl)
         line["cpu_baseline"] = {k: base[k] for k in ("value", "unit", "cores", "kind", "sample")}
@@ -276,6 +297,7 @@ def main():
     ap.add_argument("--workload", default="llama7b")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="keep only the first LAYERS layers (profiling aid)")
+    ap.add_argument("--adamw", action="store_true", help="also time the fused AdamW of the non-projected parameters")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

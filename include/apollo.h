@@ -170,6 +170,23 @@ APOLLO_API int apollo_set_timing(apollo_ctx* ctx, int32_t on);
 APOLLO_API int apollo_get_timing(apollo_ctx* ctx, int32_t steps_back, float* h_ms);
 
 /*
+ * AdamW for the parameters the method does not project (embeddings, norms, output head;
+ * the paper states APOLLO for 2-D weight matrices and keeps the base optimizer elsewhere).
+ * Eq. 1 with decoupled weight decay:  m <- b1 m + (1-b1) g,  v <- b2 v + (1-b2) g^2,
+ *   p <- p - lr ((m / c1) / (sqrt(v / c2) + eps) + wd p),  c_i = 1 - b_i^(t+1) with
+ * bias_correction = 1 (the usual AdamW), c_i = 1 with 0 (Eq. 1 as printed).
+ * d_P, d_G, d_M, d_V: HOST arrays of n_tensors DEVICE pointers (16-byte aligned); P and G
+ * have `dtype` (APOLLO_DT_*), M and V are fp32 of the same length, owned and zero-initialised
+ * by the caller; numel: HOST.  t = steps already taken.  d_dP: optional HOST array of DEVICE
+ * fp32 buffers that receive the update before it is added and rounded (entries or the array
+ * may be NULL).  Stateless, needs no workspace, asynchronous on `cuda_stream`.
+ */
+APOLLO_API int apollo_adamw_step(void* const* d_P, const void* const* d_G, float* const* d_M, float* const* d_V,
+                                 const int64_t* numel, int32_t n_tensors, int32_t dtype, float lr, float beta1,
+                                 float beta2, float eps, float wd, int64_t t, int32_t bias_correction,
+                                 float* const* d_dP, void* cuda_stream);
+
+/*
  * A rank-1 step for one matrix that allocates nothing and needs no workspace.  (The
  * paper has no counterpart to this entry point; it computes exactly what apollo_step
  * computes for a one-matrix list with rank 1.)

@@ -28,7 +28,7 @@ EXPORTS = [
     "apollo_workspace_bytes", "apollo_create", "apollo_step", "apollo_destroy", "apollo_step_count",
     "apollo_get_scales", "apollo_get_limiter", "apollo_get_state", "apollo_set_delta_out", "apollo_status",
     "apollo_philox_draws", "apollo_projection", "apollo_get_path", "apollo_last_launches", "apollo_strerror",
-    "apollo_set_timing", "apollo_get_timing", "apollo_mini_step_static", "apollo_cuda_error_string",
+    "apollo_set_timing", "apollo_get_timing", "apollo_mini_step_static", "apollo_cuda_error_string", "apollo_adamw_step",
 ]
 
 
@@ -87,6 +87,9 @@ def load():
                                             ctypes.POINTER(Config), u32, ctypes.c_int64, f32, f32, vp]
     lib.apollo_strerror.argtypes = [ctypes.c_int]
     lib.apollo_strerror.restype = ctypes.c_char_p
+    lib.apollo_adamw_step.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp),
+                                      ctypes.POINTER(ctypes.c_int64), i32, i32, f32, f32, f32, f32, f32,
+                                      ctypes.c_int64, i32, ctypes.POINTER(vp), vp]
     lib.apollo_cuda_error_string.argtypes = []
     lib.apollo_cuda_error_string.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -166,6 +169,23 @@ def mini_step_static(W, G, M, V, prev_norm, cfg: Config, matrix: int, t: int, lr
     _check(load().apollo_mini_step_static(W.data_ptr(), G.data_ptr(), rows, cols, M.data_ptr(), V.data_ptr(),
                                           prev_norm.data_ptr(), ctypes.byref(cfg), matrix, t, lr, wd,
                                           _stream_ptr(stream)), "apollo_mini_step_static")
+
+
+def adamw_step(params, grads, ms, vs, t, lr, beta1=0.9, beta2=0.999, eps=1e-8, wd=0.0, bias_correction=True,
+               deltas=None, stream=None):
+    """apollo_adamw_step over lists of CUDA tensors (params/grads of one dtype; ms/vs fp32, same numel)."""
+    n = len(params)
+    dtype = DT_BF16 if params[0].dtype == torch.bfloat16 else DT_F32
+
+    def arr(ts):
+        a = (ctypes.c_void_p * n)()
+        for i, x in enumerate(ts):
+            a[i] = None if x is None else x.data_ptr()
+        return a
+    numel = (ctypes.c_int64 * n)(*[p.numel() for p in params])
+    _check(load().apollo_adamw_step(arr(params), arr(grads), arr(ms), arr(vs), numel, n, dtype, lr, beta1, beta2, eps,
+                                    wd, t, int(bool(bias_correction)), arr(deltas) if deltas is not None else None,
+                                    _stream_ptr(stream)), "apollo_adamw_step")
 
 
 class Apollo:

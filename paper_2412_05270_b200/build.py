@@ -8,7 +8,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libapollo.so"
-SOURCES = ["apollo_api.cu", "kernels_basic.cu", "kernels_tensor.cu", "apollo_static.cu"]
+SOURCES = ["apollo_api.cu", "kernels_basic.cu", "kernels_tensor.cu", "apollo_static.cu", "kernels_adamw.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden",
