@@ -159,6 +159,22 @@ APOLLO_API int apollo_projection(uint64_t seed, uint32_t matrix, uint32_t epoch,
 APOLLO_API int apollo_get_path(const apollo_ctx* ctx, int32_t matrix, int32_t* out);
 
 /*
+ * Checkpoint and resume.  The optimizer state of Algorithm 1 is, per matrix, the moments M^R
+ * and V^R, the limiter's previous norm, the seed and the step counter t (the paper's table of
+ * state sizes: "2nr + 2"); P is not part of it because it is regenerated from (seed, matrix
+ * index, floor(t / T)).  apollo_state_bytes gives the size of the flat DEVICE buffer:
+ * per matrix in list order M (r x n floats), V (r x n floats), one float (previous norm).
+ * apollo_state_export copies the state out (after at least one step or an import);
+ * apollo_state_import copies it in and sets the step counter; the context must have been
+ * created with the same shapes and configuration (the seed and t are the caller's to keep:
+ * read t with apollo_step_count).  Both are asynchronous on `cuda_stream`.  A resumed run
+ * continues bit for bit like the uninterrupted one.
+ */
+APOLLO_API int apollo_state_bytes(const apollo_ctx* ctx, size_t* out_bytes);
+APOLLO_API int apollo_state_export(apollo_ctx* ctx, void* d_out, void* cuda_stream);
+APOLLO_API int apollo_state_import(apollo_ctx* ctx, const void* d_in, int64_t step_count, void* cuda_stream);
+
+/*
  * Per-phase device timing.  apollo_set_timing(ctx, 1) makes every later apollo_step record
  * CUDA events on its stream around the three phases (projection, finalize, update); the
  * last APOLLO_TIMING_SLOTS steps are kept.  apollo_get_timing waits for the chosen step

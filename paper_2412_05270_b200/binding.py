@@ -29,6 +29,7 @@ EXPORTS = [
     "apollo_get_scales", "apollo_get_limiter", "apollo_get_state", "apollo_set_delta_out", "apollo_status",
     "apollo_philox_draws", "apollo_projection", "apollo_get_path", "apollo_last_launches", "apollo_strerror",
     "apollo_set_timing", "apollo_get_timing", "apollo_mini_step_static", "apollo_cuda_error_string", "apollo_adamw_step",
+    "apollo_state_bytes", "apollo_state_export", "apollo_state_import",
 ]
 
 
@@ -90,6 +91,9 @@ def load():
     lib.apollo_adamw_step.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp),
                                       ctypes.POINTER(ctypes.c_int64), i32, i32, f32, f32, f32, f32, f32,
                                       ctypes.c_int64, i32, ctypes.POINTER(vp), vp]
+    lib.apollo_state_bytes.argtypes = [vp, ctypes.POINTER(ctypes.c_size_t)]
+    lib.apollo_state_export.argtypes = [vp, vp, vp]
+    lib.apollo_state_import.argtypes = [vp, vp, ctypes.c_int64, vp]
     lib.apollo_cuda_error_string.argtypes = []
     lib.apollo_cuda_error_string.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -283,6 +287,21 @@ class Apollo:
         out = ctypes.c_int64(0)
         _check(self.lib.apollo_step_count(self.ctx, ctypes.byref(out)), "apollo_step_count")
         return out.value
+
+    def state_export(self, stream=None) -> torch.Tensor:
+        """The optimizer state (moments and limiter norms) as one flat uint8 CUDA tensor."""
+        n = ctypes.c_size_t(0)
+        _check(self.lib.apollo_state_bytes(self.ctx, ctypes.byref(n)), "apollo_state_bytes")
+        out = torch.empty(n.value, dtype=torch.uint8, device=self.device)
+        _check(self.lib.apollo_state_export(self.ctx, out.data_ptr(), _stream_ptr(stream)), "apollo_state_export")
+        return out
+
+    def state_import(self, flat: torch.Tensor, step_count: int, stream=None):
+        n = ctypes.c_size_t(0)
+        _check(self.lib.apollo_state_bytes(self.ctx, ctypes.byref(n)), "apollo_state_bytes")
+        assert flat.is_cuda and flat.dtype == torch.uint8 and flat.numel() == n.value and flat.is_contiguous()
+        _check(self.lib.apollo_state_import(self.ctx, flat.data_ptr(), step_count, _stream_ptr(stream)),
+               "apollo_state_import")
 
     def set_timing(self, on: bool):
         _check(self.lib.apollo_set_timing(self.ctx, int(on)), "apollo_set_timing")

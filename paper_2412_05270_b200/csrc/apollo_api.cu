@@ -187,6 +187,7 @@ struct apollo_ctx {
     std::vector<float*> delta;
     bool delta_on;
     bool first;
+    bool imported;   // the moments came from apollo_state_import: the first step must not zero them
     bool descs_dirty;
     int64_t t;
     int device;
@@ -289,6 +290,7 @@ int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_ma
     ctx->delta.assign(n_matrices, nullptr);
     ctx->delta_on = false;
     ctx->first = true;
+    ctx->imported = false;
     ctx->descs_dirty = true;
     ctx->t = 0;
     ctx->last_launches = 0;
@@ -346,7 +348,8 @@ int apollo_step(apollo_ctx* ctx, void* const* d_W, const void* const* d_G, float
 
     if (ctx->first) {
         if (cudaMemsetAsync(ctx->ws + plan.off_status, 0, ALIGN, stream) != cudaSuccess) return APOLLO_ERR_CUDA;
-        if (cudaMemsetAsync(ctx->ws + plan.zero_begin, 0, plan.zero_end - plan.zero_begin, stream) != cudaSuccess)
+        if (!ctx->imported &&
+            cudaMemsetAsync(ctx->ws + plan.zero_begin, 0, plan.zero_end - plan.zero_begin, stream) != cudaSuccess)
             return APOLLO_ERR_CUDA;
         for (int t = 0; t < 4; ++t)
             if (cudaMemcpyAsync(ctx->d_prefix[t], ctx->h_prefix[t].data(), sizeof(int) * (ctx->n_mat + 1),
@@ -468,6 +471,56 @@ int apollo_status(apollo_ctx* ctx, void* cuda_stream)
         cudaMemset(ctx->d_status, 0, sizeof(word));
         return APOLLO_ERR_TIMEOUT;
     }
+    return APOLLO_OK;
+}
+
+// Checkpoint layout: for each matrix in list order M (r x n floats), V (r x n floats), then one
+// float: the limiter's previous norm.
+int apollo_state_bytes(const apollo_ctx* ctx, size_t* out_bytes)
+{
+    if (!ctx || !out_bytes) return APOLLO_ERR_INVALID_ARG;
+    size_t total = 0;
+    for (int i = 0; i < ctx->n_mat; ++i)
+        total += sizeof(float) * (2 * (size_t)ctx->cfg.rank * (size_t)ctx->h_descs[i].n + 1);
+    *out_bytes = total;
+    return APOLLO_OK;
+}
+
+static int state_copy(apollo_ctx* ctx, char* d_flat, bool to_flat, cudaStream_t stream)
+{
+    if (((uintptr_t)d_flat % 4) != 0) return APOLLO_ERR_ALIGN;
+    size_t at = 0;
+    for (int i = 0; i < ctx->n_mat; ++i) {
+        const MatDesc& d = ctx->h_descs[i];
+        const size_t bytes = sizeof(float) * (size_t)ctx->cfg.rank * (size_t)d.n;
+        void* parts[3] = { d.M, d.V, d.prev };
+        const size_t sizes[3] = { bytes, bytes, sizeof(float) };
+        for (int k = 0; k < 3; ++k) {
+            const cudaError_t e = to_flat
+                ? cudaMemcpyAsync(d_flat + at, parts[k], sizes[k], cudaMemcpyDeviceToDevice, stream)
+                : cudaMemcpyAsync(parts[k], d_flat + at, sizes[k], cudaMemcpyDeviceToDevice, stream);
+            if (!cuda_ok(e)) return APOLLO_ERR_CUDA;
+            at += sizes[k];
+        }
+    }
+    return APOLLO_OK;
+}
+
+int apollo_state_export(apollo_ctx* ctx, void* d_out, void* cuda_stream)
+{
+    if (!ctx || !d_out) return APOLLO_ERR_INVALID_ARG;
+    if (ctx->first && !ctx->imported) return APOLLO_ERR_INVALID_ARG;   // no step has run: nothing to export yet
+    return state_copy(ctx, static_cast<char*>(d_out), true, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int apollo_state_import(apollo_ctx* ctx, const void* d_in, int64_t step_count, void* cuda_stream)
+{
+    if (!ctx || !d_in || step_count < 0) return APOLLO_ERR_INVALID_ARG;
+    const int rc = state_copy(ctx, const_cast<char*>(static_cast<const char*>(d_in)), false,
+                              static_cast<cudaStream_t>(cuda_stream));
+    if (rc != APOLLO_OK) return rc;
+    ctx->t = step_count;
+    ctx->imported = true;
     return APOLLO_OK;
 }
 

@@ -141,3 +141,38 @@ def test_misaligned_and_null_pointers_are_rejected_before_any_launch():
     assert e.value.code == B.ERR_ALIGN
     assert opt.step_count() == 0
     opt.close()
+
+
+@pytest.mark.parametrize("rank,mode,flags", [(32, "channel", 0), (1, "tensor", 0), (5, "channel", B.FLAG_NO_TENSOR_CORES)])
+def test_checkpoint_and_resume_continue_bit_for_bit(rank, mode, flags):
+    wl = _wl([(200, 336), (336, 200), (64, 64)], rank, mode=mode, dtype="bf16", T=2, steps=6, wd=0.01)
+    dev = torch.device("cuda")
+    cfg = B.config_for(wl, flags)
+
+    def run(opt, Ws, t0, t1):
+        for t in range(t0, t1):
+            opt.step(Ws, [WL.make_grad(wl, i, t).to(dev) for i in range(3)], wl.lr, wl.wd)
+        torch.cuda.synchronize()
+
+    whole = B.Apollo(wl.shapes, cfg)
+    W_whole = [WL.make_weight(wl, i).to(dev) for i in range(3)]
+    run(whole, W_whole, 0, 6)
+
+    first = B.Apollo(wl.shapes, cfg)
+    W_part = [WL.make_weight(wl, i).to(dev) for i in range(3)]
+    run(first, W_part, 0, 3)                       # stops right after a refresh step (T = 2)
+    blob, t = first.state_export(), first.step_count()
+    assert t == 3
+    first.close()
+    second = B.Apollo(wl.shapes, cfg)
+    second.state_import(blob.clone(), t)
+    run(second, W_part, 3, 6)
+    assert second.step_count() == 6
+    for a, b in zip(W_whole, W_part):
+        assert torch.equal(a, b)
+    for i in range(3):
+        assert torch.equal(whole.scales(i), second.scales(i))
+        assert torch.equal(whole.limiter(i), second.limiter(i))
+    fresh = B.Apollo(wl.shapes, cfg)
+    with pytest.raises(B.ApolloError):
+        fresh.state_export()                       # nothing has run yet
