@@ -113,6 +113,18 @@ APOLLO_API int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, i
 APOLLO_API int apollo_step(apollo_ctx* ctx, void* const* d_W, const void* const* d_G, float lr, float wd,
                 void* cuda_stream);
 
+/*
+ * The same step for matrices [first, first + count) only, at the current step counter
+ * (d_W, d_G: HOST arrays of `count` DEVICE pointers).  This is what a layer-wise update
+ * strategy needs (the paper's Figure 1 caption and its paragraph on training under 12 GB:
+ * run the optimizer for a layer as soon as its gradient exists and free the gradient): call it once per layer during the backward
+ * pass, in any order, each matrix exactly once per step, and pass close_step != 0 on the
+ * last call of the step so that t advances.  apollo_step is apollo_step_range over the
+ * whole list with close_step = 1.
+ */
+APOLLO_API int apollo_step_range(apollo_ctx* ctx, int32_t first, int32_t count, void* const* d_W,
+                                 const void* const* d_G, float lr, float wd, int32_t close_step, void* cuda_stream);
+
 APOLLO_API int apollo_destroy(apollo_ctx* ctx);
 
 /* Number of steps taken so far (t of Algorithm 1).  out: HOST. */

@@ -29,7 +29,7 @@ EXPORTS = [
     "apollo_get_scales", "apollo_get_limiter", "apollo_get_state", "apollo_set_delta_out", "apollo_status",
     "apollo_philox_draws", "apollo_projection", "apollo_get_path", "apollo_last_launches", "apollo_strerror",
     "apollo_set_timing", "apollo_get_timing", "apollo_mini_step_static", "apollo_cuda_error_string", "apollo_adamw_step",
-    "apollo_state_bytes", "apollo_state_export", "apollo_state_import",
+    "apollo_state_bytes", "apollo_state_export", "apollo_state_import", "apollo_step_range",
 ]
 
 
@@ -71,6 +71,7 @@ def load():
     lib.apollo_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(Shape), i32, ctypes.POINTER(Config), vp,
                                   ctypes.c_size_t]
     lib.apollo_step.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), f32, f32, vp]
+    lib.apollo_step_range.argtypes = [vp, i32, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), f32, f32, i32, vp]
     lib.apollo_destroy.argtypes = [vp]
     lib.apollo_step_count.argtypes = [vp, ctypes.POINTER(ctypes.c_int64)]
     lib.apollo_get_scales.argtypes = [vp, i32, vp, vp]
@@ -240,6 +241,14 @@ class Apollo:
             self._w_arr[i] = w.data_ptr()
             self._g_arr[i] = g.data_ptr()
         _check(self.lib.apollo_step(self.ctx, self._w_arr, self._g_arr, lr, wd, _stream_ptr(stream)), "apollo_step")
+
+    def step_range(self, first: int, Ws, Gs, lr: float, wd: float = 0.0, close_step: bool = False, stream=None):
+        """apollo_step_range: the step of matrices first .. first + len(Ws) - 1 (layer-wise updates)."""
+        n = len(Ws)
+        w = (ctypes.c_void_p * n)(*[x.data_ptr() for x in Ws])
+        g = (ctypes.c_void_p * n)(*[x.data_ptr() for x in Gs])
+        _check(self.lib.apollo_step_range(self.ctx, first, n, w, g, lr, wd, int(close_step), _stream_ptr(stream)),
+               "apollo_step_range")
 
     def set_delta_out(self, deltas):
         """deltas: list of float32 CUDA tensors shaped like the weights (None entries skip a matrix), or None."""

@@ -333,15 +333,20 @@ int apollo_set_delta_out(apollo_ctx* ctx, float* const* d_dW)
     return APOLLO_OK;
 }
 
-int apollo_step(apollo_ctx* ctx, void* const* d_W, const void* const* d_G, float lr, float wd,
-                void* cuda_stream)
+// One step of matrices [first, first + count) at the current step counter; d_W and d_G hold
+// `count` pointers.  `advance` closes the step (t <- t + 1).
+static int step_range(apollo_ctx* ctx, int first, int count, void* const* d_W, const void* const* d_G, float lr,
+                      float wd, bool advance, void* cuda_stream)
 {
     if (!ctx || !d_W || !d_G) return APOLLO_ERR_INVALID_ARG;
+    if (first < 0 || count < 1 || first + count > ctx->n_mat) return APOLLO_ERR_INVALID_ARG;
     if (!std::isfinite(lr) || !std::isfinite(wd)) return APOLLO_ERR_INVALID_ARG;
-    for (int i = 0; i < ctx->n_mat; ++i) {
+    for (int i = 0; i < count; ++i) {
         if (!d_W[i] || !d_G[i]) return APOLLO_ERR_INVALID_ARG;
         if (((uintptr_t)d_W[i] % 16) || ((uintptr_t)d_G[i] % 16)) return APOLLO_ERR_ALIGN;
     }
+    const int last = first + count;
+    const bool whole = count == ctx->n_mat;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const apollo_config& cfg = ctx->cfg;
     const Plan& plan = ctx->plan;
@@ -357,10 +362,10 @@ int apollo_step(apollo_ctx* ctx, void* const* d_W, const void* const* d_G, float
                 return APOLLO_ERR_CUDA;
     }
     bool changed = ctx->descs_dirty;
-    for (int i = 0; i < ctx->n_mat; ++i) {
+    for (int i = first; i < last; ++i) {
         MatDesc& d = ctx->h_descs[i];
-        if (d.W != d_W[i] || d.G != d_G[i] || d.dW != ctx->delta[i]) {
-            d.W = d_W[i]; d.G = d_G[i]; d.dW = ctx->delta[i];
+        if (d.W != d_W[i - first] || d.G != d_G[i - first] || d.dW != ctx->delta[i]) {
+            d.W = d_W[i - first]; d.G = d_G[i - first]; d.dW = ctx->delta[i];
             changed = true;
         }
     }
@@ -390,46 +395,68 @@ int apollo_step(apollo_ctx* ctx, void* const* d_W, const void* const* d_G, float
     }
 
     int launches = 0;
-    cudaEvent_t* ev = ctx->timing_on ? ctx->ev[ctx->t % APOLLO_TIMING_SLOTS] : nullptr;
+    cudaEvent_t* ev = (ctx->timing_on && whole) ? ctx->ev[ctx->t % APOLLO_TIMING_SLOTS] : nullptr;
     if (ev) cudaEventRecord(ev[0], stream);
-    if (plan.tiles[PATH_STREAM] > 0) {
-        launch_project_stream(cfg.dtype, ctx->d_descs, ctx->d_prefix[PATH_STREAM], ctx->n_mat,
-                              (int)plan.tiles[PATH_STREAM], sp, ctx->sm_count, stream);
+    auto tiles_of = [&](int path, int a, int b, int& tb, int& te) {
+        tb = ctx->h_prefix[path][a]; te = ctx->h_prefix[path][b];
+        return te > tb;
+    };
+    int tb = 0, te = 0;
+    if (tiles_of(PATH_STREAM, first, last, tb, te)) {
+        launch_project_stream(cfg.dtype, ctx->d_descs, ctx->d_prefix[PATH_STREAM], ctx->n_mat, tb, te, sp,
+                              ctx->sm_count, stream);
         ++launches;
     }
-    if (plan.tiles[PATH_SIMT] > 0) {
-        launch_project_simt(cfg.dtype, ctx->d_descs, ctx->d_prefix[PATH_SIMT], ctx->n_mat,
-                            (int)plan.tiles[PATH_SIMT], sp, ctx->sm_count, stream);
+    if (tiles_of(PATH_SIMT, first, last, tb, te)) {
+        launch_project_simt(cfg.dtype, ctx->d_descs, ctx->d_prefix[PATH_SIMT], ctx->n_mat, tb, te, sp, ctx->sm_count,
+                            stream);
         ++launches;
     }
-    if (plan.tiles[PATH_TENSOR] > 0) {
+    if (tiles_of(PATH_TENSOR, first, last, tb, te)) {
         if (plan.any_repitch) {
-            launch_repitch(ctx->d_descs, ctx->n_mat, stream);
+            launch_repitch(ctx->d_descs, first, count, stream);
             ++launches;
         }
         for (const StageGroup& g : plan.groups) {
-            if (g.tile_end <= g.tile_begin) continue;
+            // the part of this staging group inside the range
+            const int mb = g.mat_begin > first ? g.mat_begin : first;
+            const int me = g.mat_end < last ? g.mat_end : last;
+            if (me <= mb || !tiles_of(PATH_TENSOR, mb, me, tb, te)) continue;
             if (tensor_path_staged()) {
-                launch_generate_p(ctx->d_descs, g.mat_begin, g.mat_end, sp, stream);
+                launch_generate_p(ctx->d_descs, mb, me, sp, stream);
                 ++launches;
             }
-            launch_project_tensor(ctx->d_descs, ctx->d_prefix[PATH_TENSOR], ctx->n_mat, g.tile_begin, g.tile_end, sp,
-                                  ctx->sm_count, ctx->d_status, stream);
+            launch_project_tensor(ctx->d_descs, ctx->d_prefix[PATH_TENSOR], ctx->n_mat, tb, te, sp, ctx->sm_count,
+                                  ctx->d_status, stream);
             ++launches;
         }
     }
     if (ev) cudaEventRecord(ev[1], stream);
-    launch_finalize(ctx->d_descs, ctx->n_mat, sp, stream);
+    launch_finalize(ctx->d_descs, first, count, sp, stream);
     ++launches;
     if (ev) cudaEventRecord(ev[2], stream);
-    launch_update(cfg.dtype, ctx->d_descs, ctx->d_prefix[3], ctx->n_mat, (int)plan.tiles[3], sp, ctx->sm_count, stream);
+    tiles_of(3, first, last, tb, te);
+    launch_update(cfg.dtype, ctx->d_descs, ctx->d_prefix[3], ctx->n_mat, tb, te, sp, ctx->sm_count, stream);
     ++launches;
     if (ev) cudaEventRecord(ev[3], stream);
     if (!cuda_ok(cudaGetLastError())) return APOLLO_ERR_CUDA;
     ctx->first = false;
-    ctx->t += 1;
+    if (advance) ctx->t += 1;
     ctx->last_launches = launches;
     return APOLLO_OK;
+}
+
+int apollo_step(apollo_ctx* ctx, void* const* d_W, const void* const* d_G, float lr, float wd,
+                void* cuda_stream)
+{
+    if (!ctx) return APOLLO_ERR_INVALID_ARG;
+    return step_range(ctx, 0, ctx->n_mat, d_W, d_G, lr, wd, true, cuda_stream);
+}
+
+int apollo_step_range(apollo_ctx* ctx, int32_t first, int32_t count, void* const* d_W, const void* const* d_G,
+                      float lr, float wd, int32_t close_step, void* cuda_stream)
+{
+    return step_range(ctx, first, count, d_W, d_G, lr, wd, close_step != 0, cuda_stream);
 }
 
 int apollo_get_scales(apollo_ctx* ctx, int32_t matrix, float* d_out, void* cuda_stream)

@@ -150,9 +150,9 @@ extern "C" int apollo_mini_step_static(void* d_W, const void* d_G, int64_t rows,
     const MatDesc* d_desc = reinterpret_cast<const MatDesc*>(base + OFF_DESC);
     static_setup_kernel<<<1, 1, 0, stream>>>(d, (int)proj_tiles, (int)update_tiles);
     launch_project_stream(cfg->dtype, d_desc, reinterpret_cast<const int*>(base + OFF_PREFIX_P), 1,
-                          (int)proj_tiles, sp, sm_count, stream);
-    launch_finalize(d_desc, 1, sp, stream);
-    launch_update(cfg->dtype, d_desc, reinterpret_cast<const int*>(base + OFF_PREFIX_U), 1, (int)update_tiles,
+                          0, (int)proj_tiles, sp, sm_count, stream);
+    launch_finalize(d_desc, 0, 1, sp, stream);
+    launch_update(cfg->dtype, d_desc, reinterpret_cast<const int*>(base + OFF_PREFIX_U), 1, 0, (int)update_tiles,
                   sp, sm_count, stream);
     return cudaGetLastError() == cudaSuccess ? APOLLO_OK : APOLLO_ERR_CUDA;
 }

@@ -8,12 +8,12 @@ void launch_philox_draws(uint32_t key0, uint32_t key1, uint32_t matrix, uint32_t
                          uint32_t* d_out, cudaStream_t stream);
 void launch_projection(uint32_t key0, uint32_t key1, uint32_t matrix, uint32_t epoch, int r, int m,
                        float* d_out, cudaStream_t stream);
-void launch_project_stream(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int total_tiles,
+void launch_project_stream(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int tile_begin, int tile_end,
                            const StepParams& sp, int sm_count, cudaStream_t stream);
-void launch_project_simt(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int total_tiles,
+void launch_project_simt(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int tile_begin, int tile_end,
                          const StepParams& sp, int sm_count, cudaStream_t stream);
-void launch_finalize(const MatDesc* d_descs, int n_mat, const StepParams& sp, cudaStream_t stream);
-void launch_update(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int total_tiles,
+void launch_finalize(const MatDesc* d_descs, int first, int count, const StepParams& sp, cudaStream_t stream);
+void launch_update(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int tile_begin, int tile_end,
                    const StepParams& sp, int sm_count, cudaStream_t stream);
 
 
@@ -29,7 +29,7 @@ size_t tensor_path_stage_bytes(int rows, int cols, int rank);
 // each 256-byte slot) and queues their upload to `d_tmaps`.  Returns an APOLLO_* code.
 int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, void* d_tmaps, cudaStream_t stream);
 // Copies the gradients whose row pitch is not a multiple of 16 bytes into their padded buffers.
-void launch_repitch(const MatDesc* d_descs, int n_mat, cudaStream_t stream);
+void launch_repitch(const MatDesc* d_descs, int first, int count, cudaStream_t stream);
 // Fills the staging buffer with the standard normals of matrices [mat_begin, mat_end).
 void launch_generate_p(const MatDesc* d_descs, int mat_begin, int mat_end, const StepParams& sp, cudaStream_t stream);
 // Projection over tiles [tile_begin, tile_end) of the tensor-path prefix table.

@@ -77,13 +77,13 @@ constexpr int STREAM_TALL_CHUNK = 2048;   // entries of P staged per pass over a
 template <typename T>
 __global__ void __launch_bounds__(STREAM_THREADS)
 project_stream_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix, int n_mat,
-                      int total_tiles, StepParams sp)
+                      int tile_begin, int tile_end, StepParams sp)
 {
     __shared__ float Ps[STREAM_TALL_CHUNK];
     __shared__ float red[2][8][STREAM_COLS];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+    for (int tile = tile_begin + blockIdx.x; tile < tile_end; tile += gridDim.x) {
         const int mat = find_matrix(prefix, n_mat, tile);
         const MatDesc& d = descs[mat];
         const int local = tile - __ldg(prefix + mat);
@@ -208,7 +208,7 @@ constexpr int SIMT_THREADS = 256;
 template <typename T>
 __global__ void __launch_bounds__(SIMT_THREADS)
 project_simt_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix, int n_mat,
-                    int total_tiles, StepParams sp)
+                    int tile_begin, int tile_end, StepParams sp)
 {
     __shared__ float Ps[SIMT_BK][SIMT_BR + 1];     // [kk][row of R]
     __shared__ float Gs[SIMT_BK][SIMT_BN + 1];     // [kk][channel]
@@ -216,7 +216,7 @@ project_simt_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
 
     const int tid = threadIdx.x;
     const int tx = tid & 15, ty = tid >> 4;       // tx: 4 channels each, ty: 4 rows of R each
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+    for (int tile = tile_begin + blockIdx.x; tile < tile_end; tile += gridDim.x) {
         const int mat = find_matrix(prefix, n_mat, tile);
         const MatDesc& d = descs[mat];
         const int local = tile - __ldg(prefix + mat);
@@ -320,10 +320,10 @@ project_simt_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
 constexpr int FINALIZE_THREADS = 1024;
 
 __global__ void __launch_bounds__(FINALIZE_THREADS)
-finalize_kernel(const MatDesc* __restrict__ descs, StepParams sp)
+finalize_kernel(const MatDesc* __restrict__ descs, int first, StepParams sp)
 {
     __shared__ double scratch[32];
-    const MatDesc& d = descs[blockIdx.x];
+    const MatDesc& d = descs[first + blockIdx.x];
     const int n = d.n;
     const bool tensor_mode = sp.mode == 1;
     double sum_num = 0.0, sum_den = 0.0, sum_g2 = 0.0, sum_sq = 0.0;
@@ -405,9 +405,9 @@ __device__ __forceinline__ void store1(__nv_bfloat16* p, float v) { *p = __float
 template <typename T>
 __global__ void __launch_bounds__(UPDATE_THREADS)
 update_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix, int n_mat,
-              int total_tiles, StepParams sp)
+              int tile_begin, int tile_end, StepParams sp)
 {
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+    for (int tile = tile_begin + blockIdx.x; tile < tile_end; tile += gridDim.x) {
         const int mat = find_matrix(prefix, n_mat, tile);
         const MatDesc& d = descs[mat];
         const int local = tile - __ldg(prefix + mat);
@@ -520,43 +520,46 @@ static int grid_for(int total_tiles, int per_sm, int sm_count)
     return total_tiles < cap ? total_tiles : cap;
 }
 
-void launch_project_stream(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int total_tiles,
+void launch_project_stream(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int tile_begin, int tile_end,
                            const StepParams& sp, int sm_count, cudaStream_t stream)
 {
+    const int total_tiles = tile_end - tile_begin;
     if (total_tiles <= 0) return;
     const int grid = grid_for(total_tiles, 6, sm_count);
     if (dtype == 0)
-        project_stream_kernel<float><<<grid, STREAM_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, total_tiles, sp);
+        project_stream_kernel<float><<<grid, STREAM_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end, sp);
     else
-        project_stream_kernel<__nv_bfloat16><<<grid, STREAM_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, total_tiles, sp);
+        project_stream_kernel<__nv_bfloat16><<<grid, STREAM_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end, sp);
 }
 
-void launch_project_simt(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int total_tiles,
+void launch_project_simt(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int tile_begin, int tile_end,
                          const StepParams& sp, int sm_count, cudaStream_t stream)
 {
+    const int total_tiles = tile_end - tile_begin;
     if (total_tiles <= 0) return;
     const int grid = grid_for(total_tiles, 4, sm_count);
     if (dtype == 0)
-        project_simt_kernel<float><<<grid, SIMT_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, total_tiles, sp);
+        project_simt_kernel<float><<<grid, SIMT_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end, sp);
     else
-        project_simt_kernel<__nv_bfloat16><<<grid, SIMT_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, total_tiles, sp);
+        project_simt_kernel<__nv_bfloat16><<<grid, SIMT_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end, sp);
 }
 
-void launch_finalize(const MatDesc* d_descs, int n_mat, const StepParams& sp, cudaStream_t stream)
+void launch_finalize(const MatDesc* d_descs, int first, int count, const StepParams& sp, cudaStream_t stream)
 {
-    if (n_mat <= 0) return;
-    finalize_kernel<<<n_mat, FINALIZE_THREADS, 0, stream>>>(d_descs, sp);
+    if (count <= 0) return;
+    finalize_kernel<<<count, FINALIZE_THREADS, 0, stream>>>(d_descs, first, sp);
 }
 
-void launch_update(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int total_tiles,
+void launch_update(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int tile_begin, int tile_end,
                    const StepParams& sp, int sm_count, cudaStream_t stream)
 {
+    const int total_tiles = tile_end - tile_begin;
     if (total_tiles <= 0) return;
     const int grid = grid_for(total_tiles, 8, sm_count);
     if (dtype == 0)
-        update_kernel<float><<<grid, UPDATE_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, total_tiles, sp);
+        update_kernel<float><<<grid, UPDATE_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end, sp);
     else
-        update_kernel<__nv_bfloat16><<<grid, UPDATE_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, total_tiles, sp);
+        update_kernel<__nv_bfloat16><<<grid, UPDATE_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end, sp);
 }
 
 }  // namespace apollo

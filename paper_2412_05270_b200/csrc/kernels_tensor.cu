@@ -1017,9 +1017,9 @@ __global__ void generate_p_kernel(const MatDesc* __restrict__ descs, int mat_beg
 }  // namespace
 
 // G with an odd row pitch -> copy with the pitch rounded up to 8 elements (TMA needs 16-byte rows).
-__global__ void repitch_kernel(const MatDesc* __restrict__ descs)
+__global__ void repitch_kernel(const MatDesc* __restrict__ descs, int first)
 {
-    const MatDesc* dp = descs + blockIdx.y;
+    const MatDesc* dp = descs + first + blockIdx.y;
     unsigned short* dst = static_cast<unsigned short*>(dp->gpad);
     if (!dst) return;
     const unsigned short* __restrict__ src = static_cast<const unsigned short*>(dp->G);
@@ -1031,11 +1031,11 @@ __global__ void repitch_kernel(const MatDesc* __restrict__ descs)
     }
 }
 
-void launch_repitch(const MatDesc* d_descs, int n_mat, cudaStream_t stream)
+void launch_repitch(const MatDesc* d_descs, int first, int count, cudaStream_t stream)
 {
-    if (n_mat <= 0) return;
-    const dim3 grid(128, (unsigned)n_mat);
-    repitch_kernel<<<grid, 256, 0, stream>>>(d_descs);
+    if (count <= 0) return;
+    const dim3 grid(128, (unsigned)count);
+    repitch_kernel<<<grid, 256, 0, stream>>>(d_descs, first);
 }
 
 void launch_generate_p(const MatDesc* d_descs, int mat_begin, int mat_end, const StepParams& sp, cudaStream_t stream)

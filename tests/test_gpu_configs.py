@@ -136,3 +136,61 @@ def test_llama7b_full_list_sampled_channels_and_limiter():
             np.testing.assert_allclose(V[:, idx].cpu().numpy(), orc[i].V, rtol=4e-3, atol=5e-3 * np.median(np.abs(orc[i].V)))
         del Gg
     opt.close()
+
+
+def test_matrix_with_more_than_2_31_elements_rank1():
+    """Flat indices above 2^31: 70000 x 32768 bf16 (2.29 G elements), Mini step checked with torch on the
+    GPU (the generator itself is pinned bit-exactly against the oracle elsewhere)."""
+    dev = torch.device("cuda")
+    rows, cols = 70000, 32768
+    assert rows * cols > 2 ** 31
+    g = torch.Generator(device=dev).manual_seed(11)
+    W = torch.empty(rows, cols, dtype=torch.bfloat16, device=dev).normal_(0, 0.02, generator=g)
+    G = torch.empty(rows, cols, dtype=torch.bfloat16, device=dev).normal_(0, 1e-3, generator=g)
+    W0_tail = W[-3:].float().clone()
+    W0_head = W[:2].float().clone()
+    alpha = math.sqrt(128.0)
+    cfg = B.make_config(rank=1, mode=B.SCALE_TENSOR, dtype=B.DT_BF16, T=5, seed=77, alpha=alpha, gamma=1.01)
+    opt = B.Apollo([(rows, cols)], cfg)
+    assert opt.path(0) == B.PATH_STREAM
+    opt.step([W], [G], 1e-2, 0.0)
+    torch.cuda.synchronize()
+    assert opt.status() == B.OK
+    # tall matrix: project along the 32768 columns, one channel per row
+    z = B.projection(77, 0, 0, 1, cols)[0].double()
+    R = torch.empty(rows, dtype=torch.float64, device=dev)
+    for a in range(0, rows, 10000):
+        R[a:a + 10000] = G[a:a + 10000].double() @ z
+    Rt = (0.1 * R) / (torch.sqrt(0.001 * R * R) + 1e-8)
+    s_want = (Rt.norm() / R.norm()).item()
+    s_gpu = opt.scales(0)
+    assert torch.all(s_gpu == s_gpu[0])
+    assert abs(s_gpu[0].item() - s_want) <= 1e-4 * s_want
+    lim = opt.limiter(0).cpu().numpy()
+    g_norm = math.sqrt(sum(float(G[a:a + 10000].float().square().sum()) for a in range(0, rows, 10000)))
+    assert abs(lim[2] - s_want * g_norm) <= 1e-3 * s_want * g_norm and lim[1] == 1.0
+    M, V = opt.state(0)
+    assert torch.allclose(M[0].double(), 0.1 * R, rtol=1e-3, atol=1e-3 * float(R.abs().median()) * 0.1)
+    # the update at the very end of the flat array (indices above 2^31) and at its start
+    step = 1e-2 * alpha * s_gpu[0].item()
+    for sl, before in ((slice(rows - 3, rows), W0_tail), (slice(0, 2), W0_head)):
+        want = (before - step * G[sl].float()).to(torch.bfloat16)
+        got = W[sl]
+        assert (want.float() - got.float()).abs().max().item() <= 2.0 ** -7 * before.abs().max().item()
+        assert (want == got).float().mean().item() > 0.99
+    opt.close()
+
+
+def test_one_by_one_matrix():
+    dev = torch.device("cuda")
+    opt = B.Apollo([(1, 1)], B.make_config(rank=1, mode=B.SCALE_CHANNEL, dtype=B.DT_F32, seed=3, gamma=0.0, eps=0.0))
+    W = torch.tensor([[0.5]], device=dev)
+    G = torch.tensor([[2.0]], device=dev)
+    opt.step([W], [G], 0.1, 0.0)
+    torch.cuda.synchronize()
+    # R = z g, M = 0.1 R, V = 0.001 R^2 -> |R~| / |R| = sqrt(10) / |z g|; update = lr s g
+    z = abs(B.projection(3, 0, 0, 1, 1).item())
+    s = math.sqrt(10.0) / (z * 2.0)
+    assert abs(opt.scales(0).item() - s) <= 1e-5 * s
+    assert abs(W.item() - (0.5 - 0.1 * s * 2.0)) <= 1e-5
+    opt.close()

@@ -176,3 +176,29 @@ def test_checkpoint_and_resume_continue_bit_for_bit(rank, mode, flags):
     fresh = B.Apollo(wl.shapes, cfg)
     with pytest.raises(B.ApolloError):
         fresh.state_export()                       # nothing has run yet
+
+
+@pytest.mark.parametrize("rank,mode,flags", [(32, "channel", 0), (1, "tensor", 0), (5, "channel", B.FLAG_NO_TENSOR_CORES)])
+def test_layer_wise_range_steps_equal_the_whole_list_step(rank, mode, flags):
+    shapes = [(200, 336), (336, 200), (64, 64), (128, 520), (96, 203), (72, 64), (64, 72)]
+    wl = _wl(shapes, rank, mode=mode, dtype="bf16", T=2, steps=4, wd=0.01)
+    dev = torch.device("cuda")
+    cfg = B.config_for(wl, flags)
+    n = len(shapes)
+    whole, ranged = B.Apollo(wl.shapes, cfg), B.Apollo(wl.shapes, cfg)
+    Wa = [WL.make_weight(wl, i).to(dev) for i in range(n)]
+    Wb = [w.clone() for w in Wa]
+    layers = [(4, 7), (2, 4), (0, 2)]          # visited in backward order
+    for t in range(4):
+        G = [WL.make_grad(wl, i, t).to(dev) for i in range(n)]
+        whole.step(Wa, G, wl.lr, wl.wd)
+        for k, (a, b) in enumerate(layers):
+            ranged.step_range(a, Wb[a:b], G[a:b], wl.lr, wl.wd, close_step=(k == len(layers) - 1))
+        torch.cuda.synchronize()
+        assert ranged.step_count() == t + 1
+        for i in range(n):
+            assert torch.equal(Wa[i], Wb[i]), (t, i)
+            assert torch.equal(whole.scales(i), ranged.scales(i))
+    assert whole.status() == B.OK and ranged.status() == B.OK
+    with pytest.raises(B.ApolloError):
+        ranged.step_range(5, Wb[5:8] + [Wb[0]], G[5:8] + [G[0]], wl.lr)     # runs past the end of the list
