@@ -1051,7 +1051,11 @@ void launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_ma
     const int tiles = tile_end - tile_begin;
     if (tiles <= 0) return;
     const TcTiling tl = choose_tiling(sp.rank);
-    static bool attr_set = false;
+    // the shared-memory opt-in is a per-device attribute of the kernels
+    static bool attr_set_on[64] = {};
+    int device = 0;
+    cudaGetDevice(&device);
+    bool& attr_set = attr_set_on[device & 63];
     if (!attr_set) {
         cudaFuncSetAttribute(project_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
         cudaFuncSetAttribute(project_staged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
@@ -1071,7 +1075,8 @@ void launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_ma
         cfg.numAttrs = 1;
         // the tile loop is persistent: launch exactly as many pairs as can be resident at once
         // (pairs must sit in one GPC, so this can be fewer than half the SMs)
-        static int max_pairs = 0;
+        static int max_pairs_on[64] = {};
+        int& max_pairs = max_pairs_on[device & 63];
         if (max_pairs == 0) {
             int clusters = 0;
             if (cudaOccupancyMaxActiveClusters(&clusters, project_pair_kernel, &cfg) != cudaSuccess || clusters < 1) {
