@@ -171,6 +171,18 @@ APOLLO_API int apollo_projection(uint64_t seed, uint32_t matrix, uint32_t epoch,
 APOLLO_API int apollo_get_path(const apollo_ctx* ctx, int32_t matrix, int32_t* out);
 
 /*
+ * A projection supplied by the caller instead of the seeded Gaussian one: the paper's
+ * "APOLLO w. SVD" variant takes P from a decomposition of the gradient and notes that it
+ * works as well at a much higher cost; the decomposition is the caller's business, this call
+ * only swaps the operand.  d_P: DEVICE, r x m floats, row-major (m = min(rows, cols)), used
+ * as is (R = P G, no 1/sqrt(r) factor) in every later step until replaced; NULL returns
+ * the matrix to the generator.  For bf16 gradients at rank > 1, P is rounded to bfloat16 as
+ * the generated one is.  The buffer stays owned by the caller and must stay alive.  Not
+ * available when the tensor path generates P in shared memory (APOLLO_ERR_UNSUPPORTED).
+ */
+APOLLO_API int apollo_set_projection(apollo_ctx* ctx, int32_t matrix, const float* d_P);
+
+/*
  * Checkpoint and resume.  The optimizer state of Algorithm 1 is, per matrix, the moments M^R
  * and V^R, the limiter's previous norm, the seed and the step counter t (the paper's table of
  * state sizes: "2nr + 2"); P is not part of it because it is regenerated from (seed, matrix

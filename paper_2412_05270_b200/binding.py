@@ -29,7 +29,7 @@ EXPORTS = [
     "apollo_get_scales", "apollo_get_limiter", "apollo_get_state", "apollo_set_delta_out", "apollo_status",
     "apollo_philox_draws", "apollo_projection", "apollo_get_path", "apollo_last_launches", "apollo_strerror",
     "apollo_set_timing", "apollo_get_timing", "apollo_mini_step_static", "apollo_cuda_error_string", "apollo_adamw_step",
-    "apollo_state_bytes", "apollo_state_export", "apollo_state_import", "apollo_step_range",
+    "apollo_state_bytes", "apollo_state_export", "apollo_state_import", "apollo_step_range", "apollo_set_projection",
 ]
 
 
@@ -72,6 +72,7 @@ def load():
                                   ctypes.c_size_t]
     lib.apollo_step.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), f32, f32, vp]
     lib.apollo_step_range.argtypes = [vp, i32, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), f32, f32, i32, vp]
+    lib.apollo_set_projection.argtypes = [vp, i32, vp]
     lib.apollo_destroy.argtypes = [vp]
     lib.apollo_step_count.argtypes = [vp, ctypes.POINTER(ctypes.c_int64)]
     lib.apollo_get_scales.argtypes = [vp, i32, vp, vp]
@@ -249,6 +250,16 @@ class Apollo:
         g = (ctypes.c_void_p * n)(*[x.data_ptr() for x in Gs])
         _check(self.lib.apollo_step_range(self.ctx, first, n, w, g, lr, wd, int(close_step), _stream_ptr(stream)),
                "apollo_step_range")
+
+    def set_projection(self, mat: int, P):
+        """Use the fp32 CUDA tensor P (r x m) as the projection of matrix `mat`; None restores the generator."""
+        if P is not None:
+            m = min(self.shapes[mat])
+            assert P.is_cuda and P.dtype == torch.float32 and tuple(P.shape) == (self.cfg.rank, m) and P.is_contiguous()
+            self._ext_p = getattr(self, "_ext_p", {})
+            self._ext_p[mat] = P                      # keep it alive
+        _check(self.lib.apollo_set_projection(self.ctx, mat, None if P is None else P.data_ptr()),
+               "apollo_set_projection")
 
     def set_delta_out(self, deltas):
         """deltas: list of float32 CUDA tensors shaped like the weights (None entries skip a matrix), or None."""

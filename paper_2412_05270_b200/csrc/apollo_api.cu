@@ -280,6 +280,8 @@ int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_ma
         d.m_pad = (p.m + 63) / 64 * 64;
         d.gpad = p.gpad_bytes ? ctx->ws + p.off_gpad : nullptr;
         d.g_pitch = p.gpad_bytes ? (p.cols + 7) / 8 * 8 : p.cols;
+        d.ext_p = nullptr;
+        d.r_scale = (float)(1.0 / std::sqrt((double)cfg->rank));
         d.rows = p.rows; d.cols = p.cols; d.m = p.m; d.n = p.n; d.tall = p.tall; d.path = p.path;
         d.slices = p.slices; d.g2_slices = p.g2_slices; d.matrix_id = i;
         d.tiles_n = p.tiles_n; d.tiles_k = p.tiles_k;
@@ -548,6 +550,18 @@ int apollo_state_import(apollo_ctx* ctx, const void* d_in, int64_t step_count, v
     if (rc != APOLLO_OK) return rc;
     ctx->t = step_count;
     ctx->imported = true;
+    return APOLLO_OK;
+}
+
+int apollo_set_projection(apollo_ctx* ctx, int32_t matrix, const float* d_P)
+{
+    if (!ctx || matrix < 0 || matrix >= ctx->n_mat) return APOLLO_ERR_INVALID_ARG;
+    if (d_P && ((uintptr_t)d_P % 4)) return APOLLO_ERR_ALIGN;
+    MatDesc& d = ctx->h_descs[matrix];
+    if (d_P && d.path == PATH_TENSOR && !tensor_path_staged()) return APOLLO_ERR_UNSUPPORTED;
+    d.ext_p = d_P;
+    d.r_scale = d_P ? 1.0f : (float)(1.0 / std::sqrt((double)ctx->cfg.rank));
+    ctx->descs_dirty = true;
     return APOLLO_OK;
 }
 

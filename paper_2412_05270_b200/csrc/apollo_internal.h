@@ -36,6 +36,7 @@ struct MatDesc {
     const void* tmap; // 128-byte TMA tensor map of G in device memory (tensor path only)
     const void* tmap_p; // tensor map of the staged P (tensor path with L2 staging)
     void* pstage;     // this matrix's r x m_pad bf16 standard normals in the staging buffer
+    const float* ext_p; // caller-supplied projection (r x m fp32, row-major) used instead of the generator, or nullptr
     void* gpad;       // copy of G with a 16-byte row pitch when cols % 8 != 0 (tensor path), else nullptr
     int32_t rows, cols;
     int32_t m, n;     // m = min(rows, cols) = projected side; n = max = number of channels
@@ -48,7 +49,7 @@ struct MatDesc {
     int32_t tiles_k;  // projection tiles along the other tiled axis (rows of G, or rows of R)
     int32_t m_pad;    // m rounded up to 64: row length of the staged P
     int32_t g_pitch;  // row pitch (elements) of the array the tensor path reads: cols, or cols rounded up to 8
-    int32_t pad1;
+    float r_scale;    // factor applied to the contraction: 1/sqrt(r) for generated standard normals, 1 for a supplied P
 };
 
 struct StepParams {

@@ -130,6 +130,8 @@ extern "C" int apollo_mini_step_static(void* d_W, const void* d_G, int64_t rows,
     d.part = reinterpret_cast<float*>(base + OFF_ARRAYS + bytes_s);
     d.g2 = d.part;   // unused by the streaming path
     d.g2_slices = 0;
+    d.ext_p = nullptr;
+    d.r_scale = 1.0f;
 
     StepParams sp;
     sp.key0 = (uint32_t)(cfg->seed & 0xFFFFFFFFull);

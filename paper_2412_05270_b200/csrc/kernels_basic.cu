@@ -97,8 +97,15 @@ project_stream_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
             const int rows_here = min(STREAM_ROWS, d.rows - i0);
             __syncthreads();   // readers of Ps / red from the previous tile are done
             for (int q = tid; q < STREAM_ROWS / 4; q += STREAM_THREADS) {
-                const float4 z = normal_quad((uint32_t)(i0 / 4 + q), 0u, (uint32_t)d.matrix_id, sp.epoch,
-                                             sp.key0, sp.key1);
+                float4 z;
+                if (d.ext_p) {
+                    const float* src = d.ext_p + i0 + 4 * q;
+                    const int left = d.m - (i0 + 4 * q);
+                    z.x = left > 0 ? __ldg(src) : 0.f; z.y = left > 1 ? __ldg(src + 1) : 0.f;
+                    z.z = left > 2 ? __ldg(src + 2) : 0.f; z.w = left > 3 ? __ldg(src + 3) : 0.f;
+                } else {
+                    z = normal_quad((uint32_t)(i0 / 4 + q), 0u, (uint32_t)d.matrix_id, sp.epoch, sp.key0, sp.key1);
+                }
                 Ps[4 * q + 0] = z.x; Ps[4 * q + 1] = z.y;
                 Ps[4 * q + 2] = z.z; Ps[4 * q + 3] = z.w;
             }
@@ -144,7 +151,7 @@ project_stream_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
 #pragma unroll
                 for (int w = 0; w < 8; ++w) { r += red[0][w][tid]; g2 += red[1][w][tid]; }
                 float2* out = reinterpret_cast<float2*>(d.part) + ((int64_t)tk * d.n + j);
-                *out = make_float2(r * sp.inv_sqrt_r, g2);
+                *out = make_float2(r * d.r_scale, g2);
             }
         } else {
             // channels are the stored rows; the contraction runs along the contiguous side
@@ -155,8 +162,15 @@ project_stream_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
             for (int c0 = 0; c0 < cols; c0 += STREAM_TALL_CHUNK) {
                 __syncthreads();
                 for (int q = tid; q < STREAM_TALL_CHUNK / 4; q += STREAM_THREADS) {
-                    const float4 z = normal_quad((uint32_t)(c0 / 4 + q), 0u, (uint32_t)d.matrix_id, sp.epoch,
-                                                 sp.key0, sp.key1);
+                    float4 z;
+                    if (d.ext_p) {
+                        const float* src = d.ext_p + c0 + 4 * q;
+                        const int left = d.m - (c0 + 4 * q);
+                        z.x = left > 0 ? __ldg(src) : 0.f; z.y = left > 1 ? __ldg(src + 1) : 0.f;
+                        z.z = left > 2 ? __ldg(src + 2) : 0.f; z.w = left > 3 ? __ldg(src + 3) : 0.f;
+                    } else {
+                        z = normal_quad((uint32_t)(c0 / 4 + q), 0u, (uint32_t)d.matrix_id, sp.epoch, sp.key0, sp.key1);
+                    }
                     Ps[4 * q + 0] = z.x; Ps[4 * q + 1] = z.y;
                     Ps[4 * q + 2] = z.z; Ps[4 * q + 3] = z.w;
                 }
@@ -190,7 +204,7 @@ project_stream_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                 }
                 const int j = j_base + rr;
                 if (lane == 0 && j < d.rows)
-                    reinterpret_cast<float2*>(d.part)[j] = make_float2(r * sp.inv_sqrt_r, g2);
+                    reinterpret_cast<float2*>(d.part)[j] = make_float2(r * d.r_scale, g2);
             }
         }
     }
@@ -224,6 +238,8 @@ project_simt_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
         const int j0 = tn * SIMT_BN, k0 = tr * SIMT_BR;
         const T* __restrict__ G = static_cast<const T*>(d.G);
         const int cols = d.cols, m = d.m, n = d.n, r = sp.rank;
+        const float r_scale = d.r_scale;
+        const float* __restrict__ ext_p = d.ext_p;
 
         float acc[4][4];
 #pragma unroll
@@ -238,9 +254,17 @@ project_simt_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             for (int at = tid; at < SIMT_BR * (SIMT_BK / 4); at += SIMT_THREADS) {
                 const int row = at / (SIMT_BK / 4), q = at % (SIMT_BK / 4);
                 float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (k0 + row < r)
-                    z = normal_quad((uint32_t)(i0 / 4 + q), (uint32_t)(k0 + row), (uint32_t)d.matrix_id, sp.epoch,
-                                    sp.key0, sp.key1);
+                if (k0 + row < r) {
+                    if (ext_p) {
+                        const float* src = ext_p + (int64_t)(k0 + row) * m + i0 + 4 * q;
+                        const int left = m - (i0 + 4 * q);
+                        z.x = left > 0 ? __ldg(src) : 0.f; z.y = left > 1 ? __ldg(src + 1) : 0.f;
+                        z.z = left > 2 ? __ldg(src + 2) : 0.f; z.w = left > 3 ? __ldg(src + 3) : 0.f;
+                    } else {
+                        z = normal_quad((uint32_t)(i0 / 4 + q), (uint32_t)(k0 + row), (uint32_t)d.matrix_id, sp.epoch,
+                                        sp.key0, sp.key1);
+                    }
+                }
                 if (sizeof(T) == 2) {   // bf16 gradients: P has the precision of the GEMM operands
                     z.x = round_to_bf16(z.x); z.y = round_to_bf16(z.y); z.z = round_to_bf16(z.z); z.w = round_to_bf16(z.w);
                 }
@@ -287,7 +311,7 @@ project_simt_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             for (int y = 0; y < 4; ++y) {
                 const int j = j0 + tx * 4 + y;
                 if (k < r && j < n) {
-                    const float rv = acc[x][y] * sp.inv_sqrt_r;
+                    const float rv = acc[x][y] * r_scale;
                     const int64_t at = (int64_t)k * n + j;
                     const float mv = sp.beta1 * d.M[at] + (1.0f - sp.beta1) * rv;
                     const float vv = sp.beta2 * d.V[at] + (1.0f - sp.beta2) * rv * rv;

@@ -279,6 +279,7 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
         const uint32_t matrix_id = (uint32_t)__ldg(&dp->matrix_id);
         const void* tmap = dp->tmap;
         const void* tmap_p = dp->tmap_p;
+        const float r_scale = __ldg(&dp->r_scale);
         float* const Mbase = dp->M;
         float* const Vbase = dp->V;
         float* const part = dp->part;
@@ -460,7 +461,7 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                     for (int k = 0; k < 16; ++k) { mv[k] = Mp[(int64_t)k * n]; vv[k] = Vp[(int64_t)k * n]; }
 #pragma unroll
                     for (int k = 0; k < 16; ++k) {
-                        const float r = rv[k] * sp.inv_sqrt_r;
+                        const float r = rv[k] * r_scale;
                         const float mn = sp.beta1 * mv[k] + (1.0f - sp.beta1) * r;
                         const float vn = sp.beta2 * vv[k] + (1.0f - sp.beta2) * r * r;
                         Mp[(int64_t)k * n] = mn; Vp[(int64_t)k * n] = vn;
@@ -693,6 +694,7 @@ project_staged_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
             const int ch = q * 32 + lane, j = j0 + ch;
             float* const Mbase = dp->M;
             float* const Vbase = dp->V;
+            const float r_scale = __ldg(&dp->r_scale);
             wait_phase(bar_acc_full + 8 * buf, use & 1, abort_flag, status);
             ptx::tc_fence_after_sync();
             float num = 0.f, den = 0.f;
@@ -708,7 +710,7 @@ project_staged_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                     for (int k = 0; k < 16; ++k) { mv[k] = Mp[(int64_t)k * n]; vv[k] = Vp[(int64_t)k * n]; }
 #pragma unroll
                     for (int k = 0; k < 16; ++k) {
-                        const float r = rv[k] * sp.inv_sqrt_r;
+                        const float r = rv[k] * r_scale;
                         const float mn = sp.beta1 * mv[k] + (1.0f - sp.beta1) * r;
                         const float vn = sp.beta2 * vv[k] + (1.0f - sp.beta2) * r * r;
                         Mp[(int64_t)k * n] = mn; Vp[(int64_t)k * n] = vn;
@@ -948,6 +950,7 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             const int ch = q * 32 + lane, j = j0 + ch;
             float* const Mbase = dp->M;
             float* const Vbase = dp->V;
+            const float r_scale = __ldg(&dp->r_scale);
             wait_phase(bar_acc_full + 8 * buf, use & 1, abort_flag, status);
             ptx::tc_fence_after_sync();
             float num = 0.f, den = 0.f;
@@ -963,7 +966,7 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                     for (int k = 0; k < 16; ++k) { mv[k] = Mp[(int64_t)k * n]; vv[k] = Vp[(int64_t)k * n]; }
 #pragma unroll
                     for (int k = 0; k < 16; ++k) {
-                        const float r = rv[k] * sp.inv_sqrt_r;
+                        const float r = rv[k] * r_scale;
                         const float mn = sp.beta1 * mv[k] + (1.0f - sp.beta1) * r;
                         const float vn = sp.beta2 * vv[k] + (1.0f - sp.beta2) * r * r;
                         Mp[(int64_t)k * n] = mn; Vp[(int64_t)k * n] = vn;
@@ -1003,8 +1006,21 @@ __global__ void generate_p_kernel(const MatDesc* __restrict__ descs, int mat_beg
     uint4* out = static_cast<uint4*>(dp->pstage);
     const int chunks_per_row = m_pad / 8;
     const int total = sp.rank * chunks_per_row;
+    const float* __restrict__ ext_p = dp->ext_p;
+    const int m = __ldg(&dp->m);
     for (int c = blockIdx.x * blockDim.x + threadIdx.x; c < total; c += gridDim.x * blockDim.x) {
         const int row = c / chunks_per_row, ch = c - row * chunks_per_row;
+        if (ext_p) {
+            // a projection supplied by the caller: convert its row to bf16, zero the padding
+            float z[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) z[e] = 8 * ch + e < m ? __ldg(ext_p + (int64_t)row * m + 8 * ch + e) : 0.f;
+            uint4 v;
+            v.x = pack_bf16x2(z[0], z[1]); v.y = pack_bf16x2(z[2], z[3]);
+            v.z = pack_bf16x2(z[4], z[5]); v.w = pack_bf16x2(z[6], z[7]);
+            out[c] = v;
+            continue;
+        }
         const float4 a0 = normal_quad_fast((uint32_t)(2 * ch), (uint32_t)row, matrix_id, sp.epoch, sp.round_key);
         const float4 a1 = normal_quad_fast((uint32_t)(2 * ch + 1), (uint32_t)row, matrix_id, sp.epoch, sp.round_key);
         uint4 v;

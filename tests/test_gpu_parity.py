@@ -202,3 +202,52 @@ def test_layer_wise_range_steps_equal_the_whole_list_step(rank, mode, flags):
     assert whole.status() == B.OK and ranged.status() == B.OK
     with pytest.raises(B.ApolloError):
         ranged.step_range(5, Wb[5:8] + [Wb[0]], G[5:8] + [G[0]], wl.lr)     # runs past the end of the list
+
+
+@pytest.mark.parametrize("rank,dtype,flags,path", [
+    (16, "bf16", 0, B.PATH_TENSOR), (4, "f32", 0, B.PATH_SIMT), (6, "bf16", B.FLAG_NO_TENSOR_CORES, B.PATH_SIMT),
+    (1, "bf16", 0, B.PATH_STREAM),
+])
+def test_caller_supplied_projection_from_an_svd(rank, dtype, flags, path):
+    """The "APOLLO w. SVD" variant: P = top-r left singular vectors of the first gradient (computed here
+    with torch on the CPU), handed to the library and to the oracle alike."""
+    import numpy as np
+    import oracle
+    from parity import DW_ABS, DW_REL, SCALE_REL, _f32
+    shapes = [(96, 200), (203, 72)]
+    wl = _wl(shapes, rank, mode="tensor" if rank == 1 else "channel", dtype=dtype, T=100, steps=3, wd=0.01,
+             alpha=1.0)
+    dev = torch.device("cuda")
+    opt = B.Apollo(wl.shapes, B.config_for(wl, flags))
+    Ps, orc = [], []
+    for i, (rows, cols) in enumerate(shapes):
+        assert opt.path(i) == path
+        G0 = WL.make_grad(wl, i, 0).float()
+        Gv = G0 if rows <= cols else G0.T
+        U, _, _ = torch.linalg.svd(Gv.double(), full_matrices=False)
+        P = U[:, :rank].T.contiguous().float()              # r x m, orthonormal rows
+        if dtype == "bf16" and rank > 1:
+            P = P.to(torch.bfloat16).float()                # the operand precision of the projection
+        Ps.append(P.to(dev))
+        opt.set_projection(i, Ps[-1])
+        orc.append(oracle.MatrixOracle(rows, cols, rank=rank, mode=oracle.MODE_TENSOR if rank == 1 else oracle.MODE_CHANNEL,
+                                       dtype=oracle.DT_BF16 if dtype == "bf16" else oracle.DT_F32, matrix_id=i,
+                                       alpha=1.0, gamma=_f32(wl.gamma), beta1=_f32(wl.beta1), beta2=_f32(wl.beta2),
+                                       eps=_f32(wl.eps)))
+    W = [WL.make_weight(wl, i).to(dev) for i in range(2)]
+    deltas = [torch.zeros(s, dtype=torch.float32, device=dev) for s in shapes]
+    opt.set_delta_out(deltas)
+    for t in range(3):
+        G = [WL.make_grad(wl, i, t) for i in range(2)]
+        Wc = [w.float().cpu().numpy() for w in W]
+        opt.step(W, [g.to(dev) for g in G], wl.lr, wl.wd)
+        torch.cuda.synchronize()
+        for i in range(2):
+            res = orc[i].step(Wc[i], G[i].float().numpy(), _f32(wl.lr), _f32(wl.wd), P=Ps[i].double().cpu().numpy())
+            bound = DW_REL * np.max(np.abs(res.dW)) + DW_ABS
+            assert np.max(np.abs(deltas[i].cpu().numpy() - res.dW)) <= bound
+            s_gpu = opt.scales(i).cpu().numpy()
+            assert np.max(np.abs(s_gpu - res.s) / np.abs(res.s)) <= SCALE_REL
+            W[i].copy_(torch.from_numpy(res.W).to(W[i].dtype))
+    opt.set_projection(0, None)                             # back to the generator
+    opt.close()
