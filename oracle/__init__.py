@@ -41,7 +41,7 @@ def build(force: bool = False) -> Path:
 class _Config(ctypes.Structure):
     _fields_ = [
         ("rank", ctypes.c_int32), ("mode", ctypes.c_int32), ("dtype", ctypes.c_int32),
-        ("bias_correction", ctypes.c_int32),
+        ("bias_correction", ctypes.c_int32), ("state_bf16", ctypes.c_int32), ("pad_", ctypes.c_int32),
         ("alpha", ctypes.c_double), ("gamma", ctypes.c_double),
         ("beta1", ctypes.c_double), ("beta2", ctypes.c_double), ("eps", ctypes.c_double),
     ]
@@ -125,10 +125,10 @@ class MatrixOracle:
     def __init__(self, rows: int, cols: int, rank: int, mode: int = MODE_CHANNEL, dtype: int = DT_F32,
                  seed: int = 0, matrix_id: int = 0, T: int = 200, alpha: float = 1.0, gamma: float = 1.01,
                  beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
-                 bias_correction: bool = False, p_round_bf16: bool = False):
+                 bias_correction: bool = False, p_round_bf16: bool = False, state_bf16: bool = False):
         self.rows, self.cols = int(rows), int(cols)
         self.m, self.n = min(rows, cols), max(rows, cols)
-        self.cfg = _Config(rank, mode, dtype, int(bias_correction), alpha, gamma, beta1, beta2, eps)
+        self.cfg = _Config(rank, mode, dtype, int(bias_correction), int(state_bf16), 0, alpha, gamma, beta1, beta2, eps)
         self.seed, self.matrix_id, self.T = int(seed), int(matrix_id), int(T)
         self.p_round_bf16 = bool(p_round_bf16)
         self.M = np.zeros((rank, self.n), dtype=np.float64)

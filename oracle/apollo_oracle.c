@@ -160,6 +160,8 @@ typedef struct {
     int32_t mode;             /* 0 = channel-wise scales (APOLLO), 1 = one tensor-wise scale (Mini) */
     int32_t dtype;            /* 0 = fp32 weights, 1 = bf16 weights (only the final store differs) */
     int32_t bias_correction;  /* 0 = moment equations exactly as printed; 1 = Adam's 1/(1-beta^t) terms */
+    int32_t state_bf16;       /* 1 = M and V are kept in bfloat16: rounded after each update (R~ uses the unrounded values) */
+    int32_t pad_;
     double alpha, gamma;      /* gradient scale factor; limiter threshold (<= 0 disables it) */
     double beta1, beta2, eps;
 } oracle_config;
@@ -215,6 +217,7 @@ int oracle_apollo_step_with_P(const oracle_config* cfg, const double* P,
         M[e] = cfg->beta1 * M[e] + (1.0 - cfg->beta1) * R[e];
         V[e] = cfg->beta2 * V[e] + (1.0 - cfg->beta2) * R[e] * R[e];
         Rt[e] = (M[e] / bc1) / (sqrt(V[e] / bc2) + cfg->eps);
+        if (cfg->state_bf16) { M[e] = oracle_round_bf16(M[e]); V[e] = oracle_round_bf16(V[e]); }
     }
 
     /* step 4: scales (Eq. 5 per channel; one ratio of Frobenius norms for Mini) */

@@ -311,3 +311,23 @@ def test_rank_above_short_side_is_rejected():
     mo = MatrixOracle(4, 9, rank=5)
     with pytest.raises(ValueError):
         mo.step(np.zeros((4, 9), dtype=np.float32), np.zeros((4, 9), dtype=np.float32), 0.1, 0.0)
+
+
+def test_bf16_state_variant_rounds_the_moments_after_each_update():
+    # Table 3's optimizer-state size (1.6 G at r = 256 for the 7B model) is two bytes per moment entry.
+    import torch
+    m, n, r = 6, 9, 3
+    P = oracle.projection(4, 0, 0, r, m)
+    mo = MatrixOracle(m, n, rank=r, seed=4, T=1000, gamma=0.0, state_bf16=True)
+    W = np.zeros((m, n), dtype=np.float32)
+    M = np.zeros((r, n)); V = np.zeros((r, n))
+    rb = lambda a: torch.from_numpy(a).float().to(torch.bfloat16).double().numpy()
+    for G in _grads(m, n, 4, seed=23, scale=1.0):
+        res = mo.step(W, G, lr=0.1, wd=0.0, want_R=True)
+        R = P @ G.astype(np.float64)
+        Mn = 0.9 * M + 0.1 * R
+        Vn = 0.999 * V + 0.001 * R * R
+        s = np.linalg.norm(Mn / (np.sqrt(Vn) + 1e-8), axis=0) / np.linalg.norm(R, axis=0)   # from the unrounded values
+        np.testing.assert_allclose(res.s, s, rtol=1e-12)
+        M, V = rb(Mn), rb(Vn)
+        assert np.array_equal(mo.M, M) and np.array_equal(mo.V, V)
