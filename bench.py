@@ -37,15 +37,16 @@ def measured_peaks():
     return dict(FALLBACK_PEAKS) | {"source": "fallback"}
 
 
-def step_bytes(wl: WL.Workload):
+def step_bytes(wl: WL.Workload, state_elem: int = 4):
     """Algorithmic HBM bytes of one step: G read by both passes, W read and written,
-    fp32 M and V read and written (B_2p), and the single-read-of-G variant (B_min)."""
+    M and V (state_elem bytes per entry) read and written (B_2p), and the single-read-of-G
+    variant (B_min)."""
     e = 2 if wl.dtype == "bf16" else 4
     two_pass = minimal = flops = update = 0
     for rows, cols in wl.shapes:
         n = max(rows, cols)
-        two_pass += 4 * e * rows * cols + 16 * wl.rank * n
-        minimal += 3 * e * rows * cols + 16 * wl.rank * n
+        two_pass += 4 * e * rows * cols + 4 * state_elem * wl.rank * n
+        minimal += 3 * e * rows * cols + 4 * state_elem * wl.rank * n
         update += 3 * e * rows * cols
         flops += 2 * wl.rank * rows * cols
     return two_pass, minimal, update, flops
@@ -173,7 +174,7 @@ def run_ours(args, wl, rank, world, local_rank):
     n = len(wl.shapes)
     Ws = [WL.make_weight(wl, i, device=dev) for i in range(n)]
     Gs = [WL.make_grad(wl, i, 0, device=dev) for i in range(n)]
-    opt = B.Apollo(wl.shapes, B.config_for(wl), device=dev)
+    opt = B.Apollo(wl.shapes, B.config_for(wl, B.FLAG_BF16_STATES if args.bf16_states else 0), device=dev)
     opt.set_timing(True)
     stream = torch.cuda.current_stream()
 
@@ -232,7 +233,7 @@ def run_ours(args, wl, rank, world, local_rank):
 
     peaks = measured_peaks()
     ms_step = ms_total / args.steps
-    two_pass, minimal, update_bytes, flops = step_bytes(wl)
+    two_pass, minimal, update_bytes, flops = step_bytes(wl, 2 if args.bf16_states else 4)
     value = whole_job_value(wl.params, world, ms_step)
     hbm, tc = peaks["hbm_gbs"] * 1e9, peaks["bf16_tflops_sustained"] * 1e12
     t_roof = max(two_pass / hbm, flops / tc)
@@ -243,7 +244,7 @@ def run_ours(args, wl, rank, world, local_rank):
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32",
         "data": "synthetic",
         "config": {"workload": wl.name, "matrices": n, "params": wl.params, "rank": wl.rank, "mode": wl.mode,
-                   "T": wl.T, "lr": wl.lr, "wd": wl.wd, "states": "f32", "replicas": world,
+                   "T": wl.T, "lr": wl.lr, "wd": wl.wd, "states": "bf16" if args.bf16_states else "f32", "replicas": world,
                    "l2": "inputs (W, G: %.1f GB) exceed L2, no flush" % (2 * wl.params * 2 / 1e9)},
         "roofline": {"bound": "hbm", "kernel": "update_kernel", "achieved": upd_gbs, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": upd_gbs / peaks["hbm_gbs"],
@@ -298,6 +299,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="keep only the first LAYERS layers (profiling aid)")
     ap.add_argument("--adamw", action="store_true", help="also time the fused AdamW of the non-projected parameters")
+    ap.add_argument("--bf16-states", action="store_true", help="keep M and V in bfloat16 (a variant, not the headline)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

@@ -64,6 +64,8 @@ extern "C" {
 
 /* apollo_config.flags */
 #define APOLLO_FLAG_NO_TENSOR_CORES 1u /* run the projection on the CUDA cores (test and comparison aid) */
+#define APOLLO_FLAG_BF16_STATES 2u     /* keep M and V in bfloat16 (two bytes per entry, as the paper's state-size
+                                          figures assume); R~ is formed from the unrounded update */
 
 typedef struct apollo_ctx apollo_ctx; /* opaque HOST object */
 
@@ -135,7 +137,8 @@ APOLLO_API int apollo_step_count(const apollo_ctx* ctx, int64_t* out);
  * apollo_get_scales:  d_out DEVICE, n floats: s_j of the last step (Eq. 5), n = max(rows, cols).
  * apollo_get_limiter: d_out DEVICE, 4 floats: {norm after limiting (Eq. 4), factor c,
  *                     norm before limiting, tensor-wise scale (tensor mode, else 0)}.
- * apollo_get_state:   d_M, d_V DEVICE, r x n floats each, row-major (channel index contiguous).
+ * apollo_get_state:   d_M, d_V DEVICE, r x n floats each, row-major (channel index contiguous);
+ *                     bfloat16 states are widened to float.
  */
 APOLLO_API int apollo_get_scales(apollo_ctx* ctx, int32_t matrix, float* d_out, void* cuda_stream);
 APOLLO_API int apollo_get_limiter(apollo_ctx* ctx, int32_t matrix, float* d_out, void* cuda_stream);
@@ -187,7 +190,8 @@ APOLLO_API int apollo_set_projection(apollo_ctx* ctx, int32_t matrix, const floa
  * and V^R, the limiter's previous norm, the seed and the step counter t (the paper's table of
  * state sizes: "2nr + 2"); P is not part of it because it is regenerated from (seed, matrix
  * index, floor(t / T)).  apollo_state_bytes gives the size of the flat DEVICE buffer:
- * per matrix in list order M (r x n floats), V (r x n floats), one float (previous norm).
+ * per matrix in list order M (r x n entries), V (r x n entries), one float (previous norm);
+ * entries are floats, or bfloat16 with APOLLO_FLAG_BF16_STATES.
  * apollo_state_export copies the state out (after at least one step or an import);
  * apollo_state_import copies it in and sets the step counter; the context must have been
  * created with the same shapes and configuration (the seed and t are the caller's to keep:

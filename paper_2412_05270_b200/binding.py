@@ -22,6 +22,7 @@ STATIC_SCRATCH_BYTES = 8 << 20
 SCALE_CHANNEL, SCALE_TENSOR = 0, 1
 DT_F32, DT_BF16 = 0, 1
 FLAG_NO_TENSOR_CORES = 1
+FLAG_BF16_STATES = 2
 PATH_STREAM, PATH_SIMT, PATH_TENSOR = 0, 1, 2
 
 EXPORTS = [

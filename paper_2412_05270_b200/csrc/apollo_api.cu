@@ -146,7 +146,7 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
     plan.zero_begin = off;
     for (int i = 0; i < n_mat; ++i) {
         MatPlan& p = plan.mats[i];
-        const size_t state = sizeof(float) * (size_t)r * (size_t)p.n;
+        const size_t state = ((cfg->flags & APOLLO_FLAG_BF16_STATES) ? 2 : sizeof(float)) * (size_t)r * (size_t)p.n;
         p.off_M = off; off = align_up(off + state);
         p.off_V = off; off = align_up(off + state);
         p.off_scal = off; off += ALIGN;     // scal[4] then prev at float index 8
@@ -385,6 +385,7 @@ static int step_range(apollo_ctx* ctx, int first, int count, void* const* d_W, c
     sp.key0 = (uint32_t)(cfg.seed & 0xFFFFFFFFull);
     sp.key1 = (uint32_t)(cfg.seed >> 32);
     fill_round_keys(sp);
+    sp.state_bf16 = (cfg.flags & APOLLO_FLAG_BF16_STATES) ? 1 : 0;
     sp.epoch = (uint32_t)(ctx->t / cfg.T);
     sp.rank = cfg.rank; sp.mode = cfg.mode;
     sp.inv_sqrt_r = (float)(1.0 / std::sqrt((double)cfg.rank));
@@ -481,10 +482,15 @@ int apollo_get_state(apollo_ctx* ctx, int32_t matrix, float* d_M, float* d_V, vo
 {
     if (!ctx || !d_M || !d_V || matrix < 0 || matrix >= ctx->n_mat) return APOLLO_ERR_INVALID_ARG;
     const MatDesc& d = ctx->h_descs[matrix];
-    const size_t bytes = sizeof(float) * (size_t)ctx->cfg.rank * (size_t)d.n;
+    const size_t count = (size_t)ctx->cfg.rank * (size_t)d.n;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    if (cudaMemcpyAsync(d_M, d.M, bytes, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) return APOLLO_ERR_CUDA;
-    if (cudaMemcpyAsync(d_V, d.V, bytes, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) return APOLLO_ERR_CUDA;
+    if (ctx->cfg.flags & APOLLO_FLAG_BF16_STATES) {
+        launch_widen_bf16(d.M, d_M, count, stream);
+        launch_widen_bf16(d.V, d_V, count, stream);
+        return cuda_ok(cudaGetLastError()) ? APOLLO_OK : APOLLO_ERR_CUDA;
+    }
+    if (cudaMemcpyAsync(d_M, d.M, sizeof(float) * count, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) return APOLLO_ERR_CUDA;
+    if (cudaMemcpyAsync(d_V, d.V, sizeof(float) * count, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) return APOLLO_ERR_CUDA;
     return APOLLO_OK;
 }
 
@@ -503,6 +509,8 @@ int apollo_status(apollo_ctx* ctx, void* cuda_stream)
     return APOLLO_OK;
 }
 
+static size_t state_elem_bytes(const apollo_ctx* ctx) { return (ctx->cfg.flags & APOLLO_FLAG_BF16_STATES) ? 2 : sizeof(float); }
+
 // Checkpoint layout: for each matrix in list order M (r x n floats), V (r x n floats), then one
 // float: the limiter's previous norm.
 int apollo_state_bytes(const apollo_ctx* ctx, size_t* out_bytes)
@@ -510,18 +518,18 @@ int apollo_state_bytes(const apollo_ctx* ctx, size_t* out_bytes)
     if (!ctx || !out_bytes) return APOLLO_ERR_INVALID_ARG;
     size_t total = 0;
     for (int i = 0; i < ctx->n_mat; ++i)
-        total += sizeof(float) * (2 * (size_t)ctx->cfg.rank * (size_t)ctx->h_descs[i].n + 1);
+        total += state_elem_bytes(ctx) * 2 * (size_t)ctx->cfg.rank * (size_t)ctx->h_descs[i].n + sizeof(float);
     *out_bytes = total;
     return APOLLO_OK;
 }
 
 static int state_copy(apollo_ctx* ctx, char* d_flat, bool to_flat, cudaStream_t stream)
 {
-    if (((uintptr_t)d_flat % 4) != 0) return APOLLO_ERR_ALIGN;
+    if (((uintptr_t)d_flat % 2) != 0) return APOLLO_ERR_ALIGN;
     size_t at = 0;
     for (int i = 0; i < ctx->n_mat; ++i) {
         const MatDesc& d = ctx->h_descs[i];
-        const size_t bytes = sizeof(float) * (size_t)ctx->cfg.rank * (size_t)d.n;
+        const size_t bytes = state_elem_bytes(ctx) * (size_t)ctx->cfg.rank * (size_t)d.n;
         void* parts[3] = { d.M, d.V, d.prev };
         const size_t sizes[3] = { bytes, bytes, sizeof(float) };
         for (int k = 0; k < 3; ++k) {

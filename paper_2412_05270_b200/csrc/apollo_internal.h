@@ -26,7 +26,7 @@ struct MatDesc {
     void* W;
     const void* G;
     float* dW;        // optional fp32 capture of the update, or nullptr
-    float* M;         // r x n, row-major
+    float* M;         // r x n, row-major; fp32, or bfloat16 behind the same pointer when StepParams::state_bf16
     float* V;         // r x n
     float* s;         // n scales of the last step
     float* part;      // projection partial sums, layout depends on the path (see kernels)
@@ -60,6 +60,7 @@ struct StepParams {
     float lr, wd, alpha, gamma;
     float beta1, beta2, eps;
     float inv_bc1, inv_bc2;   // 1/(1-beta^t) with bias correction, else 1
+    int32_t state_bf16;       // 1: M and V are stored as bfloat16 (APOLLO_FLAG_BF16_STATES)
     uint32_t round_key[20];   // Philox key schedule: {key0 + i W0, key1 + i W1}, i = 0..9
 };
 

@@ -137,6 +137,7 @@ extern "C" int apollo_mini_step_static(void* d_W, const void* d_G, int64_t rows,
     sp.key0 = (uint32_t)(cfg->seed & 0xFFFFFFFFull);
     sp.key1 = (uint32_t)(cfg->seed >> 32);
     fill_round_keys(sp);
+    sp.state_bf16 = 0;
     sp.epoch = (uint32_t)(t / cfg->T);
     sp.rank = 1; sp.mode = cfg->mode;
     sp.inv_sqrt_r = 1.0f;

@@ -104,6 +104,17 @@ __device__ __forceinline__ void load8_guarded(const T* p, int count, float (&v)[
     for (int e = 0; e < 8; ++e) v[e] = e < count ? load1(p + e) : 0.0f;
 }
 
+// Moment storage: fp32, or bfloat16 behind the same pointer (rounded to nearest even on store).
+__device__ __forceinline__ float state_load(const float* base, int64_t idx, bool bf16)
+{
+    return bf16 ? bf16_bits_to_float((uint32_t)reinterpret_cast<const unsigned short*>(base)[idx]) : base[idx];
+}
+__device__ __forceinline__ void state_store(float* base, int64_t idx, float v, bool bf16)
+{
+    if (bf16) reinterpret_cast<__nv_bfloat16*>(base)[idx] = __float2bfloat16_rn(v);
+    else base[idx] = v;
+}
+
 // Sum of one double per thread over the block, in a fixed order (deterministic).
 // `scratch` holds at least 32 doubles; every thread gets the result.
 __device__ __forceinline__ double block_sum(double v, double* scratch)

@@ -17,6 +17,9 @@ void launch_update(int dtype, const MatDesc* d_descs, const int* d_prefix, int n
                    const StepParams& sp, int sm_count, cudaStream_t stream);
 
 
+// bfloat16 -> float copy (observability of bfloat16 states).
+void launch_widen_bf16(const void* d_src, float* d_dst, size_t count, cudaStream_t stream);
+
 // Tensor-core projection (TMA + tcgen05 + TMEM).
 bool tensor_path_supports(int rows, int cols, int rank, int dtype);
 void tensor_path_tiling(int rows, int cols, int rank, int32_t* tiles_n, int32_t* tiles_k);

@@ -313,9 +313,10 @@ project_simt_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                 if (k < r && j < n) {
                     const float rv = acc[x][y] * r_scale;
                     const int64_t at = (int64_t)k * n + j;
-                    const float mv = sp.beta1 * d.M[at] + (1.0f - sp.beta1) * rv;
-                    const float vv = sp.beta2 * d.V[at] + (1.0f - sp.beta2) * rv * rv;
-                    d.M[at] = mv; d.V[at] = vv;
+                    const bool sb = sp.state_bf16 != 0;
+                    const float mv = sp.beta1 * state_load(d.M, at, sb) + (1.0f - sp.beta1) * rv;
+                    const float vv = sp.beta2 * state_load(d.V, at, sb) + (1.0f - sp.beta2) * rv * rv;
+                    state_store(d.M, at, mv, sb); state_store(d.V, at, vv, sb);
                     const float rt = (mv * sp.inv_bc1) / (sqrtf(vv * sp.inv_bc2) + sp.eps);
                     num[y] = fmaf(rt, rt, num[y]);
                     den[y] = fmaf(rv, rv, den[y]);
@@ -360,9 +361,10 @@ finalize_kernel(const MatDesc* __restrict__ descs, int first, StepParams sp)
                 const float2 p = reinterpret_cast<const float2*>(d.part)[(int64_t)sl * n + j];
                 r += p.x; g2 += p.y;
             }
-            const float mv = sp.beta1 * d.M[j] + (1.0f - sp.beta1) * r;
-            const float vv = sp.beta2 * d.V[j] + (1.0f - sp.beta2) * r * r;
-            d.M[j] = mv; d.V[j] = vv;
+            const bool sb = sp.state_bf16 != 0;
+            const float mv = sp.beta1 * state_load(d.M, j, sb) + (1.0f - sp.beta1) * r;
+            const float vv = sp.beta2 * state_load(d.V, j, sb) + (1.0f - sp.beta2) * r * r;
+            state_store(d.M, j, mv, sb); state_store(d.V, j, vv, sb);
             const float rt = (mv * sp.inv_bc1) / (sqrtf(vv * sp.inv_bc2) + sp.eps);
             num = rt * rt; den = r * r;
         } else {
@@ -533,6 +535,18 @@ update_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix,
             }
         }
     }
+}
+
+__global__ void widen_bf16_kernel(const unsigned short* __restrict__ src, float* __restrict__ dst, size_t count)
+{
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < count; i += (size_t)gridDim.x * blockDim.x)
+        dst[i] = bf16_bits_to_float((uint32_t)src[i]);
+}
+
+void launch_widen_bf16(const void* d_src, float* d_dst, size_t count, cudaStream_t stream)
+{
+    if (count == 0) return;
+    widen_bf16_kernel<<<blocks_for((int64_t)count), 256, 0, stream>>>(static_cast<const unsigned short*>(d_src), d_dst, count);
 }
 
 // ----------------------------------------------------------------------------------------

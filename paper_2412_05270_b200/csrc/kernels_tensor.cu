@@ -454,17 +454,20 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                 ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * r_slice + cchunk * 16), rv);
                 const int j = j0 + b * 128 + ch_in_blk;
                 if (j < n) {
-                    float* Mp = Mbase + (int64_t)(r0 + cchunk * 16) * n + j;
-                    float* Vp = Vbase + (int64_t)(r0 + cchunk * 16) * n + j;
+                    const int64_t at = (int64_t)(r0 + cchunk * 16) * n + j;
+                    const bool sb = sp.state_bf16 != 0;
                     float mv[16], vv[16];
 #pragma unroll
-                    for (int k = 0; k < 16; ++k) { mv[k] = Mp[(int64_t)k * n]; vv[k] = Vp[(int64_t)k * n]; }
+                    for (int k = 0; k < 16; ++k) {
+                        mv[k] = state_load(Mbase, at + (int64_t)k * n, sb);
+                        vv[k] = state_load(Vbase, at + (int64_t)k * n, sb);
+                    }
 #pragma unroll
                     for (int k = 0; k < 16; ++k) {
                         const float r = rv[k] * r_scale;
                         const float mn = sp.beta1 * mv[k] + (1.0f - sp.beta1) * r;
                         const float vn = sp.beta2 * vv[k] + (1.0f - sp.beta2) * r * r;
-                        Mp[(int64_t)k * n] = mn; Vp[(int64_t)k * n] = vn;
+                        state_store(Mbase, at + (int64_t)k * n, mn, sb); state_store(Vbase, at + (int64_t)k * n, vn, sb);
                         const float rt = __fdividef(mn * sp.inv_bc1, fast_sqrt(vn * sp.inv_bc2) + sp.eps);
                         num = fmaf(rt, rt, num);
                         den = fmaf(r, r, den);
@@ -703,17 +706,20 @@ project_staged_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                 float rv[16];
                 ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + buf * (uint32_t)r_slice + (uint32_t)(cchunk * 16), rv);
                 if (j < n) {
-                    float* Mp = Mbase + (int64_t)(r0 + cchunk * 16) * n + j;
-                    float* Vp = Vbase + (int64_t)(r0 + cchunk * 16) * n + j;
+                    const int64_t at = (int64_t)(r0 + cchunk * 16) * n + j;
+                    const bool sb = sp.state_bf16 != 0;
                     float mv[16], vv[16];
 #pragma unroll
-                    for (int k = 0; k < 16; ++k) { mv[k] = Mp[(int64_t)k * n]; vv[k] = Vp[(int64_t)k * n]; }
+                    for (int k = 0; k < 16; ++k) {
+                        mv[k] = state_load(Mbase, at + (int64_t)k * n, sb);
+                        vv[k] = state_load(Vbase, at + (int64_t)k * n, sb);
+                    }
 #pragma unroll
                     for (int k = 0; k < 16; ++k) {
                         const float r = rv[k] * r_scale;
                         const float mn = sp.beta1 * mv[k] + (1.0f - sp.beta1) * r;
                         const float vn = sp.beta2 * vv[k] + (1.0f - sp.beta2) * r * r;
-                        Mp[(int64_t)k * n] = mn; Vp[(int64_t)k * n] = vn;
+                        state_store(Mbase, at + (int64_t)k * n, mn, sb); state_store(Vbase, at + (int64_t)k * n, vn, sb);
                         const float rt = __fdividef(mn * sp.inv_bc1, fast_sqrt(vn * sp.inv_bc2) + sp.eps);
                         num = fmaf(rt, rt, num);
                         den = fmaf(r, r, den);
@@ -959,17 +965,20 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                 float rv[16];
                 ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + buf * (uint32_t)r_slice + (uint32_t)(cchunk * 16), rv);
                 if (j < n) {
-                    float* Mp = Mbase + (int64_t)(r0 + cchunk * 16) * n + j;
-                    float* Vp = Vbase + (int64_t)(r0 + cchunk * 16) * n + j;
+                    const int64_t at = (int64_t)(r0 + cchunk * 16) * n + j;
+                    const bool sb = sp.state_bf16 != 0;
                     float mv[16], vv[16];
 #pragma unroll
-                    for (int k = 0; k < 16; ++k) { mv[k] = Mp[(int64_t)k * n]; vv[k] = Vp[(int64_t)k * n]; }
+                    for (int k = 0; k < 16; ++k) {
+                        mv[k] = state_load(Mbase, at + (int64_t)k * n, sb);
+                        vv[k] = state_load(Vbase, at + (int64_t)k * n, sb);
+                    }
 #pragma unroll
                     for (int k = 0; k < 16; ++k) {
                         const float r = rv[k] * r_scale;
                         const float mn = sp.beta1 * mv[k] + (1.0f - sp.beta1) * r;
                         const float vn = sp.beta2 * vv[k] + (1.0f - sp.beta2) * r * r;
-                        Mp[(int64_t)k * n] = mn; Vp[(int64_t)k * n] = vn;
+                        state_store(Mbase, at + (int64_t)k * n, mn, sb); state_store(Vbase, at + (int64_t)k * n, vn, sb);
                         const float rt = __fdividef(mn * sp.inv_bc1, fast_sqrt(vn * sp.inv_bc2) + sp.eps);
                         num = fmaf(rt, rt, num);
                         den = fmaf(r, r, den);

@@ -25,7 +25,7 @@ def _f32(x) -> float:
     return float(np.float32(x))
 
 
-def oracle_of(wl: WL.Workload, mats=None, bias_correction=False):
+def oracle_of(wl: WL.Workload, mats=None, bias_correction=False, state_bf16=False):
     mats = range(len(wl.shapes)) if mats is None else mats
     # P has the precision of the projection's operands: bfloat16 for bf16 gradients at rank > 1
     # (tensor-core operands), fp32 for fp32 gradients and for the rank-1 matrix-vector pass.
@@ -35,7 +35,8 @@ def oracle_of(wl: WL.Workload, mats=None, bias_correction=False):
                                    dtype=oracle.DT_BF16 if wl.dtype == "bf16" else oracle.DT_F32,
                                    seed=wl.seed, matrix_id=i, T=wl.T, alpha=_f32(wl.alpha), gamma=_f32(wl.gamma),
                                    beta1=_f32(wl.beta1), beta2=_f32(wl.beta2), eps=_f32(wl.eps),
-                                   bias_correction=bias_correction, p_round_bf16=p_bf16) for i in mats}
+                                   bias_correction=bias_correction, p_round_bf16=p_bf16, state_bf16=state_bf16)
+            for i in mats}
 
 
 def run_parity(wl: WL.Workload, steps=None, flags=0, bias_correction=False, check_mats=None, expect_path=None,
@@ -56,7 +57,7 @@ def run_parity(wl: WL.Workload, steps=None, flags=0, bias_correction=False, chec
     deltas = [torch.zeros(wl.shapes[i], dtype=torch.float32, device=dev) if i in check_mats else None
               for i in range(n)]
     opt.set_delta_out(deltas)
-    orc = oracle_of(wl, check_mats, bias_correction)
+    orc = oracle_of(wl, check_mats, bias_correction, state_bf16=bool(flags & B.FLAG_BF16_STATES))
     Wo = {i: Wg[i].float().cpu().numpy() for i in check_mats}
     worst = {"dw": 0.0, "s": 0.0}
     for t in range(steps):

@@ -251,3 +251,29 @@ def test_caller_supplied_projection_from_an_svd(rank, dtype, flags, path):
             W[i].copy_(torch.from_numpy(res.W).to(W[i].dtype))
     opt.set_projection(0, None)                             # back to the generator
     opt.close()
+
+
+@pytest.mark.parametrize("rank,mode,flags,shapes", [
+    (64, "channel", B.FLAG_BF16_STATES, [(200, 1000), (1000, 200), (520, 264)]),
+    (256, "channel", B.FLAG_BF16_STATES, [(512, 1376), (1376, 512)]),
+    (5, "channel", B.FLAG_BF16_STATES | B.FLAG_NO_TENSOR_CORES, [(33, 130), (130, 33)]),
+    (1, "tensor", B.FLAG_BF16_STATES, [(600, 2600), (3000, 2100)]),
+])
+def test_bf16_moment_storage(rank, mode, flags, shapes):
+    wl = _wl(shapes, rank, mode=mode, dtype="bf16", steps=5, T=2, wd=0.01,
+             alpha=math.sqrt(128.0) if mode == "tensor" else 1.0)
+    run_parity(wl, flags=flags)
+    # the workspace shrinks by two bytes per moment entry
+    full = B.workspace_bytes(shapes, B.config_for(wl, flags & ~B.FLAG_BF16_STATES))
+    half = B.workspace_bytes(shapes, B.config_for(wl, flags))
+    moments = sum(2 * rank * max(s) for s in shapes)
+    assert full - half >= 2 * moments - 4096 * len(shapes)
+    # state read-back is widened to float and holds bfloat16 values
+    opt = B.Apollo(shapes, B.config_for(wl, flags))
+    W = [WL.make_weight(wl, i).cuda() for i in range(len(shapes))]
+    opt.step(W, [WL.make_grad(wl, i, 0).cuda() for i in range(len(shapes))], 1e-2)
+    M, V = opt.state(0)
+    assert torch.equal(M, M.to(torch.bfloat16).float()) and torch.equal(V, V.to(torch.bfloat16).float())
+    blob = opt.state_export()
+    assert blob.numel() == sum(2 * 2 * rank * max(s) + 4 for s in shapes)
+    opt.close()
