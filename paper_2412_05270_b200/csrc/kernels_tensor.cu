@@ -36,7 +36,8 @@ constexpr int TC_EPI_THREADS = 384;       // warps 2-13
 constexpr int TC_BLOCK_BYTES = 128 * TC_BK * 2;   // one 128-channel block of a G stage: 16 KiB
 constexpr int TC_MISC_BYTES = 256 + 3 * 512 * 8 + 8 * 512 * 4 + 1024;   // barriers, red, g2s, alignment slack
 constexpr int TC_MAX_SMEM = 227 * 1024;
-constexpr int TC_PREFETCH = 6;             // k-blocks of G requested into L2 ahead of their load
+constexpr int TC_PREFETCH = 2;             // k-blocks of G asked into L2 ahead of the load that needs them
+constexpr uint32_t TC_PACE_CAP = 1u << 12; // polls (100 ns apart) of the prefetchers' pacing wait; expiry is harmless
 constexpr uint32_t TC_WAIT_CAP = 1u << 20;   // polls before a wait gives up (normal waits are far below 1 ms)
 
 TcTiling choose_tiling(int rank)
@@ -183,13 +184,24 @@ namespace {
 
 // Bounded wait on an mbarrier phase.  On expiry the CTA-wide abort flag and the global
 // status word are set; later waits return at once, so the kernel always terminates.
-__device__ __forceinline__ void wait_phase(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status)
+// Bounded wait on an mbarrier phase.  false = this wait, or an earlier one of this CTA, gave up: the
+// caller stops issuing work and falls through to the barriers and the drain at the end of the kernel.
+__device__ __forceinline__ bool wait_phase(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status)
 {
-    if (*abort_flag) return;
+    if (*abort_flag) return false;
     for (uint32_t i = 0; i < TC_WAIT_CAP; ++i)
-        if (ptx::mbar_try_wait(bar, parity)) return;
+        if (ptx::mbar_try_wait(bar, parity)) return true;
     *abort_flag = 1;
     atomicExch(status, STATUS_TIMEOUT);
+    return false;
+}
+
+// Bounded wait that neither reads nor sets the abort flag: lets copies and MMAs that are already in
+// flight finish before the CTA gives up its shared memory and TMEM.
+__device__ __forceinline__ void drain_phase(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t i = 0; i < TC_WAIT_CAP; ++i)
+        if (ptx::mbar_try_wait(bar, parity)) return;
 }
 
 __device__ __forceinline__ float sum_sq_bf16x8(const uint4& v)
@@ -240,6 +252,8 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
     const uint32_t bar_g_full = bars, bar_p_full = bars + 32, bar_empty = bars + 64, bar_acc = bars + 96;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + stages * stage_bytes + 104);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + stages * stage_bytes + 108);
+    const uint32_t bar_drain = bars + 112;
+    volatile uint32_t* issued = reinterpret_cast<volatile uint32_t*>(smem_gen + stages * stage_bytes + 120);   // k-blocks the producer has requested
     float2* red = reinterpret_cast<float2*>(smem_gen + stages * stage_bytes + 256);          // [3][nblk*128]
     float* g2s = reinterpret_cast<float*>(smem_gen + stages * stage_bytes + 256 + 3 * 512 * 8);   // [8][nblk*128]
 
@@ -253,7 +267,9 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
             ptx::mbar_init(bar_empty + 8 * s, 1 + TC_NORM_THREADS / 32);
         }
         ptx::mbar_init(bar_acc, 1);
+        ptx::mbar_init(bar_drain, 1);
         *abort_flag = 0;
+        *issued = 0;
         ptx::fence_mbar_init();
     }
     if (warp == 1) {
@@ -294,20 +310,9 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
             if (lane == 0) {
                 ptx::fence_tensormap_acquire(tmap);
                 if (staged) ptx::fence_tensormap_acquire(tmap_p);
-                // G tiles are pulled into L2 TC_PREFETCH k-blocks ahead of the load that needs them, so the
-                // load into shared memory sees L2 latency and a shallow ring suffices
-                auto prefetch = [&](int kb) {
-                    if (tall) {
-                        for (int b = 0; b < nblk; ++b) ptx::tma_prefetch_2d(tmap, kb * TC_BK, j0 + b * 128);
-                    } else {
-                        for (int b = 0; b < 2 * nblk; ++b) ptx::tma_prefetch_2d(tmap, j0 + b * 64, kb * TC_BK);
-                    }
-                };
-                for (int kb = 0; kb < TC_PREFETCH && kb < num_kb; ++kb) prefetch(kb);
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                    if (kb + TC_PREFETCH < num_kb) prefetch(kb + TC_PREFETCH);
                     const uint32_t s = it % stages, ph = (it / stages) & 1;
-                    wait_phase(bar_empty + 8 * s, ph ^ 1, abort_flag, status);
+                    if (!wait_phase(bar_empty + 8 * s, ph ^ 1, abort_flag, status)) break;
                     const uint32_t g_s = smem_base + s * stage_bytes;
                     ptx::mbar_arrive_expect_tx(bar_g_full + 8 * s,
                                                (uint32_t)(nblk * TC_BLOCK_BYTES + (staged ? r_slice * 128 : 0)));
@@ -319,19 +324,19 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                         for (int b = 0; b < 2 * nblk; ++b)
                             ptx::tma_load_2d(g_s + b * (TC_BLOCK_BYTES / 2), tmap, j0 + b * 64, kb * TC_BK, bar_g_full + 8 * s);
                     }
+                    *issued = it + 1;
                 }
-            } else {
-                it += num_kb;
             }
-            it = __shfl_sync(0xFFFFFFFFu, it, 0);
+            it = __shfl_sync(0xFFFFFFFFu, it, 0);     // after a wait gave up: the k-blocks requested so far
         } else if (warp == 1) {
             // ---------------- MMA issuer ----------------
             if (lane == 0) {
                 const uint32_t idesc = ptx::instr_desc_bf16((uint32_t)r_slice, !tall);
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                int kb = 0;
+                for (; kb < num_kb; ++kb, ++it) {
                     const uint32_t s = it % stages, ph = (it / stages) & 1;
-                    wait_phase(bar_g_full + 8 * s, ph, abort_flag, status);
-                    if (!staged) wait_phase(bar_p_full + 8 * s, ph, abort_flag, status);
+                    if (!wait_phase(bar_g_full + 8 * s, ph, abort_flag, status)) break;
+                    if (!staged && !wait_phase(bar_p_full + 8 * s, ph, abort_flag, status)) break;
                     ptx::tc_fence_after_sync();
                     const uint32_t g_s = smem_base + s * stage_bytes, p_s = g_s + p_off;
                     for (int b = 0; b < nblk; ++b) {
@@ -347,18 +352,61 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                     }
                     ptx::mma_commit(bar_empty + 8 * s);
                 }
-                ptx::mma_commit(bar_acc);
-            } else {
-                it += num_kb;
+                if (kb == num_kb) ptx::mma_commit(bar_acc);
             }
             it = __shfl_sync(0xFFFFFFFFu, it, 0);
         } else if (warp < 10) {
             // ---------------- generators: P tile for every k-block ----------------
             const int g = tid - 64;
-            if (staged) it += num_kb;     // P arrives by TMA from the staging buffer
+            if (staged) {
+                // P arrives by TMA from the staging buffer.  These warps instead ask L2 for the lines of G
+                // TC_PREFETCH k-blocks ahead of the producer (into the next tile at the end of this one), so
+                // that the loads into the shared-memory ring find them there.
+                struct Ahead { const char* base; size_t pitch; int m, n, j0, nkb; bool tall; };
+                auto ask = [&](const Ahead& a, int kb) {
+                    for (int id = g; id < chan_tile; id += TC_GEN_THREADS) {
+                        if (a.tall) {
+                            if (a.j0 + id < a.n)
+                                ptx::prefetch_l2(a.base + (size_t)(a.j0 + id) * a.pitch + (size_t)kb * (TC_BK * 2));
+                        } else {
+                            const int lines = chan_tile / 64;
+                            const int row = kb * TC_BK + id / lines, col = a.j0 + (id % lines) * 64;
+                            if (row < a.m && col < a.n)
+                                ptx::prefetch_l2(a.base + (size_t)row * a.pitch + (size_t)col * 2);
+                        }
+                    }
+                };
+                const Ahead cur = { static_cast<const char*>(dp->gpad ? dp->gpad : dp->G),
+                                    (size_t)__ldg(&dp->g_pitch) * 2, m, n, j0, num_kb, tall };
+                Ahead nxt = cur;
+                nxt.nkb = 0;
+                const int next_tile = tile + (int)gridDim.x;
+                if (tile_iter == 0)
+                    for (int kb = 0; kb < TC_PREFETCH && kb < num_kb; ++kb) ask(cur, kb);
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int want = kb + TC_PREFETCH;
+                    if (want < num_kb) {
+                        ask(cur, want);
+                    } else if (next_tile < tile_end) {
+                        if (want == num_kb || (kb == 0 && want > num_kb)) {
+                            const int nm = find_matrix(prefix, n_mat, next_tile);
+                            const MatDesc* q = descs + nm;
+                            nxt.base = static_cast<const char*>(q->gpad ? q->gpad : q->G);
+                            nxt.pitch = (size_t)__ldg(&q->g_pitch) * 2;
+                            nxt.m = __ldg(&q->m); nxt.n = __ldg(&q->n); nxt.tall = __ldg(&q->tall) != 0;
+                            nxt.j0 = ((next_tile - __ldg(prefix + nm)) / __ldg(&q->tiles_k)) * chan_tile;
+                            nxt.nkb = (nxt.m + TC_BK - 1) / TC_BK;
+                        }
+                        if (want - num_kb < nxt.nkb) ask(nxt, want - num_kb);
+                    }
+                    // pacing only: nothing waits for these warps, so an expired wait costs nothing
+                    for (uint32_t i = 0; i < TC_PACE_CAP && (int32_t)(*issued - it) <= 0 && !*abort_flag; ++i)
+                        __nanosleep(100);
+                }
+            }
             for (int kb = 0; kb < num_kb && !staged; ++kb, ++it) {
                 const uint32_t s = it % stages, ph = (it / stages) & 1;
-                wait_phase(bar_empty + 8 * s, ph ^ 1, abort_flag, status);
+                if (!wait_phase(bar_empty + 8 * s, ph ^ 1, abort_flag, status)) break;
                 const uint32_t p_s = smem_base + s * stage_bytes + p_off;
                 // two rows per pass (32 rows apart) so that four Philox chains are in flight per thread
                 const int total = r_slice * 8;
@@ -396,7 +444,7 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
             const int rows_pp = TC_BK / parts;
             for (int kb = 0; kb < num_kb; ++kb, ++it) {
                 const uint32_t s = it % stages, ph = (it / stages) & 1;
-                wait_phase(bar_g_full + 8 * s, ph, abort_flag, status);
+                if (!wait_phase(bar_g_full + 8 * s, ph, abort_flag, status)) break;
                 const uint32_t g_s = smem_base + s * stage_bytes;
                 if (tall) {
                     // block b, row t: 128 bytes = 8 chunks; the order of the chunks does not matter
@@ -439,9 +487,9 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
             const int q = warp & 3, widx = (warp - 2) >> 2;
             const int ch_in_blk = q * 32 + lane;
             for (int b = 0; b < nblk; ++b) red[widx * chan_tile + b * 128 + ch_in_blk] = make_float2(0.f, 0.f);
-            wait_phase(bar_acc, tile_iter & 1, abort_flag, status);
+            const bool acc_ok = wait_phase(bar_acc, tile_iter & 1, abort_flag, status);
             ptx::tc_fence_after_sync();
-            const int chunks = r_slice / 16, items = nblk * chunks;
+            const int chunks = r_slice / 16, items = acc_ok ? nblk * chunks : 0;
             float num = 0.f, den = 0.f;
             int cur_b = -1;
             for (int item = widx; item < items; item += 3) {
@@ -491,14 +539,30 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                 }
             }
         }
-        // the accumulator is drained: the issuer may start the next tile
+        // the accumulator is drained: the issuer may start the next tile.  After a wait gave up, all
+        // warps of the barrier leave together; the producer leaves on its own
         if (warp >= 1) {
             ptx::tc_fence_before_sync();
-            ptx::named_barrier(2, TC_THREADS - 32);
+            const bool stop = ptx::named_barrier_or(2, TC_THREADS - 32, *abort_flag != 0);
             ptx::tc_fence_after_sync();
+            if (stop) break;
+        } else if (__shfl_sync(0xFFFFFFFFu, *abort_flag, 0) != 0) {
+            break;
         }
     }
 
+    // Whatever is still in flight lands before shared memory and TMEM are given up.  On the normal
+    // path every load was consumed and every MMA committed, so these waits return at once.
+    if (tid == 0) {
+        for (uint32_t s = 0; s < (uint32_t)stages && s < it; ++s) {
+            const uint32_t last = s + (it - 1 - s) / stages * stages;    // last k-block requested into stage s
+            drain_phase(bar_g_full + 8 * s, (last / stages) & 1);
+        }
+    }
+    if (tid == 32) {
+        ptx::mma_commit(bar_drain);
+        drain_phase(bar_drain, 0);
+    }
     ptx::tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) ptx::tmem_dealloc(tmem_base, 512);

@@ -84,13 +84,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* tmap, int3
         : "memory");
 }
 
-// Prefetch of the same box into L2 only (no shared memory, no completion to wait for).
-__device__ __forceinline__ void tma_prefetch_2d(const void* tmap, int32_t x, int32_t y)
-{
-    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(tmap), "r"(x), "r"(y)
-                 : "memory");
-}
-
 // ---- tensor memory ------------------------------------------------------------------------
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols)   // whole warp
 {
@@ -200,6 +193,22 @@ __device__ __forceinline__ void mma_commit_pair(uint32_t bar, uint16_t cta_mask)
 __device__ __forceinline__ void named_barrier(uint32_t id, uint32_t threads)
 {
     asm volatile("barrier.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+// Named barrier that also ORs a predicate over its participants: every one of them gets the same answer.
+__device__ __forceinline__ bool named_barrier_or(uint32_t id, uint32_t threads, bool pred)
+{
+    uint32_t out;
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %3, 0;\n\tbarrier.red.or.pred p, %1, %2, q;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(out) : "r"(id), "r"(threads), "r"((uint32_t)pred) : "memory");
+    return out != 0;
+}
+
+// Asks L2 for the 128-byte line that holds p; nothing waits for it.
+__device__ __forceinline__ void prefetch_l2(const void* p)
+{
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
 }
 
 // ---- descriptors ----------------------------------------------------------------------------
