@@ -189,6 +189,7 @@ struct apollo_ctx {
     bool first;
     bool imported;   // the moments came from apollo_state_import: the first step must not zero them
     bool descs_dirty;
+    std::vector<int64_t> staged_epoch;   // per matrix: the epoch whose P its staging slot holds, -1 = none
     int64_t t;
     int device;
     int sm_count;
@@ -293,6 +294,7 @@ int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_ma
     ctx->delta_on = false;
     ctx->first = true;
     ctx->imported = false;
+    ctx->staged_epoch.assign((size_t)ctx->n_mat, -1);
     ctx->descs_dirty = true;
     ctx->t = 0;
     ctx->last_launches = 0;
@@ -426,8 +428,23 @@ static int step_range(apollo_ctx* ctx, int first, int count, void* const* d_W, c
             const int me = g.mat_end < last ? g.mat_end : last;
             if (me <= mb || !tiles_of(PATH_TENSOR, mb, me, tb, te)) continue;
             if (tensor_path_staged()) {
-                launch_generate_p(ctx->d_descs, mb, me, sp, stream);
-                ++launches;
+                // P changes only with the epoch (every T steps).  When every matrix owns its staging slot
+                // (one group), a slot filled in this epoch is read again instead of being regenerated.
+                // A projection supplied by the caller is converted every step: its buffer may have been rewritten.
+                int lo = mb, hi = me;
+                if (plan.groups.size() == 1) {
+                    auto fresh = [&](int i) {
+                        const MatDesc& d = ctx->h_descs[i];
+                        return d.path != PATH_TENSOR || (!d.ext_p && ctx->staged_epoch[i] == (int64_t)sp.epoch);
+                    };
+                    while (lo < hi && fresh(lo)) ++lo;
+                    while (hi > lo && fresh(hi - 1)) --hi;
+                    for (int i = lo; i < hi; ++i) ctx->staged_epoch[i] = (int64_t)sp.epoch;
+                }
+                if (hi > lo) {
+                    launch_generate_p(ctx->d_descs, lo, hi, sp, stream);
+                    ++launches;
+                }
             }
             launch_project_tensor(ctx->d_descs, ctx->d_prefix[PATH_TENSOR], ctx->n_mat, tb, te, sp, ctx->sm_count,
                                   ctx->d_status, stream);
@@ -558,6 +575,7 @@ int apollo_state_import(apollo_ctx* ctx, const void* d_in, int64_t step_count, v
     if (rc != APOLLO_OK) return rc;
     ctx->t = step_count;
     ctx->imported = true;
+    ctx->staged_epoch.assign((size_t)ctx->n_mat, -1);
     return APOLLO_OK;
 }
 
@@ -568,6 +586,7 @@ int apollo_set_projection(apollo_ctx* ctx, int32_t matrix, const float* d_P)
     MatDesc& d = ctx->h_descs[matrix];
     if (d_P && d.path == PATH_TENSOR && !tensor_path_staged()) return APOLLO_ERR_UNSUPPORTED;
     d.ext_p = d_P;
+    ctx->staged_epoch[matrix] = -1;
     d.r_scale = d_P ? 1.0f : (float)(1.0 / std::sqrt((double)ctx->cfg.rank));
     ctx->descs_dirty = true;
     return APOLLO_OK;
