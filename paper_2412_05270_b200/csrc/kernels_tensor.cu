@@ -310,19 +310,21 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
             if (lane == 0) {
                 ptx::fence_tensormap_acquire(tmap);
                 if (staged) ptx::fence_tensormap_acquire(tmap_p);
+                // G is read once in this pass, every CTA of a matrix reads the same P: tell L2 which to keep
+                const uint64_t pol_g = ptx::policy_evict_first(), pol_p = ptx::policy_evict_last();
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
                     const uint32_t s = it % stages, ph = (it / stages) & 1;
                     if (!wait_phase(bar_empty + 8 * s, ph ^ 1, abort_flag, status)) break;
                     const uint32_t g_s = smem_base + s * stage_bytes;
                     ptx::mbar_arrive_expect_tx(bar_g_full + 8 * s,
                                                (uint32_t)(nblk * TC_BLOCK_BYTES + (staged ? r_slice * 128 : 0)));
-                    if (staged) ptx::tma_load_2d(g_s + p_off, tmap_p, kb * TC_BK, r0, bar_g_full + 8 * s);
+                    if (staged) ptx::tma_load_2d_hint(g_s + p_off, tmap_p, kb * TC_BK, r0, bar_g_full + 8 * s, pol_p);
                     if (tall) {
                         for (int b = 0; b < nblk; ++b)
-                            ptx::tma_load_2d(g_s + b * TC_BLOCK_BYTES, tmap, kb * TC_BK, j0 + b * 128, bar_g_full + 8 * s);
+                            ptx::tma_load_2d_hint(g_s + b * TC_BLOCK_BYTES, tmap, kb * TC_BK, j0 + b * 128, bar_g_full + 8 * s, pol_g);
                     } else {
                         for (int b = 0; b < 2 * nblk; ++b)
-                            ptx::tma_load_2d(g_s + b * (TC_BLOCK_BYTES / 2), tmap, j0 + b * 64, kb * TC_BK, bar_g_full + 8 * s);
+                            ptx::tma_load_2d_hint(g_s + b * (TC_BLOCK_BYTES / 2), tmap, j0 + b * 64, kb * TC_BK, bar_g_full + 8 * s, pol_g);
                     }
                     *issued = it + 1;
                 }
