@@ -78,8 +78,7 @@ struct TcTiling {
     int32_t nblk;      // 128-channel blocks per tile (1, 2 or 4); nblk * r_slice <= 512 TMEM columns
     int32_t stages;    // shared-memory pipeline depth
     int32_t smem_bytes;
-    int32_t staged;    // 0: P generated in shared memory; 1: P staged in L2 (ring kernel); 2: staged, double-buffered kernels
-    int32_t pair;      // 1: staged kernel on CTA pairs (cta_group::2), pair tile of 256 channels
+    int32_t staged;    // 0: P generated in shared memory; 1: P loaded from the staging buffer
 };
 
 // Device status word values.

@@ -1,17 +1,23 @@
 // Tensor-core projection: R = P G on tcgen05 with TMEM accumulators (Algorithm 1, step 1),
-// with P generated straight into shared memory (never stored) and the moment update and
-// per-channel norm sums fused into the epilogue (Algorithm 1, step 2; Eq. 5).
+// with the moment update and the per-channel norm sums fused into the epilogue (Algorithm 1,
+// step 2; Eq. 5).  P is either loaded from a staging buffer that generate_p_kernel fills once
+// per epoch (default) or generated straight into shared memory by every CTA.
 //
-// Roles of the 14 warps of a CTA (one CTA per SM, persistent over tiles):
-//   warp 0      TMA producer: G tiles (128-byte swizzle) into a shared-memory ring
+// Roles of the 14 warps of a CTA (one CTA per SM, persistent over tiles of 256 channels):
+//   warp 0      TMA producer: G tiles (and staged P tiles) into a shared-memory ring, 128-byte swizzle
 //   warp 1      MMA issuer (one thread) and owner of the 512 TMEM columns
-//   warps 2-9   generators: Philox -> Box-Muller -> bf16 P tile in the UMMA K-major layout
+//   warps 2-9   staged P: L2 prefetch of the G lines the producer will ask for next;
+//               otherwise generators: Philox -> Box-Muller -> bf16 P tile in the UMMA K-major layout
 //   warps 10-13 column norms of G from the landed tiles
 //   warps 2-13  epilogue: tcgen05.ld of R, read-modify-write of M and V, partial sums
 //
 // Operand roles: D[128 channels x r_slice] = A[128 channels x 64] * B[r_slice x 64]^T, so
 // a TMEM lane is a channel and the reductions over r are per thread.  A = G tile: K-major
 // for a tall matrix (channels are stored rows), MN-major for a wide one.  B = P tile.
+//
+// Every wait on an mbarrier is bounded.  When one gives up, the CTA sets the status word, stops
+// issuing loads and MMAs, leaves the tile loop through a barrier vote, waits (bounded again) for
+// the loads and MMAs already in flight, frees its TMEM and returns.
 #include "kernels.h"
 
 #include <cuda.h>
@@ -55,22 +61,6 @@ TcTiling choose_tiling(int rank)
         if ((v == 1 || v == 2 || v == 4) && v * t.r_slice <= 512) t.nblk = v;
     }
     t.staged = tensor_path_staged() ? 1 : 0;
-    t.pair = 0;
-    // Staged P has three kernels (APOLLO_TC_KERNEL): "ring" (default, fastest measured): 256 channels
-    // per CTA on one ring of G+P stages; "overlap": 128 channels per CTA, double-buffered accumulator,
-    // epilogue under the next main loop; "pair": the same on CTA pairs sharing each MMA (cta_group::2).
-    const char* kernel = std::getenv("APOLLO_TC_KERNEL");
-    const bool overlap = kernel && (std::strcmp(kernel, "overlap") == 0 || std::strcmp(kernel, "pair") == 0);
-    if (t.staged && overlap) {
-        t.pair = std::strcmp(kernel, "pair") == 0 ? 1 : 0;
-        t.staged = 2;                 // 2: one of the double-buffered kernels
-        t.nblk = t.pair ? 2 : 1;
-        const int p_ring = t.pair ? 6 * (t.r_slice / 2) * 128 : 2 * t.r_slice * 128;   // pair: T2P_P_STAGES half tiles
-        t.stages = (TC_MAX_SMEM - 13824 - p_ring) / (128 * TC_BK * 2);
-        if (t.stages > 12) t.stages = 12;
-        t.smem_bytes = t.stages * (128 * TC_BK * 2) + p_ring + 13824;
-        return t;
-    }
     const int stage = t.nblk * TC_BLOCK_BYTES + t.r_slice * 128;
     t.stages = (TC_MAX_SMEM - TC_MISC_BYTES) / stage;
     if (t.stages > 4) t.stages = 4;
@@ -166,7 +156,7 @@ int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, void* d_tmaps, cu
             // staged P: rank rows of m_pad bf16, loaded as 64 x r_slice boxes (K-major UMMA tiles)
             const cuuint64_t pdims[2] = { (cuuint64_t)d.m_pad, (cuuint64_t)rank };
             const cuuint64_t pstrides[1] = { (cuuint64_t)d.m_pad * 2 };
-            const cuuint32_t pbox[2] = { 64u, (cuuint32_t)(tl.pair ? tl.r_slice / 2 : tl.r_slice) };
+            const cuuint32_t pbox[2] = { 64u, (cuuint32_t)tl.r_slice };
             const CUresult rp = encode(&maps[2 * i + 1], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, d.pstage, pdims, pstrides,
                                        pbox, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -570,507 +560,6 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
     if (warp == 1) ptx::tmem_dealloc(tmem_base, 512);
 }
 
-// ----------------------------------------------------------------------------------------
-// Staged-P kernel.  Tile = 128 channels x r_slice rows of R.  The accumulator is double
-// buffered in TMEM (2 x r_slice <= 512 columns) so the epilogue of one tile runs under the
-// main loop of the next; G and P have separate shared-memory rings, a deep one for G (it
-// comes from HBM) and a two-slot one for P (it comes from L2).
-//   warp 0      G producer (TMA)            warp 1   MMA issuer, owner of TMEM
-//   warp 2      P producer (TMA)            warp 3   spare
-//   warps 4-7   squared column norms of G   warps 8-15  epilogue (moments, partial sums)
-// ----------------------------------------------------------------------------------------
-constexpr int T2_THREADS = 512;
-constexpr int T2_G_BYTES = 128 * TC_BK * 2;        // one G stage: 16 KiB
-constexpr int T2_MAX_G_STAGES = 12;
-constexpr int T2_MISC_BYTES = 512 + 2 * 2 * 128 * 8 + 2 * 8 * 128 * 4 + 1024;   // barriers, red, g2s, slack
-static_assert(T2_MISC_BYTES == 13824, "choose_tiling() reserves this many bytes");
-
-__global__ void __launch_bounds__(T2_THREADS, 1)
-project_staged_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix, int n_mat, int tile_begin,
-                      int tile_end, StepParams sp, TcTiling tl, int32_t* __restrict__ status)
-{
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
-    uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_addr(smem_raw));
-
-    const int r_slice = tl.r_slice, ng = tl.stages;
-    const uint32_t p_bytes = (uint32_t)r_slice * 128u;
-    const uint32_t g_ring = smem_base, p_ring = smem_base + (uint32_t)ng * T2_G_BYTES;
-    const uint32_t misc = (uint32_t)ng * T2_G_BYTES + 2u * p_bytes;
-    const uint32_t bars = smem_base + misc;
-    const uint32_t bar_g_full = bars, bar_g_empty = bars + 96, bar_p_full = bars + 192, bar_p_empty = bars + 208,
-                   bar_acc_full = bars + 224, bar_acc_empty = bars + 240;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + misc + 256);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + misc + 260);
-    float2* red = reinterpret_cast<float2*>(smem_gen + misc + 512);                 // [2 tiles][2 halves][128]
-    float* g2s = reinterpret_cast<float*>(smem_gen + misc + 512 + 2 * 2 * 128 * 8);   // [2 tiles][8 parts][128]
-
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-
-    if (tid == 0) {
-        for (int s = 0; s < ng; ++s) {
-            ptx::mbar_init(bar_g_full + 8 * s, 1);
-            ptx::mbar_init(bar_g_empty + 8 * s, 1 + 4);     // MMA commit + four norm warps
-        }
-        for (int s = 0; s < 2; ++s) {
-            ptx::mbar_init(bar_p_full + 8 * s, 1);
-            ptx::mbar_init(bar_p_empty + 8 * s, 1);         // MMA commit
-            ptx::mbar_init(bar_acc_full + 8 * s, 1);        // MMA commit
-            ptx::mbar_init(bar_acc_empty + 8 * s, 8);       // eight epilogue warps
-        }
-        *abort_flag = 0;
-        ptx::fence_mbar_init();
-    }
-    if (warp == 1) {
-        ptx::tmem_alloc(ptx::smem_addr(tmem_slot), 512);
-        ptx::tmem_relinquish();
-    }
-    ptx::tc_fence_before_sync();
-    __syncthreads();
-    ptx::tc_fence_after_sync();
-    const uint32_t tmem_base = *tmem_slot;
-
-    uint32_t git = 0, pit = 0, tile_iter = 0;   // G-ring, P-ring and tile counters of this role
-
-    for (int tile = tile_begin + blockIdx.x; tile < tile_end; tile += gridDim.x, ++tile_iter) {
-        const int mat = find_matrix(prefix, n_mat, tile);
-        const MatDesc* dp = descs + mat;
-        const int tiles_k = __ldg(&dp->tiles_k);
-        const int m = __ldg(&dp->m), n = __ldg(&dp->n);
-        const bool tall = __ldg(&dp->tall) != 0;
-        const int local = tile - __ldg(prefix + mat);
-        const int tr = local % tiles_k, tn = local / tiles_k;
-        const int j0 = tn * 128, r0 = tr * r_slice;
-        const int num_kb = (m + TC_BK - 1) / TC_BK;
-        const uint32_t buf = tile_iter & 1, use = tile_iter >> 1;
-
-        if (warp == 0) {
-            if (lane == 0) {
-                const void* tmap = dp->tmap;
-                ptx::fence_tensormap_acquire(tmap);
-                for (int kb = 0; kb < num_kb; ++kb, ++git) {
-                    const uint32_t s = git % ng, ph = (git / ng) & 1;
-                    wait_phase(bar_g_empty + 8 * s, ph ^ 1, abort_flag, status);
-                    const uint32_t g_s = g_ring + s * T2_G_BYTES;
-                    ptx::mbar_arrive_expect_tx(bar_g_full + 8 * s, (uint32_t)T2_G_BYTES);
-                    if (tall) {
-                        ptx::tma_load_2d(g_s, tmap, kb * TC_BK, j0, bar_g_full + 8 * s);
-                    } else {
-                        ptx::tma_load_2d(g_s, tmap, j0, kb * TC_BK, bar_g_full + 8 * s);
-                        ptx::tma_load_2d(g_s + T2_G_BYTES / 2, tmap, j0 + 64, kb * TC_BK, bar_g_full + 8 * s);
-                    }
-                }
-            }
-            __syncwarp();
-        } else if (warp == 2) {
-            if (lane == 0) {
-                const void* tmap_p = dp->tmap_p;
-                ptx::fence_tensormap_acquire(tmap_p);
-                for (int kb = 0; kb < num_kb; ++kb, ++pit) {
-                    const uint32_t s = pit & 1, ph = (pit >> 1) & 1;
-                    wait_phase(bar_p_empty + 8 * s, ph ^ 1, abort_flag, status);
-                    ptx::mbar_arrive_expect_tx(bar_p_full + 8 * s, p_bytes);
-                    ptx::tma_load_2d(p_ring + s * p_bytes, tmap_p, kb * TC_BK, r0, bar_p_full + 8 * s);
-                }
-            }
-            __syncwarp();
-        } else if (warp == 1) {
-            if (lane == 0) {
-                const uint32_t idesc = ptx::instr_desc_bf16((uint32_t)r_slice, !tall);
-                const uint32_t d_tmem = tmem_base + buf * (uint32_t)r_slice;
-                wait_phase(bar_acc_empty + 8 * buf, (use & 1) ^ 1, abort_flag, status);   // epilogue of the tile before last
-                ptx::tc_fence_after_sync();
-                for (int kb = 0; kb < num_kb; ++kb, ++git, ++pit) {
-                    const uint32_t gs = git % ng, gph = (git / ng) & 1, ps = pit & 1, pph = (pit >> 1) & 1;
-                    wait_phase(bar_g_full + 8 * gs, gph, abort_flag, status);
-                    wait_phase(bar_p_full + 8 * ps, pph, abort_flag, status);
-                    ptx::tc_fence_after_sync();
-                    const uint32_t g_s = g_ring + gs * T2_G_BYTES, p_s = p_ring + ps * p_bytes;
-#pragma unroll
-                    for (int kk = 0; kk < TC_BK / 16; ++kk) {
-                        const uint64_t a_desc = tall ? ptx::smem_desc_sw128(g_s + kk * 32, 16, 1024)
-                                                     : ptx::smem_desc_sw128(g_s + kk * 2048, T2_G_BYTES / 2, 1024);
-                        const uint64_t b_desc = ptx::smem_desc_sw128(p_s + kk * 32, 16, 1024);
-                        ptx::mma_bf16(d_tmem, a_desc, b_desc, idesc, (kb | kk) != 0 ? 1u : 0u);
-                    }
-                    ptx::mma_commit(bar_g_empty + 8 * gs);
-                    ptx::mma_commit(bar_p_empty + 8 * ps);
-                }
-                ptx::mma_commit(bar_acc_full + 8 * buf);
-            }
-            __syncwarp();
-        } else if (warp >= 4 && warp < 8) {
-            // ---------------- squared column norms of the 128 channels of this tile ----------------
-            const int t = tid - 128;
-            float acc[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-            const int cc = t & 15, part = t >> 4;     // wide: 16 chunk columns x 8 row groups
-            for (int kb = 0; kb < num_kb; ++kb, ++git) {
-                const uint32_t s = git % ng, ph = (git / ng) & 1;
-                wait_phase(bar_g_full + 8 * s, ph, abort_flag, status);
-                const uint32_t g_s = g_ring + s * T2_G_BYTES;
-                if (tall) {
-                    // units (row, half): 256 units over 128 threads; the order of the chunks is free
-#pragma unroll
-                    for (int pass = 0; pass < 2; ++pass) {
-                        const int u = t + pass * 128, row = u >> 1, half = u & 1;
-                        const uint32_t base = g_s + row * 128 + half * 64;
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) acc[pass] += sum_sq_bf16x8(ld_shared_v4(base + (((i + row) & 3) << 4)));
-                    }
-                } else {
-                    const uint32_t colbase = g_s + (cc >> 3) * (T2_G_BYTES / 2);
-                    const int c = cc & 7;
-#pragma unroll
-                    for (int i8 = 0; i8 < 8; ++i8) {
-                        const int k = part + 8 * i8;
-                        const uint4 v = ld_shared_v4(colbase + k * 128 + ((c ^ (k & 7)) << 4));
-                        const uint32_t w[4] = { v.x, v.y, v.z, v.w };
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
-                            acc[2 * i] = fmaf(lo, lo, acc[2 * i]);
-                            acc[2 * i + 1] = fmaf(hi, hi, acc[2 * i + 1]);
-                        }
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(bar_g_empty + 8 * s);
-            }
-            float* mine = g2s + buf * (8 * 128);
-            if (tall) {
-#pragma unroll
-                for (int pass = 0; pass < 2; ++pass) {
-                    const int u = t + pass * 128;
-                    mine[(u & 1) * 128 + (u >> 1)] = acc[pass];
-                }
-            } else {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) mine[part * 128 + cc * 8 + e] = acc[e];
-            }
-            ptx::named_barrier(3, 128);
-            const int j = j0 + t;
-            if (tr == 0 && j < n) {
-                float g2 = 0.f;
-                const int parts = tall ? 2 : 8;
-                for (int p = 0; p < parts; ++p) g2 += mine[p * 128 + t];
-                dp->g2[j] = g2;
-            }
-        } else if (warp >= 8) {
-            // ---------------- epilogue of this tile, overlapped with the next tile's main loop ----------------
-            const int q = warp & 3, half = (warp - 8) >> 2;
-            const int ch = q * 32 + lane, j = j0 + ch;
-            float* const Mbase = dp->M;
-            float* const Vbase = dp->V;
-            const float r_scale = __ldg(&dp->r_scale);
-            wait_phase(bar_acc_full + 8 * buf, use & 1, abort_flag, status);
-            ptx::tc_fence_after_sync();
-            float num = 0.f, den = 0.f;
-            const int chunks = r_slice / 16;
-            for (int cchunk = half; cchunk < chunks; cchunk += 2) {
-                float rv[16];
-                ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + buf * (uint32_t)r_slice + (uint32_t)(cchunk * 16), rv);
-                if (j < n) {
-                    const int64_t at = (int64_t)(r0 + cchunk * 16) * n + j;
-                    const bool sb = sp.state_bf16 != 0;
-                    float mv[16], vv[16];
-#pragma unroll
-                    for (int k = 0; k < 16; ++k) {
-                        mv[k] = state_load(Mbase, at + (int64_t)k * n, sb);
-                        vv[k] = state_load(Vbase, at + (int64_t)k * n, sb);
-                    }
-#pragma unroll
-                    for (int k = 0; k < 16; ++k) {
-                        const float r = rv[k] * r_scale;
-                        const float mn = sp.beta1 * mv[k] + (1.0f - sp.beta1) * r;
-                        const float vn = sp.beta2 * vv[k] + (1.0f - sp.beta2) * r * r;
-                        state_store(Mbase, at + (int64_t)k * n, mn, sb); state_store(Vbase, at + (int64_t)k * n, vn, sb);
-                        const float rt = __fdividef(mn * sp.inv_bc1, fast_sqrt(vn * sp.inv_bc2) + sp.eps);
-                        num = fmaf(rt, rt, num);
-                        den = fmaf(r, r, den);
-                    }
-                }
-            }
-            // this warp has read its share of the accumulator: hand the buffer back to the issuer
-            ptx::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(bar_acc_empty + 8 * buf);
-            float2* mine = red + buf * (2 * 128);
-            mine[half * 128 + ch] = make_float2(num, den);
-            ptx::named_barrier(1, 256);
-            if (half == 0 && j < n) {
-                const float2 a = mine[ch], b = mine[128 + ch];
-                reinterpret_cast<float2*>(dp->part)[(int64_t)tr * n + j] = make_float2(a.x + b.x, a.y + b.y);
-            }
-        }
-    }
-
-    ptx::tc_fence_before_sync();
-    __syncthreads();
-    if (warp == 1) ptx::tmem_dealloc(tmem_base, 512);
-}
-
-// ----------------------------------------------------------------------------------------
-// Pair variant of the staged-P kernel: two CTAs of a cluster share every MMA (cta_group::2,
-// M = 256).  A pair tile is 256 channels x r_slice rows of R; each CTA loads the G tile of its
-// own 128 channels and only half of the rows of the P tile, so P costs half the shared-memory
-// fill per channel while the accumulator (r_slice columns per CTA) stays double buffered.
-// Extra plumbing: warp 3 of the peer reports landed tiles to the leader, the leader's commits
-// are multicast to both CTAs, the peer's epilogue warps release the accumulator remotely.
-// ----------------------------------------------------------------------------------------
-constexpr int T2P_P_STAGES = 6;
-constexpr int T2P_MISC_BYTES = 512 + 2 * 2 * 128 * 8 + 2 * 8 * 128 * 4 + 1024;
-
-__global__ void __launch_bounds__(T2_THREADS, 1)
-project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix, int n_mat, int tile_begin,
-                      int tile_end, StepParams sp, TcTiling tl, int32_t* __restrict__ status)
-{
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
-    uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_addr(smem_raw));
-
-    // This CTA is one half of a pair (cluster of two): it owns 128 of the pair tile's 256 channels and
-    // half of the rows of every P tile; the leader (rank 0) issues the pair's MMAs.
-    const uint32_t rank = ptx::cluster_ctarank();
-    const int r_slice = tl.r_slice, ng = tl.stages, r_half = r_slice / 2;
-    const uint32_t p_bytes = (uint32_t)r_half * 128u;
-    const uint32_t g_ring = smem_base, p_ring = smem_base + (uint32_t)ng * T2_G_BYTES;
-    const uint32_t misc = (uint32_t)ng * T2_G_BYTES + (uint32_t)T2P_P_STAGES * p_bytes;
-    const uint32_t bars = smem_base + misc;
-    const uint32_t bar_g_full = bars, bar_g_empty = bars + 96, bar_p_full = bars + 192, bar_p_empty = bars + 256,
-                   bar_acc_full = bars + 320, bar_acc_empty = bars + 336, bar_peer = bars + 352;   // bar_peer: 16 slots
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + misc + 480);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + misc + 484);
-    float2* red = reinterpret_cast<float2*>(smem_gen + misc + 512);                 // [2 tiles][2 halves][128]
-    float* g2s = reinterpret_cast<float*>(smem_gen + misc + 512 + 2 * 2 * 128 * 8);   // [2 tiles][8 parts][128]
-
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-
-    if (tid == 0) {
-        for (int s = 0; s < ng; ++s) {
-            ptx::mbar_init(bar_g_full + 8 * s, 1);
-            ptx::mbar_init(bar_g_empty + 8 * s, 1 + 4);     // the leader's commit + four norm warps of this CTA
-        }
-        for (int s = 0; s < T2P_P_STAGES; ++s) {
-            ptx::mbar_init(bar_p_full + 8 * s, 1);
-            ptx::mbar_init(bar_p_empty + 8 * s, 1);         // the leader's commit
-        }
-        for (int s = 0; s < 2; ++s) {
-            ptx::mbar_init(bar_acc_full + 8 * s, 1);        // the leader's commit
-            ptx::mbar_init(bar_acc_empty + 8 * s, 16);      // eight epilogue warps of each CTA (leader's copy is used)
-        }
-        for (int s = 0; s < 16; ++s) ptx::mbar_init(bar_peer + 8 * s, 1);   // peer's tiles of a k-block have landed
-        *abort_flag = 0;
-        ptx::fence_mbar_init();
-    }
-    if (warp == 1) {
-        ptx::tmem_alloc_pair(ptx::smem_addr(tmem_slot), 512);
-        ptx::tmem_relinquish_pair();
-    }
-    ptx::tc_fence_before_sync();
-    __syncthreads();
-    ptx::cluster_sync();          // both CTAs' barriers exist before any remote arrive or multicast commit
-    ptx::tc_fence_after_sync();
-    const uint32_t tmem_base = *tmem_slot;
-
-    uint32_t git = 0, pit = 0, tile_iter = 0;   // G-ring, P-ring and tile counters of this role
-
-    const int pair = blockIdx.x >> 1, pairs = gridDim.x >> 1;
-    for (int tile = tile_begin + pair; tile < tile_end; tile += pairs, ++tile_iter) {
-        const int mat = find_matrix(prefix, n_mat, tile);
-        const MatDesc* dp = descs + mat;
-        const int tiles_k = __ldg(&dp->tiles_k);
-        const int m = __ldg(&dp->m), n = __ldg(&dp->n);
-        const bool tall = __ldg(&dp->tall) != 0;
-        const int local = tile - __ldg(prefix + mat);
-        const int tr = local % tiles_k, tn = local / tiles_k;
-        const int j0 = tn * 256 + (int)rank * 128, r0 = tr * r_slice;
-        const int num_kb = (m + TC_BK - 1) / TC_BK;
-        const uint32_t buf = tile_iter & 1, use = tile_iter >> 1;
-
-        if (warp == 0) {
-            if (lane == 0) {
-                const void* tmap = dp->tmap;
-                ptx::fence_tensormap_acquire(tmap);
-                for (int kb = 0; kb < num_kb; ++kb, ++git) {
-                    const uint32_t s = git % ng, ph = (git / ng) & 1;
-                    wait_phase(bar_g_empty + 8 * s, ph ^ 1, abort_flag, status);
-                    const uint32_t g_s = g_ring + s * T2_G_BYTES;
-                    ptx::mbar_arrive_expect_tx(bar_g_full + 8 * s, (uint32_t)T2_G_BYTES);
-                    if (tall) {
-                        ptx::tma_load_2d(g_s, tmap, kb * TC_BK, j0, bar_g_full + 8 * s);
-                    } else {
-                        ptx::tma_load_2d(g_s, tmap, j0, kb * TC_BK, bar_g_full + 8 * s);
-                        ptx::tma_load_2d(g_s + T2_G_BYTES / 2, tmap, j0 + 64, kb * TC_BK, bar_g_full + 8 * s);
-                    }
-                }
-            }
-            __syncwarp();
-        } else if (warp == 2) {
-            if (lane == 0) {
-                const void* tmap_p = dp->tmap_p;
-                ptx::fence_tensormap_acquire(tmap_p);
-                for (int kb = 0; kb < num_kb; ++kb, ++pit) {
-                    const uint32_t s = pit % T2P_P_STAGES, ph = (pit / T2P_P_STAGES) & 1;
-                    wait_phase(bar_p_empty + 8 * s, ph ^ 1, abort_flag, status);
-                    ptx::mbar_arrive_expect_tx(bar_p_full + 8 * s, p_bytes);
-                    ptx::tma_load_2d(p_ring + s * p_bytes, tmap_p, kb * TC_BK, r0 + (int)rank * r_half, bar_p_full + 8 * s);
-                }
-            }
-            __syncwarp();
-        } else if (warp == 3) {
-            // the peer tells the leader when its tiles of a k-block have landed
-            if (lane == 0 && rank == 1) {
-                for (int kb = 0; kb < num_kb; ++kb, ++git, ++pit) {
-                    const uint32_t gs = git % ng, gph = (git / ng) & 1;
-                    const uint32_t ps = pit % T2P_P_STAGES, pph = (pit / T2P_P_STAGES) & 1;
-                    wait_phase(bar_g_full + 8 * gs, gph, abort_flag, status);
-                    wait_phase(bar_p_full + 8 * ps, pph, abort_flag, status);
-                    ptx::mbar_arrive_remote(ptx::map_to_cta(bar_peer + 8 * (git & 15), 0));
-                }
-            }
-            __syncwarp();
-        } else if (warp == 1) {
-            if (lane == 0 && rank == 0) {
-                const uint32_t idesc = ptx::instr_desc_bf16((uint32_t)r_slice, !tall, 256u);
-                const uint32_t d_tmem = tmem_base + buf * (uint32_t)r_slice;
-                wait_phase(bar_acc_empty + 8 * buf, (use & 1) ^ 1, abort_flag, status);   // epilogue of the tile before last
-                ptx::tc_fence_after_sync();
-                for (int kb = 0; kb < num_kb; ++kb, ++git, ++pit) {
-                    const uint32_t gs = git % ng, gph = (git / ng) & 1;
-                    const uint32_t ps = pit % T2P_P_STAGES, pph = (pit / T2P_P_STAGES) & 1;
-                    wait_phase(bar_g_full + 8 * gs, gph, abort_flag, status);
-                    wait_phase(bar_p_full + 8 * ps, pph, abort_flag, status);
-                    wait_phase(bar_peer + 8 * (git & 15), (git >> 4) & 1, abort_flag, status);
-                    ptx::tc_fence_after_sync();
-                    const uint32_t g_s = g_ring + gs * T2_G_BYTES, p_s = p_ring + ps * p_bytes;
-#pragma unroll
-                    for (int kk = 0; kk < TC_BK / 16; ++kk) {
-                        const uint64_t a_desc = tall ? ptx::smem_desc_sw128(g_s + kk * 32, 16, 1024)
-                                                     : ptx::smem_desc_sw128(g_s + kk * 2048, T2_G_BYTES / 2, 1024);
-                        const uint64_t b_desc = ptx::smem_desc_sw128(p_s + kk * 32, 16, 1024);
-                        ptx::mma_bf16_pair(d_tmem, a_desc, b_desc, idesc, (kb | kk) != 0 ? 1u : 0u);
-                    }
-                    ptx::mma_commit_pair(bar_g_empty + 8 * gs, 3);
-                    ptx::mma_commit_pair(bar_p_empty + 8 * ps, 3);
-                }
-                ptx::mma_commit_pair(bar_acc_full + 8 * buf, 3);
-            }
-            __syncwarp();
-        } else if (warp >= 4 && warp < 8) {
-            // ---------------- squared column norms of the 128 channels of this tile ----------------
-            const int t = tid - 128;
-            float acc[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-            const int cc = t & 15, part = t >> 4;     // wide: 16 chunk columns x 8 row groups
-            for (int kb = 0; kb < num_kb; ++kb, ++git) {
-                const uint32_t s = git % ng, ph = (git / ng) & 1;
-                wait_phase(bar_g_full + 8 * s, ph, abort_flag, status);
-                const uint32_t g_s = g_ring + s * T2_G_BYTES;
-                if (tall) {
-                    // units (row, half): 256 units over 128 threads; the order of the chunks is free
-#pragma unroll
-                    for (int pass = 0; pass < 2; ++pass) {
-                        const int u = t + pass * 128, row = u >> 1, half = u & 1;
-                        const uint32_t base = g_s + row * 128 + half * 64;
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) acc[pass] += sum_sq_bf16x8(ld_shared_v4(base + (((i + row) & 3) << 4)));
-                    }
-                } else {
-                    const uint32_t colbase = g_s + (cc >> 3) * (T2_G_BYTES / 2);
-                    const int c = cc & 7;
-#pragma unroll
-                    for (int i8 = 0; i8 < 8; ++i8) {
-                        const int k = part + 8 * i8;
-                        const uint4 v = ld_shared_v4(colbase + k * 128 + ((c ^ (k & 7)) << 4));
-                        const uint32_t w[4] = { v.x, v.y, v.z, v.w };
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
-                            acc[2 * i] = fmaf(lo, lo, acc[2 * i]);
-                            acc[2 * i + 1] = fmaf(hi, hi, acc[2 * i + 1]);
-                        }
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(bar_g_empty + 8 * s);
-            }
-            float* mine = g2s + buf * (8 * 128);
-            if (tall) {
-#pragma unroll
-                for (int pass = 0; pass < 2; ++pass) {
-                    const int u = t + pass * 128;
-                    mine[(u & 1) * 128 + (u >> 1)] = acc[pass];
-                }
-            } else {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) mine[part * 128 + cc * 8 + e] = acc[e];
-            }
-            ptx::named_barrier(3, 128);
-            const int j = j0 + t;
-            if (tr == 0 && j < n) {
-                float g2 = 0.f;
-                const int parts = tall ? 2 : 8;
-                for (int p = 0; p < parts; ++p) g2 += mine[p * 128 + t];
-                dp->g2[j] = g2;
-            }
-        } else if (warp >= 8) {
-            // ---------------- epilogue of this tile, overlapped with the next tile's main loop ----------------
-            const int q = warp & 3, half = (warp - 8) >> 2;
-            const int ch = q * 32 + lane, j = j0 + ch;
-            float* const Mbase = dp->M;
-            float* const Vbase = dp->V;
-            const float r_scale = __ldg(&dp->r_scale);
-            wait_phase(bar_acc_full + 8 * buf, use & 1, abort_flag, status);
-            ptx::tc_fence_after_sync();
-            float num = 0.f, den = 0.f;
-            const int chunks = r_slice / 16;
-            for (int cchunk = half; cchunk < chunks; cchunk += 2) {
-                float rv[16];
-                ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + buf * (uint32_t)r_slice + (uint32_t)(cchunk * 16), rv);
-                if (j < n) {
-                    const int64_t at = (int64_t)(r0 + cchunk * 16) * n + j;
-                    const bool sb = sp.state_bf16 != 0;
-                    float mv[16], vv[16];
-#pragma unroll
-                    for (int k = 0; k < 16; ++k) {
-                        mv[k] = state_load(Mbase, at + (int64_t)k * n, sb);
-                        vv[k] = state_load(Vbase, at + (int64_t)k * n, sb);
-                    }
-#pragma unroll
-                    for (int k = 0; k < 16; ++k) {
-                        const float r = rv[k] * r_scale;
-                        const float mn = sp.beta1 * mv[k] + (1.0f - sp.beta1) * r;
-                        const float vn = sp.beta2 * vv[k] + (1.0f - sp.beta2) * r * r;
-                        state_store(Mbase, at + (int64_t)k * n, mn, sb); state_store(Vbase, at + (int64_t)k * n, vn, sb);
-                        const float rt = __fdividef(mn * sp.inv_bc1, fast_sqrt(vn * sp.inv_bc2) + sp.eps);
-                        num = fmaf(rt, rt, num);
-                        den = fmaf(r, r, den);
-                    }
-                }
-            }
-            // this warp has read its share of the accumulator: hand the buffer back to the issuer
-            ptx::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive_remote(ptx::map_to_cta(bar_acc_empty + 8 * buf, 0));
-            float2* mine = red + buf * (2 * 128);
-            mine[half * 128 + ch] = make_float2(num, den);
-            ptx::named_barrier(1, 256);
-            if (half == 0 && j < n) {
-                const float2 a = mine[ch], b = mine[128 + ch];
-                reinterpret_cast<float2*>(dp->part)[(int64_t)tr * n + j] = make_float2(a.x + b.x, a.y + b.y);
-            }
-        }
-    }
-
-    ptx::tc_fence_before_sync();
-    __syncthreads();
-    ptx::cluster_sync();          // no remote arrive or MMA of the pair is still under way
-    if (warp == 1) ptx::tmem_dealloc_pair(tmem_base, 512);
-}
-
 // Standard normals of the staged P: one 16-byte store (8 bf16) per thread and pass.
 __global__ void generate_p_kernel(const MatDesc* __restrict__ descs, int mat_begin, StepParams sp)
 {
@@ -1149,45 +638,10 @@ void launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_ma
     bool& attr_set = attr_set_on[device & 63];
     if (!attr_set) {
         cudaFuncSetAttribute(project_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
-        cudaFuncSetAttribute(project_staged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
-        cudaFuncSetAttribute(project_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
         attr_set = true;
     }
-    if (tl.staged == 2 && tl.pair) {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(sm_count / 2 * 2);
-        cfg.blockDim = dim3(T2_THREADS);
-        cfg.dynamicSmemBytes = tl.smem_bytes;
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        // the tile loop is persistent: launch exactly as many pairs as can be resident at once
-        // (pairs must sit in one GPC, so this can be fewer than half the SMs)
-        static int max_pairs_on[64] = {};
-        int& max_pairs = max_pairs_on[device & 63];
-        if (max_pairs == 0) {
-            int clusters = 0;
-            if (cudaOccupancyMaxActiveClusters(&clusters, project_pair_kernel, &cfg) != cudaSuccess || clusters < 1) {
-                cudaGetLastError();
-                clusters = sm_count / 2;
-            }
-            max_pairs = clusters;
-        }
-        int pairs = max_pairs;
-        if (tiles < pairs) pairs = tiles;
-        cfg.gridDim = dim3(2 * pairs);
-        cudaLaunchKernelEx(&cfg, project_pair_kernel, d_descs, d_prefix, n_mat, tile_begin, tile_end, sp, tl, d_status);
-        return;
-    }
     const int grid = tiles < sm_count ? tiles : sm_count;
-    if (tl.staged == 2)
-        project_staged_kernel<<<grid, T2_THREADS, tl.smem_bytes, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end,
-                                                                        sp, tl, d_status);
-    else
-        project_tensor_kernel<<<grid, TC_THREADS, tl.smem_bytes, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end,
+    project_tensor_kernel<<<grid, TC_THREADS, tl.smem_bytes, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end,
                                                                         sp, tl, d_status);
 }
 
