@@ -597,24 +597,35 @@ __global__ void generate_p_kernel(const MatDesc* __restrict__ descs, int mat_beg
 }  // namespace
 
 // G with an odd row pitch -> copy with the pitch rounded up to 8 elements (TMA needs 16-byte rows).
+// One 16-byte store per thread and pass: its eight source elements are 2-byte loads, contiguous
+// across the warp, so every sector is fetched once; the padding columns are written as zero.
 __global__ void repitch_kernel(const MatDesc* __restrict__ descs, int first)
 {
     const MatDesc* dp = descs + first + blockIdx.y;
-    unsigned short* dst = static_cast<unsigned short*>(dp->gpad);
+    uint4* dst = static_cast<uint4*>(dp->gpad);
     if (!dst) return;
     const unsigned short* __restrict__ src = static_cast<const unsigned short*>(dp->G);
-    const int cols = __ldg(&dp->cols), pitch = __ldg(&dp->g_pitch);
-    const int64_t total = (int64_t)__ldg(&dp->rows) * cols;
-    for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t row = e / cols;
-        dst[row * pitch + (e - row * cols)] = __ldg(src + e);
+    const int rows = __ldg(&dp->rows), cols = __ldg(&dp->cols), vecs = __ldg(&dp->g_pitch) / 8;
+    for (int row = blockIdx.x; row < rows; row += gridDim.x) {
+        const unsigned short* __restrict__ in = src + (int64_t)row * cols;
+        for (int v = threadIdx.x; v < vecs; v += blockDim.x) {
+            const int c = 8 * v;
+            uint32_t w[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t lo = c + 2 * e < cols ? (uint32_t)__ldg(in + c + 2 * e) : 0u;
+                const uint32_t hi = c + 2 * e + 1 < cols ? (uint32_t)__ldg(in + c + 2 * e + 1) : 0u;
+                w[e] = lo | (hi << 16);
+            }
+            dst[(int64_t)row * vecs + v] = make_uint4(w[0], w[1], w[2], w[3]);
+        }
     }
 }
 
 void launch_repitch(const MatDesc* d_descs, int first, int count, cudaStream_t stream)
 {
     if (count <= 0) return;
-    const dim3 grid(128, (unsigned)count);
+    const dim3 grid(592, (unsigned)count);
     repitch_kernel<<<grid, 256, 0, stream>>>(d_descs, first);
 }
 
