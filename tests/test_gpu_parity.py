@@ -65,6 +65,43 @@ def test_tensor_core_path(rank, shapes):
     run_parity(wl, expect_path=B.PATH_TENSOR)
 
 
+@pytest.mark.parametrize("env", [
+    {"APOLLO_P_STAGING": "0"},                              # P generated in shared memory by every CTA
+    {"APOLLO_P_STAGING_MB": "1"},                           # staging slots shared group by group: refilled every step
+    {"APOLLO_TC_RSLICE": "64"},                             # four row slices of R per channel tile
+    {"APOLLO_TC_RSLICE": "128", "APOLLO_TC_NBLK": "2"},
+    {"APOLLO_P_STAGING": "0", "APOLLO_TC_RSLICE": "128", "APOLLO_TC_NBLK": "4"},
+])
+def test_tensor_core_path_selectable_modes(env, monkeypatch):
+    """The environment switches of the tensor path give the same parity, and the same bits as the default."""
+    shapes = [(512, 1376), (1376, 512), (512, 512), (300, 1032), (1376, 1400)]   # staged P: 1.6 MB in all
+    wl = _wl(shapes, 256, dtype="bf16", steps=4, T=2, wd=0.01)
+    dev = torch.device("cuda")
+
+    def final_weights():
+        opt = B.Apollo(wl.shapes, B.config_for(wl))
+        W = [WL.make_weight(wl, i).to(dev) for i in range(len(shapes))]
+        for t in range(4):
+            opt.step(W, [WL.make_grad(wl, i, t).to(dev) for i in range(len(shapes))], wl.lr, wl.wd)
+        assert opt.status() == B.OK
+        return W, [opt.scales(i) for i in range(len(shapes))]
+
+    W_default, s_default = final_weights()
+    for k, v in env.items():
+        monkeypatch.setenv(k, v)
+    run_parity(wl, expect_path=B.PATH_TENSOR)
+    W_mode, s_mode = final_weights()
+    if "APOLLO_TC_RSLICE" not in env and "APOLLO_TC_NBLK" not in env:
+        # same tiles, same order of every sum: the bits are the same; another tile shape only reorders sums
+        for a, b in zip(W_default, W_mode):
+            assert torch.equal(a, b)
+        for a, b in zip(s_default, s_mode):
+            assert torch.equal(a, b)
+    else:
+        for a, b in zip(s_default, s_mode):
+            torch.testing.assert_close(a, b, rtol=1e-4, atol=0)
+
+
 def test_tensor_core_path_tensor_mode_and_bias_correction():
     wl = _wl([(256, 520), (520, 256)], 32, mode="tensor", dtype="bf16", steps=3, T=2)
     run_parity(wl, expect_path=B.PATH_TENSOR, bias_correction=True)
