@@ -270,6 +270,16 @@ APOLLO_API int apollo_mini_step_static(void* d_W, const void* d_G, int64_t rows,
                                        const apollo_config* cfg, uint32_t matrix, int64_t t,
                                        float lr, float wd, void* cuda_stream);
 
+/* Self-test of the error path (the paper has no counterpart).  Every wait inside the tensor-core
+ * kernel is bounded: after 2^20 polls it gives up, sets the context's device status word and the
+ * kernel winds down instead of hanging.  This call launches, on the stream, a one-block kernel whose
+ * only wait can never be satisfied, so that the mechanism can be checked on a healthy GPU: the next
+ * apollo_status(ctx) returns APOLLO_ERR_TIMEOUT (and clears the word), and the context works on as
+ * before.  It moves no data and touches no state of the optimizer.  ctx must have run a step (the
+ * status word is set up by the first step), else APOLLO_ERR_INVALID_ARG.  The wait takes of the
+ * order of a second of GPU time before it gives up. */
+APOLLO_API int apollo_selftest_bounded_wait(apollo_ctx* ctx, void* cuda_stream);
+
 /* Kernel launches issued by the last apollo_step (HOST counter). */
 APOLLO_API int apollo_last_launches(const apollo_ctx* ctx, int32_t* out);
 

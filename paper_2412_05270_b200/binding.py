@@ -31,6 +31,7 @@ EXPORTS = [
     "apollo_philox_draws", "apollo_projection", "apollo_get_path", "apollo_last_launches", "apollo_strerror",
     "apollo_set_timing", "apollo_get_timing", "apollo_mini_step_static", "apollo_cuda_error_string", "apollo_adamw_step",
     "apollo_state_bytes", "apollo_state_export", "apollo_state_import", "apollo_step_range", "apollo_set_projection",
+    "apollo_selftest_bounded_wait",
 ]
 
 
@@ -81,6 +82,7 @@ def load():
     lib.apollo_get_state.argtypes = [vp, i32, vp, vp, vp]
     lib.apollo_set_delta_out.argtypes = [vp, ctypes.POINTER(vp)]
     lib.apollo_status.argtypes = [vp, vp]
+    lib.apollo_selftest_bounded_wait.argtypes = [vp, vp]
     lib.apollo_philox_draws.argtypes = [u64, u32, u32, i32, i32, vp, vp]
     lib.apollo_projection.argtypes = [u64, u32, u32, i32, i32, vp, vp]
     lib.apollo_get_path.argtypes = [vp, i32, ctypes.POINTER(i32)]
@@ -298,6 +300,10 @@ class Apollo:
 
     def status(self, stream=None) -> int:
         return self.lib.apollo_status(self.ctx, _stream_ptr(stream))
+
+    def selftest_bounded_wait(self, stream=None):
+        """Launches the kernel whose only wait runs out; the next status() then reports ERR_TIMEOUT."""
+        _check(self.lib.apollo_selftest_bounded_wait(self.ctx, _stream_ptr(stream)), "apollo_selftest_bounded_wait")
 
     def path(self, mat: int) -> int:
         out = ctypes.c_int32(-1)

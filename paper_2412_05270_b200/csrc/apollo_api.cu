@@ -511,6 +511,13 @@ int apollo_get_state(apollo_ctx* ctx, int32_t matrix, float* d_M, float* d_V, vo
     return APOLLO_OK;
 }
 
+int apollo_selftest_bounded_wait(apollo_ctx* ctx, void* cuda_stream)
+{
+    if (!ctx || ctx->first) return APOLLO_ERR_INVALID_ARG;   // the status word exists once a step has run
+    launch_bounded_wait_selftest(ctx->d_status, static_cast<cudaStream_t>(cuda_stream));
+    return cuda_ok(cudaGetLastError()) ? APOLLO_OK : APOLLO_ERR_CUDA;
+}
+
 int apollo_status(apollo_ctx* ctx, void* cuda_stream)
 {
     if (!ctx) return APOLLO_ERR_INVALID_ARG;

@@ -34,6 +34,8 @@ int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, void* d_tmaps, cu
 // Copies the gradients whose row pitch is not a multiple of 16 bytes into their padded buffers.
 void launch_repitch(const MatDesc* d_descs, int first, int count, cudaStream_t stream);
 // Fills the staging buffer with the standard normals of matrices [mat_begin, mat_end).
+// Test hook: a bounded wait that is left to run out (sets STATUS_TIMEOUT in *d_status).
+void launch_bounded_wait_selftest(int32_t* d_status, cudaStream_t stream);
 void launch_generate_p(const MatDesc* d_descs, int mat_begin, int mat_end, const StepParams& sp, cudaStream_t stream);
 // Projection over tiles [tile_begin, tile_end) of the tensor-path prefix table.
 void launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_mat, int tile_begin, int tile_end,

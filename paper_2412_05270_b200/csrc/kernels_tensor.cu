@@ -629,6 +629,32 @@ void launch_repitch(const MatDesc* d_descs, int first, int count, cudaStream_t s
     repitch_kernel<<<grid, 256, 0, stream>>>(d_descs, first);
 }
 
+// One thread waits, with the bound every wait of the tensor kernel has, on an mbarrier that nothing
+// arrives on.  The wait gives up, sets the status word and the block's flag; a second wait returns at
+// once because the flag is set.  The kernel then ends normally: the context stays usable.
+__global__ void bounded_wait_selftest_kernel(int32_t* status)
+{
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int flag;
+    const uint32_t bar_addr = ptx::smem_addr(&bar);
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(bar_addr, 1);
+        flag = 0;
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const bool first = wait_phase(bar_addr, 0, &flag, status);
+        const bool second = wait_phase(bar_addr, 0, &flag, status);
+        if (first || second) atomicExch(status, STATUS_OK);   // a wait that "succeeded" here would be a defect: report no timeout
+    }
+}
+
+void launch_bounded_wait_selftest(int32_t* d_status, cudaStream_t stream)
+{
+    bounded_wait_selftest_kernel<<<1, 32, 0, stream>>>(d_status);
+}
+
 void launch_generate_p(const MatDesc* d_descs, int mat_begin, int mat_end, const StepParams& sp, cudaStream_t stream)
 {
     if (mat_end <= mat_begin) return;

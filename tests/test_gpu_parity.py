@@ -314,3 +314,28 @@ def test_bf16_moment_storage(rank, mode, flags, shapes):
     blob = opt.state_export()
     assert blob.numel() == sum(2 * 2 * rank * max(s) + 4 for s in shapes)
     opt.close()
+
+
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_context_usable():
+    """Every wait of the tensor kernel is bounded; the self-test kernel lets one run out on purpose
+    (an mbarrier nothing arrives on).  The status word turns into ERR_TIMEOUT once, and the optimizer
+    goes on exactly as a context that never saw it."""
+    wl = _wl([(256, 520), (520, 256)], 32, dtype="bf16", steps=3, T=2)
+    dev = torch.device("cuda")
+    a, b = B.Apollo(wl.shapes, B.config_for(wl)), B.Apollo(wl.shapes, B.config_for(wl))
+    with pytest.raises(B.ApolloError):
+        a.selftest_bounded_wait()                 # no step yet: no status word
+    Wa = [WL.make_weight(wl, i).to(dev) for i in range(2)]
+    Wb = [w.clone() for w in Wa]
+    for t in range(3):
+        G = [WL.make_grad(wl, i, t).to(dev) for i in range(2)]
+        a.step(Wa, G, wl.lr, wl.wd)
+        b.step(Wb, G, wl.lr, wl.wd)
+        if t == 0:
+            assert a.status() == B.OK
+            a.selftest_bounded_wait()
+            assert a.status() == B.ERR_TIMEOUT     # reported once ...
+            assert a.status() == B.OK              # ... and cleared
+    assert a.status() == B.OK and b.status() == B.OK
+    for x, y in zip(Wa, Wb):
+        assert torch.equal(x, y)
