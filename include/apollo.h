@@ -88,7 +88,12 @@ typedef struct {
 
 /*
  * Bytes of DEVICE workspace a context over `shapes[0..n_matrices)` needs (moments, scales,
- * partial sums, descriptor tables, tensor maps).  shapes, cfg, out: HOST.
+ * partial sums, descriptor tables, tensor maps, and for the tensor-core path a staging buffer
+ * for the random projections: up to 512 MB, r x m bf16 values per matrix).  When every matrix
+ * has its own slot in that buffer, a projection is generated in the step that opens an epoch
+ * (every T steps, Algorithm 1 "if t mod T = 0") and read again by the following steps of the
+ * epoch, so the steps of one context must reach the GPU in order, whatever streams they use.
+ * shapes, cfg, out: HOST.
  */
 APOLLO_API int apollo_workspace_bytes(const apollo_shape* shapes, int32_t n_matrices, const apollo_config* cfg,
                            size_t* out_bytes);
