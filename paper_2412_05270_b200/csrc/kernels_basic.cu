@@ -75,7 +75,7 @@ constexpr int STREAM_THREADS = 256;
 constexpr int STREAM_TALL_CHUNK = 2048;   // entries of P staged per pass over a tall tile
 
 template <typename T>
-__global__ void __launch_bounds__(STREAM_THREADS)
+__global__ void __launch_bounds__(STREAM_THREADS, 3)     // three blocks per SM: at most 85 registers
 project_stream_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix, int n_mat,
                       int tile_begin, int tile_end, StepParams sp)
 {
@@ -176,17 +176,31 @@ project_stream_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                 }
                 __syncthreads();
                 const int chunk = min(STREAM_TALL_CHUNK, cols - c0);
+                const int rows_left = d.rows - j_base;     // rows of this warp that exist (<= 0: none)
                 for (int x = lane * 8; x < chunk; x += 256) {
                     const int count = min(8, chunk - x);
                     float p[8];
 #pragma unroll
                     for (int e = 0; e < 8; ++e) p[e] = Ps[x + e];   // entries past `chunk` meet zero-filled g
+                    if (vec_ok && rows_left >= 8) {
+                        // all eight 16-byte loads of the warp's rows are issued before the first use
+                        Raw8<T> raw[8];
+#pragma unroll
+                        for (int rr = 0; rr < 8; ++rr) raw[rr] = load_raw8_stream(G + (int64_t)(j_base + rr) * cols + c0 + x);
+#pragma unroll
+                        for (int rr = 0; rr < 8; ++rr) {
+                            float g[8];
+                            unpack_raw8(raw[rr], g);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) { accR[rr] = fmaf(p[e], g[e], accR[rr]); accG[rr] = fmaf(g[e], g[e], accG[rr]); }
+                        }
+                        continue;
+                    }
 #pragma unroll
                     for (int rr = 0; rr < 8; ++rr) {
-                        const int j = j_base + rr;
-                        if (j < d.rows) {
+                        if (rr < rows_left) {
                             float g[8];
-                            const T* src = G + (int64_t)j * cols + c0 + x;
+                            const T* src = G + (int64_t)(j_base + rr) * cols + c0 + x;
                             if (vec_ok) load8_aligned(src, g); else load8_guarded(src, count, g);
 #pragma unroll
                             for (int e = 0; e < 8; ++e) { accR[rr] = fmaf(p[e], g[e], accR[rr]); accG[rr] = fmaf(g[e], g[e], accG[rr]); }
