@@ -79,6 +79,7 @@ struct TcTiling {
     int32_t stages;    // shared-memory pipeline depth
     int32_t smem_bytes;
     int32_t staged;    // 0: P generated in shared memory; 1: P loaded from the staging buffer
+    int32_t pair;      // 1: the pair kernel (CTA pairs, cta_group::2); staged only
 };
 
 // Device status word values.

@@ -61,6 +61,20 @@ TcTiling choose_tiling(int rank)
         if ((v == 1 || v == 2 || v == 4) && v * t.r_slice <= 512) t.nblk = v;
     }
     t.staged = tensor_path_staged() ? 1 : 0;
+    t.pair = 0;
+    // Staged P has two kernels: the pair kernel (default; faster on every list measured) and the
+    // single-CTA ring kernel (APOLLO_TC_KERNEL=ring), which is also the one that can generate P itself.
+    const char* kernel = std::getenv("APOLLO_TC_KERNEL");
+    if (t.staged && !(kernel && std::strcmp(kernel, "ring") == 0)) {
+        // pair tile: 256 channels (128 per CTA) x r_slice rows, accumulator double buffered
+        t.pair = 1;
+        t.nblk = 2;
+        const int stage = 128 * TC_BK * 2 + (t.r_slice / 2) * 128;
+        t.stages = (TC_MAX_SMEM - 13824) / stage;
+        if (t.stages > 8) t.stages = 8;
+        t.smem_bytes = t.stages * stage + 13824;
+        return t;
+    }
     const int stage = t.nblk * TC_BLOCK_BYTES + t.r_slice * 128;
     t.stages = (TC_MAX_SMEM - TC_MISC_BYTES) / stage;
     if (t.stages > 4) t.stages = 4;
@@ -156,7 +170,7 @@ int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, void* d_tmaps, cu
             // staged P: rank rows of m_pad bf16, loaded as 64 x r_slice boxes (K-major UMMA tiles)
             const cuuint64_t pdims[2] = { (cuuint64_t)d.m_pad, (cuuint64_t)rank };
             const cuuint64_t pstrides[1] = { (cuuint64_t)d.m_pad * 2 };
-            const cuuint32_t pbox[2] = { 64u, (cuuint32_t)tl.r_slice };
+            const cuuint32_t pbox[2] = { 64u, (cuuint32_t)(tl.pair ? tl.r_slice / 2 : tl.r_slice) };
             const CUresult rp = encode(&maps[2 * i + 1], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, d.pstage, pdims, pstrides,
                                        pbox, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -560,6 +574,272 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
     if (warp == 1) ptx::tmem_dealloc(tmem_base, 512);
 }
 
+// ----------------------------------------------------------------------------------------
+// Pair kernel (APOLLO_TC_KERNEL=pair): two CTAs of a cluster share every MMA (cta_group::2,
+// M = 256).  A pair tile is 256 channels x r_slice rows of R.  Each CTA loads the G tile of its own
+// 128 channels and half of the rows of the P tile (so a k-block costs 32 KB of shared-memory fill per
+// CTA instead of 48 KB for the same work), and keeps r_slice accumulator columns per buffer, double
+// buffered: the epilogue of one tile runs under the main loop of the next.
+//   warp 0      producer: TMA loads of both CTAs count their bytes on the LEADER's `full` barrier
+//   warp 1      leader only: MMA issuer; its commits are multicast to both CTAs
+//   warps 4-7   squared column norms of this CTA's G tile, after the MMA that read it has finished
+//   warps 8-15  epilogue of this CTA's 128 channels
+// Barriers per stage s: full[s] (leader: one arrive.expect_tx for the bytes of both CTAs),
+// done[s] (both: the leader's commit), empty[s] (both: the four norm warps).
+// ----------------------------------------------------------------------------------------
+constexpr int P2_THREADS = 512;
+constexpr int P2_G_BYTES = 128 * TC_BK * 2;        // G of 128 channels, one k-block: 16 KiB
+constexpr int P2_MAX_STAGES = 8;
+constexpr int P2_MISC_BYTES = 512 + 2 * 2 * 128 * 8 + 2 * 8 * 128 * 4 + 1024;   // barriers, red, g2s, alignment slack
+static_assert(P2_MISC_BYTES == 13824, "choose_tiling() reserves this many bytes");
+
+__global__ void __launch_bounds__(P2_THREADS, 1)
+project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix, int n_mat, int tile_begin,
+                    int tile_end, StepParams sp, TcTiling tl, int32_t* __restrict__ status)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_addr(smem_raw));
+
+    const uint32_t rank = ptx::cluster_ctarank();          // 0: leader, 1: peer
+    const int r_slice = tl.r_slice, ns = tl.stages, r_half = r_slice / 2;
+    const uint32_t p_bytes = (uint32_t)r_half * 128u, stage_bytes = (uint32_t)P2_G_BYTES + p_bytes;
+    const uint32_t misc = (uint32_t)ns * stage_bytes;
+    const uint32_t bars = smem_base + misc;
+    const uint32_t bar_full = bars, bar_done = bars + 64, bar_empty = bars + 128, bar_acc_full = bars + 192,
+                   bar_acc_empty = bars + 208, bar_drain = bars + 224;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + misc + 240);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + misc + 244);
+    float2* red = reinterpret_cast<float2*>(smem_gen + misc + 512);                 // [2 tiles][2 halves][128]
+    float* g2s = reinterpret_cast<float*>(smem_gen + misc + 512 + 2 * 2 * 128 * 8);   // [2 tiles][8 parts][128]
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    if (tid == 0) {
+        for (int s = 0; s < ns; ++s) {
+            ptx::mbar_init(bar_full + 8 * s, 1);        // the leader's arrive.expect_tx
+            ptx::mbar_init(bar_done + 8 * s, 1);        // the leader's commit
+            ptx::mbar_init(bar_empty + 8 * s, 4);       // four norm warps of this CTA
+        }
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(bar_acc_full + 8 * b, 1);    // the leader's commit
+            ptx::mbar_init(bar_acc_empty + 8 * b, 16);  // eight epilogue warps of each CTA (the leader's copy is used)
+        }
+        ptx::mbar_init(bar_drain, 1);
+        *abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc_pair(ptx::smem_addr(tmem_slot), 512);
+        ptx::tmem_relinquish_pair();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::cluster_sync();          // both CTAs' barriers exist before any remote arrive, remote byte count or multicast commit
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    uint32_t it = 0, tile_iter = 0;   // k-block and tile counters of this role
+
+    const int pair = blockIdx.x >> 1, pairs = gridDim.x >> 1;
+    for (int tile = tile_begin + pair; tile < tile_end; tile += pairs, ++tile_iter) {
+        const int mat = find_matrix(prefix, n_mat, tile);
+        const MatDesc* dp = descs + mat;
+        const int tiles_k = __ldg(&dp->tiles_k);
+        const int m = __ldg(&dp->m), n = __ldg(&dp->n);
+        const bool tall = __ldg(&dp->tall) != 0;
+        const int local = tile - __ldg(prefix + mat);
+        const int tr = local % tiles_k, tn = local / tiles_k;
+        const int j0 = tn * 256 + (int)rank * 128, r0 = tr * r_slice;
+        const int num_kb = (m + TC_BK - 1) / TC_BK;
+        const uint32_t buf = tile_iter & 1, use = tile_iter >> 1;
+
+        if (warp == 0) {
+            // ---------------- producer (one thread in each CTA) ----------------
+            if (lane == 0) {
+                const void* tmap = dp->tmap;
+                const void* tmap_p = dp->tmap_p;
+                ptx::fence_tensormap_acquire(tmap);
+                ptx::fence_tensormap_acquire(tmap_p);
+                const uint64_t pol_g = ptx::policy_evict_first(), pol_p = ptx::policy_evict_last();
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const uint32_t s = it % ns, ph = (it / ns) & 1;
+                    if (!wait_phase(bar_empty + 8 * s, ph ^ 1, abort_flag, status)) break;
+                    const uint32_t g_s = smem_base + s * stage_bytes, p_s = g_s + P2_G_BYTES;
+                    // the bytes of both CTAs are counted on the leader's barrier; the peer's may arrive
+                    // there before the leader's expect_tx (the count is signed), never a phase early,
+                    // because the peer's stage is only free once the leader's MMA has consumed it
+                    const uint32_t full = ptx::map_to_cta(bar_full + 8 * s, 0);
+                    if (rank == 0) ptx::mbar_arrive_expect_tx(bar_full + 8 * s, 2u * stage_bytes);
+                    if (tall) {
+                        ptx::tma_load_2d_pair(g_s, tmap, kb * TC_BK, j0, full, pol_g);
+                    } else {
+                        ptx::tma_load_2d_pair(g_s, tmap, j0, kb * TC_BK, full, pol_g);
+                        ptx::tma_load_2d_pair(g_s + P2_G_BYTES / 2, tmap, j0 + 64, kb * TC_BK, full, pol_g);
+                    }
+                    ptx::tma_load_2d_pair(p_s, tmap_p, kb * TC_BK, r0 + (int)rank * r_half, full, pol_p);
+                }
+            }
+            __syncwarp();
+            if (__shfl_sync(0xFFFFFFFFu, *abort_flag, 0) != 0) break;
+        } else if (warp == 1) {
+            // ---------------- MMA issuer (leader only) ----------------
+            if (lane == 0 && rank == 0) {
+                const uint32_t idesc = ptx::instr_desc_bf16((uint32_t)r_slice, !tall, 256u);
+                const uint32_t d_tmem = tmem_base + buf * (uint32_t)r_slice;
+                bool ok = wait_phase(bar_acc_empty + 8 * buf, (use & 1) ^ 1, abort_flag, status);   // epilogue of the tile before last
+                ptx::tc_fence_after_sync();
+                int kb = 0;
+                for (; ok && kb < num_kb; ++kb, ++it) {
+                    const uint32_t s = it % ns, ph = (it / ns) & 1;
+                    if (!wait_phase(bar_full + 8 * s, ph, abort_flag, status)) break;
+                    ptx::tc_fence_after_sync();
+                    const uint32_t g_s = smem_base + s * stage_bytes, p_s = g_s + P2_G_BYTES;
+#pragma unroll
+                    for (int kk = 0; kk < TC_BK / 16; ++kk) {
+                        const uint64_t a_desc = tall ? ptx::smem_desc_sw128(g_s + kk * 32, 16, 1024)
+                                                     : ptx::smem_desc_sw128(g_s + kk * 2048, P2_G_BYTES / 2, 1024);
+                        const uint64_t b_desc = ptx::smem_desc_sw128(p_s + kk * 32, 16, 1024);
+                        ptx::mma_bf16_pair(d_tmem, a_desc, b_desc, idesc, (kb | kk) != 0 ? 1u : 0u);
+                    }
+                    ptx::mma_commit_pair(bar_done + 8 * s, 3);
+                }
+                if (ok && kb == num_kb) ptx::mma_commit_pair(bar_acc_full + 8 * buf, 3);
+            }
+            __syncwarp();
+            if (__shfl_sync(0xFFFFFFFFu, *abort_flag, 0) != 0) break;
+        } else if (warp >= 4 && warp < 8) {
+            // ---------------- squared column norms of this CTA's 128 channels ----------------
+            const int t = tid - 128;
+            float acc[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+            const int cc = t & 15, part = t >> 4;     // wide: 16 chunk columns x 8 row groups
+            for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                const uint32_t s = it % ns, ph = (it / ns) & 1;
+                if (!wait_phase(bar_done + 8 * s, ph, abort_flag, status)) break;   // landed, and the MMA has read it
+                const uint32_t g_s = smem_base + s * stage_bytes;
+                if (tall) {
+                    // units (row, half): 256 units over 128 threads; the order of the chunks is free
+#pragma unroll
+                    for (int pass = 0; pass < 2; ++pass) {
+                        const int u = t + pass * 128, row = u >> 1, half = u & 1;
+                        const uint32_t base = g_s + row * 128 + half * 64;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) acc[pass] += sum_sq_bf16x8(ld_shared_v4(base + (((i + row) & 3) << 4)));
+                    }
+                } else {
+                    const uint32_t colbase = g_s + (cc >> 3) * (P2_G_BYTES / 2);
+                    const int c = cc & 7;
+#pragma unroll
+                    for (int i8 = 0; i8 < 8; ++i8) {
+                        const int k = part + 8 * i8;
+                        const uint4 v = ld_shared_v4(colbase + k * 128 + ((c ^ (k & 7)) << 4));
+                        const uint32_t w[4] = { v.x, v.y, v.z, v.w };
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
+                            acc[2 * i] = fmaf(lo, lo, acc[2 * i]);
+                            acc[2 * i + 1] = fmaf(hi, hi, acc[2 * i + 1]);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(bar_empty + 8 * s);
+            }
+            float* mine = g2s + buf * (8 * 128);
+            if (tall) {
+#pragma unroll
+                for (int pass = 0; pass < 2; ++pass) {
+                    const int u = t + pass * 128;
+                    mine[(u & 1) * 128 + (u >> 1)] = acc[pass];
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) mine[part * 128 + cc * 8 + e] = acc[e];
+            }
+            const bool stop = ptx::named_barrier_or(3, 128, *abort_flag != 0);
+            const int j = j0 + t;
+            if (!stop && tr == 0 && j < n) {
+                float g2 = 0.f;
+                const int parts = tall ? 2 : 8;
+                for (int p = 0; p < parts; ++p) g2 += mine[p * 128 + t];
+                dp->g2[j] = g2;
+            }
+            if (stop) break;
+        } else if (warp >= 8) {
+            // ---------------- epilogue of this tile, under the main loop of the next ----------------
+            const int q = warp & 3, half = (warp - 8) >> 2;
+            const int ch = q * 32 + lane, j = j0 + ch;
+            float* const Mbase = dp->M;
+            float* const Vbase = dp->V;
+            const float r_scale = __ldg(&dp->r_scale);
+            const bool acc_ok = wait_phase(bar_acc_full + 8 * buf, use & 1, abort_flag, status);
+            ptx::tc_fence_after_sync();
+            float num = 0.f, den = 0.f;
+            const int chunks = acc_ok ? r_slice / 16 : 0;
+            for (int cchunk = half; cchunk < chunks; cchunk += 2) {
+                float rv[16];
+                ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + buf * (uint32_t)r_slice + (uint32_t)(cchunk * 16), rv);
+                if (j < n) {
+                    const int64_t at = (int64_t)(r0 + cchunk * 16) * n + j;
+                    const bool sb = sp.state_bf16 != 0;
+                    float mv[16], vv[16];
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) {
+                        mv[k] = state_load(Mbase, at + (int64_t)k * n, sb);
+                        vv[k] = state_load(Vbase, at + (int64_t)k * n, sb);
+                    }
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) {
+                        const float r = rv[k] * r_scale;
+                        const float mn = sp.beta1 * mv[k] + (1.0f - sp.beta1) * r;
+                        const float vn = sp.beta2 * vv[k] + (1.0f - sp.beta2) * r * r;
+                        state_store(Mbase, at + (int64_t)k * n, mn, sb); state_store(Vbase, at + (int64_t)k * n, vn, sb);
+                        const float rt = __fdividef(mn * sp.inv_bc1, fast_sqrt(vn * sp.inv_bc2) + sp.eps);
+                        num = fmaf(rt, rt, num);
+                        den = fmaf(r, r, den);
+                    }
+                }
+            }
+            // this warp has read its share of the accumulator: hand the buffer back to the issuer
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0 && acc_ok) ptx::mbar_arrive_remote(ptx::map_to_cta(bar_acc_empty + 8 * buf, 0));
+            float2* mine = red + buf * (2 * 128);
+            mine[half * 128 + ch] = make_float2(num, den);
+            const bool stop = ptx::named_barrier_or(1, 256, *abort_flag != 0);
+            if (!stop && half == 0 && j < n) {
+                const float2 a = mine[ch], b = mine[128 + ch];
+                reinterpret_cast<float2*>(dp->part)[(int64_t)tr * n + j] = make_float2(a.x + b.x, a.y + b.y);
+            }
+            if (stop) break;
+        } else if (__shfl_sync(0xFFFFFFFFu, *abort_flag, 0) != 0) {
+            break;                                     // spare warps
+        }
+    }
+
+    // The leader lets the loads of both CTAs (they are counted on its barriers) and its MMAs finish
+    // before either CTA gives up shared memory or TMEM; on the normal path these return at once.
+    if (rank == 0 && tid == 0) {
+        for (uint32_t s = 0; s < (uint32_t)ns && s < it; ++s) {
+            const uint32_t last = s + (it - 1 - s) / ns * ns;
+            drain_phase(bar_full + 8 * s, (last / ns) & 1);
+        }
+    }
+    if (rank == 0 && tid == 32) {
+        ptx::mma_commit_pair(bar_drain, 1);
+        drain_phase(bar_drain, 0);
+    }
+    // the peer cannot watch the leader's barriers: after a wait gave up it lets its last loads land for 2 ms
+    if (rank == 1 && tid == 0 && *abort_flag)
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::cluster_sync();          // no remote arrive, remote byte count or MMA of the pair is still under way
+    if (warp == 1) ptx::tmem_dealloc_pair(tmem_base, 512);
+}
+
 // Standard normals of the staged P: one 16-byte store (8 bf16) per thread and pass.
 __global__ void generate_p_kernel(const MatDesc* __restrict__ descs, int mat_begin, StepParams sp)
 {
@@ -675,7 +955,37 @@ void launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_ma
     bool& attr_set = attr_set_on[device & 63];
     if (!attr_set) {
         cudaFuncSetAttribute(project_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
+        cudaFuncSetAttribute(project_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
         attr_set = true;
+    }
+    if (tl.pair) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(sm_count / 2 * 2);
+        cfg.blockDim = dim3(P2_THREADS);
+        cfg.dynamicSmemBytes = tl.smem_bytes;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        // the tile loop is persistent: launch exactly as many pairs as can be resident at once
+        // (a pair sits in one GPC, so this can be fewer than half the SMs)
+        static int max_pairs_on[64] = {};
+        int& max_pairs = max_pairs_on[device & 63];
+        if (max_pairs == 0) {
+            int clusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&clusters, project_pair_kernel, &cfg) != cudaSuccess || clusters < 1) {
+                cudaGetLastError();
+                clusters = sm_count / 2;
+            }
+            max_pairs = clusters;
+        }
+        int pairs = max_pairs;
+        if (tiles < pairs) pairs = tiles;
+        cfg.gridDim = dim3(2 * pairs);
+        cudaLaunchKernelEx(&cfg, project_pair_kernel, d_descs, d_prefix, n_mat, tile_begin, tile_end, sp, tl, d_status);
+        return;
     }
     const int grid = tiles < sm_count ? tiles : sm_count;
     project_tensor_kernel<<<grid, TC_THREADS, tl.smem_bytes, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end,

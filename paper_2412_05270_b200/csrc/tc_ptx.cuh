@@ -155,6 +155,74 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16])
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// ---- CTA pairs (cluster of two, cta_group::2) ----------------------------------------------
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Address of the same shared-memory location in the CTA of rank `rank` of this cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank)
+{
+    uint32_t a;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(local_addr), "r"(rank));
+    return a;
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// 2D tile load of a CTA pair: the data lands in this CTA's shared memory, the bytes are counted on
+// the mbarrier at `bar_cluster_addr`, which may belong to either CTA of the pair (no multicast).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const void* tmap, int32_t x, int32_t y,
+                                                 uint32_t bar_cluster_addr, uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(bar_cluster_addr), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t cols)   // one warp in each CTA of the pair
+{
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// D (256 rows over the two CTAs) (+)= A * B^T; issued by one thread of the leader CTA; each CTA
+// supplies its 128 rows of A and its half of the rows of B from its own shared memory.
+__device__ __forceinline__ void mma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                              uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}\n"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Arrive, once the pair's MMAs issued so far are complete, on the barrier at this offset in
+// every CTA of `cta_mask`.
+__device__ __forceinline__ void mma_commit_pair(uint32_t bar, uint16_t cta_mask)
+{
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(bar), "h"(cta_mask)
+        : "memory");
+}
+
 // ---- named barriers, hints ---------------------------------------------------------------
 __device__ __forceinline__ void named_barrier(uint32_t id, uint32_t threads)
 {
@@ -193,10 +261,10 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr, uint32_t lbo_
     return d;
 }
 
-// Instruction descriptor for kind::f16 with bf16 A and B, fp32 D, M = 128.
+// Instruction descriptor for kind::f16 with bf16 A and B, fp32 D, M = 128 (256 for a CTA pair).
 //   bits 4..5 D format (1 = f32); 7..9 A format (1 = bf16); 10..12 B format (1 = bf16);
 //   bit 15 A major (1 = MN-major); bit 16 B major; bits 17..22 N >> 3; bits 24..28 M >> 4.
-__device__ __forceinline__ uint32_t instr_desc_bf16(uint32_t n, bool a_mn_major)
+__device__ __forceinline__ uint32_t instr_desc_bf16(uint32_t n, bool a_mn_major, uint32_t m = 128u)
 {
     uint32_t d = 0;
     d |= 1u << 4;
@@ -204,7 +272,7 @@ __device__ __forceinline__ uint32_t instr_desc_bf16(uint32_t n, bool a_mn_major)
     d |= 1u << 10;
     d |= (a_mn_major ? 1u : 0u) << 15;
     d |= (n >> 3) << 17;
-    d |= (128u >> 4) << 24;
+    d |= (m >> 4) << 24;
     return d;
 }
 

@@ -66,14 +66,17 @@ def test_tensor_core_path(rank, shapes):
 
 
 @pytest.mark.parametrize("env", [
-    {"APOLLO_P_STAGING": "0"},                              # P generated in shared memory by every CTA
     {"APOLLO_P_STAGING_MB": "1"},                           # staging slots shared group by group: refilled every step
     {"APOLLO_TC_RSLICE": "64"},                             # four row slices of R per channel tile
-    {"APOLLO_TC_RSLICE": "128", "APOLLO_TC_NBLK": "2"},
+    {"APOLLO_TC_KERNEL": "ring"},                           # single-CTA kernel, 256 channels x 256 rows per tile
+    {"APOLLO_TC_KERNEL": "ring", "APOLLO_P_STAGING_MB": "1"},
+    {"APOLLO_TC_KERNEL": "ring", "APOLLO_TC_RSLICE": "128", "APOLLO_TC_NBLK": "2"},
+    {"APOLLO_P_STAGING": "0"},                              # P generated in shared memory by every CTA (ring kernel)
     {"APOLLO_P_STAGING": "0", "APOLLO_TC_RSLICE": "128", "APOLLO_TC_NBLK": "4"},
 ])
 def test_tensor_core_path_selectable_modes(env, monkeypatch):
-    """The environment switches of the tensor path give the same parity, and the same bits as the default."""
+    """The environment switches of the tensor path give the same parity; where they leave the tiles and
+    the order of every sum alone, they give the same bits."""
     shapes = [(512, 1376), (1376, 512), (512, 512), (300, 1032), (1376, 1400)]   # staged P: 1.6 MB in all
     wl = _wl(shapes, 256, dtype="bf16", steps=4, T=2, wd=0.01)
     dev = torch.device("cuda")
@@ -86,20 +89,21 @@ def test_tensor_core_path_selectable_modes(env, monkeypatch):
         assert opt.status() == B.OK
         return W, [opt.scales(i) for i in range(len(shapes))]
 
-    W_default, s_default = final_weights()
+    # the run to compare with: the same kernel and tile shape, P staged once per epoch
+    same_tiles = {k: v for k, v in env.items() if k in ("APOLLO_TC_KERNEL", "APOLLO_TC_RSLICE", "APOLLO_TC_NBLK")}
+    if env.get("APOLLO_P_STAGING") == "0":
+        same_tiles["APOLLO_TC_KERNEL"] = "ring"             # the kernel that generates P itself
+    for k, v in same_tiles.items():
+        monkeypatch.setenv(k, v)
+    W_ref, s_ref = final_weights()
     for k, v in env.items():
         monkeypatch.setenv(k, v)
     run_parity(wl, expect_path=B.PATH_TENSOR)
     W_mode, s_mode = final_weights()
-    if "APOLLO_TC_RSLICE" not in env and "APOLLO_TC_NBLK" not in env:
-        # same tiles, same order of every sum: the bits are the same; another tile shape only reorders sums
-        for a, b in zip(W_default, W_mode):
-            assert torch.equal(a, b)
-        for a, b in zip(s_default, s_mode):
-            assert torch.equal(a, b)
-    else:
-        for a, b in zip(s_default, s_mode):
-            torch.testing.assert_close(a, b, rtol=1e-4, atol=0)
+    for a, b in zip(W_ref, W_mode):
+        assert torch.equal(a, b)
+    for a, b in zip(s_ref, s_mode):
+        assert torch.equal(a, b)
 
 
 def test_tensor_core_path_tensor_mode_and_bias_correction():
