@@ -82,9 +82,7 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
             }
         } else if (tensor_path_supports(p.rows, p.cols, r, cfg->dtype) && !(cfg->flags & APOLLO_FLAG_NO_TENSOR_CORES)) {
             p.path = PATH_TENSOR;
-            tensor_path_tiling(p.rows, p.cols, r, &p.tiles_n, &p.tiles_k);
-            p.slices = p.tiles_k;
-            p.g2_slices = 1;
+            tensor_path_tiling(p.rows, p.cols, r, &p.tiles_n, &p.tiles_k, &p.slices, &p.g2_slices);
         } else {
             p.path = PATH_SIMT;
             p.tiles_n = (p.n + SIMT_BN - 1) / SIMT_BN;

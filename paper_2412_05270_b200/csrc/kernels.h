@@ -22,7 +22,8 @@ void launch_widen_bf16(const void* d_src, float* d_dst, size_t count, cudaStream
 
 // Tensor-core projection (TMA + tcgen05 + TMEM).
 bool tensor_path_supports(int rows, int cols, int rank, int dtype);
-void tensor_path_tiling(int rows, int cols, int rank, int32_t* tiles_n, int32_t* tiles_k);
+void tensor_path_tiling(int rows, int cols, int rank, int32_t* tiles_n, int32_t* tiles_k, int32_t* slices,
+                        int32_t* g2_slices);
 // L2 staging of P: whether it is on, the byte budget of the staging buffer, and the bytes
 // one matrix needs in it (rank x round_up(m, 64) bf16).
 bool tensor_path_staged();

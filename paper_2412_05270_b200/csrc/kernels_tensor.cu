@@ -70,9 +70,9 @@ TcTiling choose_tiling(int rank)
         t.pair = 1;
         t.nblk = 2;
         const int stage = 128 * TC_BK * 2 + (t.r_slice / 2) * 128;
-        t.stages = (TC_MAX_SMEM - 13824) / stage;
+        t.stages = (TC_MAX_SMEM - 1536) / stage;
         if (t.stages > 8) t.stages = 8;
-        t.smem_bytes = t.stages * stage + 13824;
+        t.smem_bytes = t.stages * stage + 1536;
         return t;
     }
     const int stage = t.nblk * TC_BLOCK_BYTES + t.r_slice * 128;
@@ -134,12 +134,17 @@ bool tensor_path_supports(int rows, int cols, int rank, int dtype)
     return true;
 }
 
-void tensor_path_tiling(int rows, int cols, int rank, int32_t* tiles_n, int32_t* tiles_k)
+void tensor_path_tiling(int rows, int cols, int rank, int32_t* tiles_n, int32_t* tiles_k, int32_t* slices,
+                        int32_t* g2_slices)
 {
     const TcTiling t = choose_tiling(rank);
     const int n = rows > cols ? rows : cols;
     *tiles_n = (n + t.nblk * 128 - 1) / (t.nblk * 128);
     *tiles_k = rank / t.r_slice;
+    // partial sums a tile leaves for finalize_kernel: the pair kernel writes one slice per half of its
+    // epilogue warps and, for a wide matrix, one slice of squared column norms per norm warp
+    *slices = t.pair ? 2 * *tiles_k : *tiles_k;
+    *g2_slices = t.pair && rows <= cols ? 4 : 1;
 }
 
 int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, void* d_tmaps, cudaStream_t stream)
@@ -412,7 +417,7 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
             }
             for (int kb = 0; kb < num_kb && !staged; ++kb, ++it) {
                 const uint32_t s = it % stages, ph = (it / stages) & 1;
-                if (!wait_phase(bar_empty + 8 * s, ph ^ 1, abort_flag, status)) break;
+                if (!__all_sync(0xFFFFFFFFu, wait_phase(bar_empty + 8 * s, ph ^ 1, abort_flag, status))) break;
                 const uint32_t p_s = smem_base + s * stage_bytes + p_off;
                 // two rows per pass (32 rows apart) so that four Philox chains are in flight per thread
                 const int total = r_slice * 8;
@@ -450,7 +455,7 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
             const int rows_pp = TC_BK / parts;
             for (int kb = 0; kb < num_kb; ++kb, ++it) {
                 const uint32_t s = it % stages, ph = (it / stages) & 1;
-                if (!wait_phase(bar_g_full + 8 * s, ph, abort_flag, status)) break;
+                if (!__all_sync(0xFFFFFFFFu, wait_phase(bar_g_full + 8 * s, ph, abort_flag, status))) break;   // the warp stays together
                 const uint32_t g_s = smem_base + s * stage_bytes;
                 if (tall) {
                     // block b, row t: 128 bytes = 8 chunks; the order of the chunks does not matter
@@ -493,7 +498,7 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
             const int q = warp & 3, widx = (warp - 2) >> 2;
             const int ch_in_blk = q * 32 + lane;
             for (int b = 0; b < nblk; ++b) red[widx * chan_tile + b * 128 + ch_in_blk] = make_float2(0.f, 0.f);
-            const bool acc_ok = wait_phase(bar_acc, tile_iter & 1, abort_flag, status);
+            const bool acc_ok = __all_sync(0xFFFFFFFFu, wait_phase(bar_acc, tile_iter & 1, abort_flag, status));   // tcgen05.ld needs the whole warp
             ptx::tc_fence_after_sync();
             const int chunks = r_slice / 16, items = acc_ok ? nblk * chunks : 0;
             float num = 0.f, den = 0.f;
@@ -586,12 +591,15 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
 //   warps 8-15  epilogue of this CTA's 128 channels
 // Barriers per stage s: full[s] (leader: one arrive.expect_tx for the bytes of both CTAs),
 // done[s] (both: the leader's commit), empty[s] (both: the four norm warps).
+// Shared memory holds nothing but the ring and the barriers (seven 32 KB stages at r_slice = 256):
+// the per-channel partial sums go to global memory as slices that finalize_kernel adds up, one
+// per half of the epilogue warps and, for wide matrices, one per norm warp.
 // ----------------------------------------------------------------------------------------
 constexpr int P2_THREADS = 512;
 constexpr int P2_G_BYTES = 128 * TC_BK * 2;        // G of 128 channels, one k-block: 16 KiB
 constexpr int P2_MAX_STAGES = 8;
-constexpr int P2_MISC_BYTES = 512 + 2 * 2 * 128 * 8 + 2 * 8 * 128 * 4 + 1024;   // barriers, red, g2s, alignment slack
-static_assert(P2_MISC_BYTES == 13824, "choose_tiling() reserves this many bytes");
+constexpr int P2_MISC_BYTES = 512 + 1024;          // barriers and flags, alignment slack
+static_assert(P2_MISC_BYTES == 1536, "choose_tiling() reserves this many bytes");
 
 __global__ void __launch_bounds__(P2_THREADS, 1)
 project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix, int n_mat, int tile_begin,
@@ -610,8 +618,6 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                    bar_acc_empty = bars + 208, bar_drain = bars + 224;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + misc + 240);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + misc + 244);
-    float2* red = reinterpret_cast<float2*>(smem_gen + misc + 512);                 // [2 tiles][2 halves][128]
-    float* g2s = reinterpret_cast<float*>(smem_gen + misc + 512 + 2 * 2 * 128 * 8);   // [2 tiles][8 parts][128]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -717,7 +723,7 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             const int cc = t & 15, part = t >> 4;     // wide: 16 chunk columns x 8 row groups
             for (int kb = 0; kb < num_kb; ++kb, ++it) {
                 const uint32_t s = it % ns, ph = (it / ns) & 1;
-                if (!wait_phase(bar_done + 8 * s, ph, abort_flag, status)) break;   // landed, and the MMA has read it
+                if (!__all_sync(0xFFFFFFFFu, wait_phase(bar_done + 8 * s, ph, abort_flag, status))) break;   // landed, and the MMA has read it
                 const uint32_t g_s = smem_base + s * stage_bytes;
                 if (tall) {
                     // units (row, half): 256 units over 128 threads; the order of the chunks is free
@@ -747,24 +753,25 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(bar_empty + 8 * s);
             }
-            float* mine = g2s + buf * (8 * 128);
+            // squared norms of this tile's channels -> global slices (only the first row slice writes them)
+            const bool stop = __shfl_sync(0xFFFFFFFFu, *abort_flag, 0) != 0;     // one answer per warp
+            float* const g2out = dp->g2;
             if (tall) {
+                // lanes 2k and 2k+1 hold the two halves of one stored row
 #pragma unroll
                 for (int pass = 0; pass < 2; ++pass) {
-                    const int u = t + pass * 128;
-                    mine[(u & 1) * 128 + (u >> 1)] = acc[pass];
+                    const float v = acc[pass] + __shfl_xor_sync(0xFFFFFFFFu, acc[pass], 1);
+                    const int j = j0 + ((t + pass * 128) >> 1);
+                    if (!stop && tr == 0 && !(lane & 1) && j < n) g2out[j] = v;
                 }
             } else {
+                // lanes l and l + 16 hold two row groups of the same eight channels: one slice per warp
 #pragma unroll
-                for (int e = 0; e < 8; ++e) mine[part * 128 + cc * 8 + e] = acc[e];
-            }
-            const bool stop = ptx::named_barrier_or(3, 128, *abort_flag != 0);
-            const int j = j0 + t;
-            if (!stop && tr == 0 && j < n) {
-                float g2 = 0.f;
-                const int parts = tall ? 2 : 8;
-                for (int p = 0; p < parts; ++p) g2 += mine[p * 128 + t];
-                dp->g2[j] = g2;
+                for (int e = 0; e < 8; ++e) {
+                    const float v = acc[e] + __shfl_xor_sync(0xFFFFFFFFu, acc[e], 16);
+                    const int j = j0 + cc * 8 + e;
+                    if (!stop && tr == 0 && lane < 16 && j < n) g2out[(int64_t)(warp - 4) * n + j] = v;
+                }
             }
             if (stop) break;
         } else if (warp >= 8) {
@@ -774,7 +781,7 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             float* const Mbase = dp->M;
             float* const Vbase = dp->V;
             const float r_scale = __ldg(&dp->r_scale);
-            const bool acc_ok = wait_phase(bar_acc_full + 8 * buf, use & 1, abort_flag, status);
+            const bool acc_ok = __all_sync(0xFFFFFFFFu, wait_phase(bar_acc_full + 8 * buf, use & 1, abort_flag, status));   // tcgen05.ld needs the whole warp
             ptx::tc_fence_after_sync();
             float num = 0.f, den = 0.f;
             const int chunks = acc_ok ? r_slice / 16 : 0;
@@ -806,14 +813,9 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0 && acc_ok) ptx::mbar_arrive_remote(ptx::map_to_cta(bar_acc_empty + 8 * buf, 0));
-            float2* mine = red + buf * (2 * 128);
-            mine[half * 128 + ch] = make_float2(num, den);
-            const bool stop = ptx::named_barrier_or(1, 256, *abort_flag != 0);
-            if (!stop && half == 0 && j < n) {
-                const float2 a = mine[ch], b = mine[128 + ch];
-                reinterpret_cast<float2*>(dp->part)[(int64_t)tr * n + j] = make_float2(a.x + b.x, a.y + b.y);
-            }
-            if (stop) break;
+            if (acc_ok && j < n)
+                reinterpret_cast<float2*>(dp->part)[(int64_t)(tr * 2 + half) * n + j] = make_float2(num, den);
+            if (__shfl_sync(0xFFFFFFFFu, *abort_flag, 0) != 0) break;
         } else if (__shfl_sync(0xFFFFFFFFu, *abort_flag, 0) != 0) {
             break;                                     // spare warps
         }
