@@ -580,7 +580,7 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
 }
 
 // ----------------------------------------------------------------------------------------
-// Pair kernel (APOLLO_TC_KERNEL=pair): two CTAs of a cluster share every MMA (cta_group::2,
+// Pair kernel (default for staged P): two CTAs of a cluster share every MMA (cta_group::2,
 // M = 256).  A pair tile is 256 channels x r_slice rows of R.  Each CTA loads the G tile of its own
 // 128 channels and half of the rows of the P tile (so a k-block costs 32 KB of shared-memory fill per
 // CTA instead of 48 KB for the same work), and keeps r_slice accumulator columns per buffer, double
@@ -725,7 +725,9 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                 const uint32_t s = it % ns, ph = (it / ns) & 1;
                 if (!__all_sync(0xFFFFFFFFu, wait_phase(bar_done + 8 * s, ph, abort_flag, status))) break;   // landed, and the MMA has read it
                 const uint32_t g_s = smem_base + s * stage_bytes;
-                if (tall) {
+                if (tr != 0) {
+                    // the norms belong to the channel tile, not to the row slice: the first slice has them
+                } else if (tall) {
                     // units (row, half): 256 units over 128 threads; the order of the chunks is free
 #pragma unroll
                     for (int pass = 0; pass < 2; ++pass) {
