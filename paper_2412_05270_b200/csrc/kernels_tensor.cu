@@ -3,7 +3,10 @@
 // step 2; Eq. 5).  P is either loaded from a staging buffer that generate_p_kernel fills once
 // per epoch (default) or generated straight into shared memory by every CTA.
 //
-// Roles of the 14 warps of a CTA (one CTA per SM, persistent over tiles of 256 channels):
+// Two kernels share this file: project_pair_kernel (default when P is staged; CTA pairs, described
+// above its definition) and project_tensor_kernel, the single-CTA ring kernel described here.
+//
+// Roles of the 14 warps of a ring-kernel CTA (one CTA per SM, persistent over tiles of 256 channels):
 //   warp 0      TMA producer: G tiles (and staged P tiles) into a shared-memory ring, 128-byte swizzle
 //   warp 1      MMA issuer (one thread) and owner of the 512 TMEM columns
 //   warps 2-9   staged P: L2 prefetch of the G lines the producer will ask for next;
