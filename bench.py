@@ -214,10 +214,24 @@ def run_ours(args, wl, rank, world, local_rank):
         barrier()
         s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         s2.record(stream)
-        for _ in range(e2e_steps):
-            for g, h in zip(Gs, host_G):
-                g.copy_(h, non_blocking=True)
-            opt.step(Ws, Gs, wl.lr, wl.wd, check=False)
+        # layer-wise, as the gradients would arrive during a backward pass: the copy of the next layer's
+        # gradients (copy stream) runs under the optimizer step of the current layer (apollo_step_range)
+        copy_stream = torch.cuda.Stream(device=dev)
+        layers = [(a, min(a + 7, n)) for a in range(0, n, 7)]
+        landed = [torch.cuda.Event() for _ in layers]
+        consumed = [torch.cuda.Event() for _ in layers]
+        for e2e_step in range(e2e_steps):
+            with torch.cuda.stream(copy_stream):
+                for k, (a, b) in enumerate(layers):
+                    if e2e_step > 0:
+                        copy_stream.wait_event(consumed[k])      # the previous step has read this layer's G
+                    for i in range(a, b):
+                        Gs[i].copy_(host_G[i], non_blocking=True)
+                    landed[k].record(copy_stream)
+            for k, (a, b) in enumerate(layers):
+                stream.wait_event(landed[k])
+                opt.step_range(a, Ws[a:b], Gs[a:b], wl.lr, wl.wd, close_step=(k == len(layers) - 1), stream=stream)
+                consumed[k].record(stream)
             for i in range(n):
                 B._check(opt.lib.apollo_get_limiter(opt.ctx, i, norms_dev[i].data_ptr(), stream.cuda_stream), "limiter")
             norms_host.copy_(norms_dev, non_blocking=True)
