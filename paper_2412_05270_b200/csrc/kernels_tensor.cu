@@ -648,11 +648,17 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
-    uint32_t it = 0, tile_iter = 0;   // k-block and tile counters of this role
+    // k-block and tile counters of this role; the stage index and phase of k-block `it` are kept
+    // incrementally (stage = it % ns, phase = (it / ns) & 1): the single-thread roles are bound by
+    // their own instruction count, and a division per k-block is a large part of it
+    uint32_t it = 0, tile_iter = 0, stage = 0, phase = 0;
+    auto next_stage = [&]() { ++it; if (++stage == (uint32_t)ns) { stage = 0; phase ^= 1; } };
 
     const int pair = blockIdx.x >> 1, pairs = gridDim.x >> 1;
+    int mat = find_matrix(prefix, n_mat, tile_begin + pair < tile_end ? tile_begin + pair : tile_begin);
     for (int tile = tile_begin + pair; tile < tile_end; tile += pairs, ++tile_iter) {
-        const int mat = find_matrix(prefix, n_mat, tile);
+        // the tiles of a CTA come in increasing order: the matrix index only moves forward
+        while (mat + 1 < n_mat && __ldg(prefix + mat + 1) <= tile) ++mat;
         const MatDesc* dp = descs + mat;
         const int tiles_k = __ldg(&dp->tiles_k);
         const int m = __ldg(&dp->m), n = __ldg(&dp->n);
@@ -671,8 +677,8 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                 ptx::fence_tensormap_acquire(tmap);
                 ptx::fence_tensormap_acquire(tmap_p);
                 const uint64_t pol_g = ptx::policy_evict_first(), pol_p = ptx::policy_evict_last();
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                    const uint32_t s = it % ns, ph = (it / ns) & 1;
+                for (int kb = 0; kb < num_kb; ++kb, next_stage()) {
+                    const uint32_t s = stage, ph = phase;
                     if (!wait_phase(bar_empty + 8 * s, ph ^ 1, abort_flag, status)) break;
                     const uint32_t g_s = smem_base + s * stage_bytes, p_s = g_s + P2_G_BYTES;
                     // the bytes of both CTAs are counted on the leader's barrier; the peer's may arrive
@@ -698,19 +704,21 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                 const uint32_t d_tmem = tmem_base + buf * (uint32_t)r_slice;
                 bool ok = wait_phase(bar_acc_empty + 8 * buf, (use & 1) ^ 1, abort_flag, status);   // epilogue of the tile before last
                 ptx::tc_fence_after_sync();
+                // descriptors of stage 0, k-step 0; the start-address field (bits 0..13, address >> 4) is the
+                // only one that moves, and shared-memory addresses stay below 2^18, so it never carries out
+                const uint64_t a_desc0 = tall ? ptx::smem_desc_sw128(smem_base, 16, 1024)
+                                              : ptx::smem_desc_sw128(smem_base, P2_G_BYTES / 2, 1024);
+                const uint64_t b_desc0 = ptx::smem_desc_sw128(smem_base + P2_G_BYTES, 16, 1024);
+                const uint32_t a_step = tall ? 32u >> 4 : 2048u >> 4, stage_step = stage_bytes >> 4;
                 int kb = 0;
-                for (; ok && kb < num_kb; ++kb, ++it) {
-                    const uint32_t s = it % ns, ph = (it / ns) & 1;
-                    if (!wait_phase(bar_full + 8 * s, ph, abort_flag, status)) break;
+                for (; ok && kb < num_kb; ++kb, next_stage()) {
+                    const uint32_t s = stage;
+                    if (!wait_phase(bar_full + 8 * s, phase, abort_flag, status)) break;
                     ptx::tc_fence_after_sync();
-                    const uint32_t g_s = smem_base + s * stage_bytes, p_s = g_s + P2_G_BYTES;
+                    const uint64_t a_desc = a_desc0 + s * stage_step, b_desc = b_desc0 + s * stage_step;
 #pragma unroll
-                    for (int kk = 0; kk < TC_BK / 16; ++kk) {
-                        const uint64_t a_desc = tall ? ptx::smem_desc_sw128(g_s + kk * 32, 16, 1024)
-                                                     : ptx::smem_desc_sw128(g_s + kk * 2048, P2_G_BYTES / 2, 1024);
-                        const uint64_t b_desc = ptx::smem_desc_sw128(p_s + kk * 32, 16, 1024);
-                        ptx::mma_bf16_pair(d_tmem, a_desc, b_desc, idesc, (kb | kk) != 0 ? 1u : 0u);
-                    }
+                    for (int kk = 0; kk < TC_BK / 16; ++kk)
+                        ptx::mma_bf16_pair(d_tmem, a_desc + kk * a_step, b_desc + kk * 2, idesc, (kb | kk) != 0 ? 1u : 0u);
                     ptx::mma_commit_pair(bar_done + 8 * s, 3);
                 }
                 if (ok && kb == num_kb) ptx::mma_commit_pair(bar_acc_full + 8 * buf, 3);
@@ -724,8 +732,8 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc[e] = 0.f;
             const int cc = t & 15, part = t >> 4;     // wide: 16 chunk columns x 8 row groups
-            for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                const uint32_t s = it % ns, ph = (it / ns) & 1;
+            for (int kb = 0; kb < num_kb; ++kb, next_stage()) {
+                const uint32_t s = stage, ph = phase;
                 if (!__all_sync(0xFFFFFFFFu, wait_phase(bar_done + 8 * s, ph, abort_flag, status))) break;   // landed, and the MMA has read it
                 const uint32_t g_s = smem_base + s * stage_bytes;
                 if (tr != 0) {
