@@ -588,7 +588,8 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
 // 128 channels and half of the rows of the P tile (so a k-block costs 32 KB of shared-memory fill per
 // CTA instead of 48 KB for the same work), and keeps r_slice accumulator columns per buffer, double
 // buffered: the epilogue of one tile runs under the main loop of the next.
-//   warp 0      producer: TMA loads of both CTAs count their bytes on the LEADER's `full` barrier
+//   warp 0      G producer, warp 2  P producer: the TMA loads of both CTAs count their bytes on the
+//               LEADER's `full` barrier of the stage
 //   warp 1      leader only: MMA issuer; its commits are multicast to both CTAs
 //   warps 4-7   squared column norms of this CTA's G tile, after the MMA that read it has finished
 //   warps 8-15  epilogue of this CTA's 128 channels
@@ -670,29 +671,42 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
         const uint32_t buf = tile_iter & 1, use = tile_iter >> 1;
 
         if (warp == 0) {
-            // ---------------- producer (one thread in each CTA) ----------------
+            // ---------------- G producer (one thread in each CTA) ----------------
             if (lane == 0) {
                 const void* tmap = dp->tmap;
-                const void* tmap_p = dp->tmap_p;
                 ptx::fence_tensormap_acquire(tmap);
-                ptx::fence_tensormap_acquire(tmap_p);
-                const uint64_t pol_g = ptx::policy_evict_first(), pol_p = ptx::policy_evict_last();
+                const uint64_t pol_g = ptx::policy_evict_first();
+                // the bytes of both CTAs are counted on the leader's barrier; the peer's may arrive
+                // there before the leader's expect_tx (the count is signed), never a phase early,
+                // because the peer's stage is only free once the leader's MMA has consumed it
+                const uint32_t full0 = ptx::map_to_cta(bar_full, 0);
                 for (int kb = 0; kb < num_kb; ++kb, next_stage()) {
-                    const uint32_t s = stage, ph = phase;
-                    if (!wait_phase(bar_empty + 8 * s, ph ^ 1, abort_flag, status)) break;
-                    const uint32_t g_s = smem_base + s * stage_bytes, p_s = g_s + P2_G_BYTES;
-                    // the bytes of both CTAs are counted on the leader's barrier; the peer's may arrive
-                    // there before the leader's expect_tx (the count is signed), never a phase early,
-                    // because the peer's stage is only free once the leader's MMA has consumed it
-                    const uint32_t full = ptx::map_to_cta(bar_full + 8 * s, 0);
-                    if (rank == 0) ptx::mbar_arrive_expect_tx(bar_full + 8 * s, 2u * stage_bytes);
+                    const uint32_t s = stage;
+                    if (!wait_phase(bar_empty + 8 * s, phase ^ 1, abort_flag, status)) break;
+                    const uint32_t g_s = smem_base + s * stage_bytes, full = full0 + 8 * s;
+                    if (rank == 0) ptx::mbar_arrive_expect_tx(bar_full + 8 * s, 2u * stage_bytes);   // G and P of both CTAs
                     if (tall) {
                         ptx::tma_load_2d_pair(g_s, tmap, kb * TC_BK, j0, full, pol_g);
                     } else {
                         ptx::tma_load_2d_pair(g_s, tmap, j0, kb * TC_BK, full, pol_g);
                         ptx::tma_load_2d_pair(g_s + P2_G_BYTES / 2, tmap, j0 + 64, kb * TC_BK, full, pol_g);
                     }
-                    ptx::tma_load_2d_pair(p_s, tmap_p, kb * TC_BK, r0 + (int)rank * r_half, full, pol_p);
+                }
+            }
+            __syncwarp();
+            if (__shfl_sync(0xFFFFFFFFu, *abort_flag, 0) != 0) break;
+        } else if (warp == 2) {
+            // ---------------- P producer (one thread in each CTA): this CTA's half of the rows, same stage, same barrier ----------------
+            if (lane == 0) {
+                const void* tmap_p = dp->tmap_p;
+                ptx::fence_tensormap_acquire(tmap_p);
+                const uint64_t pol_p = ptx::policy_evict_last();
+                const uint32_t full0 = ptx::map_to_cta(bar_full, 0);
+                const int p_row = r0 + (int)rank * r_half;
+                for (int kb = 0; kb < num_kb; ++kb, next_stage()) {
+                    const uint32_t s = stage;
+                    if (!wait_phase(bar_empty + 8 * s, phase ^ 1, abort_flag, status)) break;
+                    ptx::tma_load_2d_pair(smem_base + s * stage_bytes + P2_G_BYTES, tmap_p, kb * TC_BK, p_row, full0 + 8 * s, pol_p);
                 }
             }
             __syncwarp();
@@ -728,9 +742,11 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
         } else if (warp >= 4 && warp < 8) {
             // ---------------- squared column norms of this CTA's 128 channels ----------------
             const int t = tid - 128;
-            float acc[8];
+            // packed pairs of fp32 accumulators (fma.rn.f32x2).  wide: acc2[i] = channels 2i, 2i+1 of this
+            // thread's eight; tall: acc2[4 pass + i] = word i of the 16-byte chunks of row unit `pass`
+            uint64_t acc2[8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+            for (int e = 0; e < 8; ++e) acc2[e] = 0ull;
             const int cc = t & 15, part = t >> 4;     // wide: 16 chunk columns x 8 row groups
             for (int kb = 0; kb < num_kb; ++kb, next_stage()) {
                 const uint32_t s = stage, ph = phase;
@@ -745,7 +761,13 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                         const int u = t + pass * 128, row = u >> 1, half = u & 1;
                         const uint32_t base = g_s + row * 128 + half * 64;
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) acc[pass] += sum_sq_bf16x8(ld_shared_v4(base + (((i + row) & 3) << 4)));
+                        for (int i = 0; i < 4; ++i) {
+                            const uint4 v = ld_shared_v4(base + (((i + row) & 3) << 4));
+                            ptx::fma_sq_f32x2(acc2[4 * pass + 0], ptx::bf16x2_to_f32x2(v.x));
+                            ptx::fma_sq_f32x2(acc2[4 * pass + 1], ptx::bf16x2_to_f32x2(v.y));
+                            ptx::fma_sq_f32x2(acc2[4 * pass + 2], ptx::bf16x2_to_f32x2(v.z));
+                            ptx::fma_sq_f32x2(acc2[4 * pass + 3], ptx::bf16x2_to_f32x2(v.w));
+                        }
                     }
                 } else {
                     const uint32_t colbase = g_s + (cc >> 3) * (P2_G_BYTES / 2);
@@ -754,13 +776,10 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                     for (int i8 = 0; i8 < 8; ++i8) {
                         const int k = part + 8 * i8;
                         const uint4 v = ld_shared_v4(colbase + k * 128 + ((c ^ (k & 7)) << 4));
-                        const uint32_t w[4] = { v.x, v.y, v.z, v.w };
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
-                            acc[2 * i] = fmaf(lo, lo, acc[2 * i]);
-                            acc[2 * i + 1] = fmaf(hi, hi, acc[2 * i + 1]);
-                        }
+                        ptx::fma_sq_f32x2(acc2[0], ptx::bf16x2_to_f32x2(v.x));
+                        ptx::fma_sq_f32x2(acc2[1], ptx::bf16x2_to_f32x2(v.y));
+                        ptx::fma_sq_f32x2(acc2[2], ptx::bf16x2_to_f32x2(v.z));
+                        ptx::fma_sq_f32x2(acc2[3], ptx::bf16x2_to_f32x2(v.w));
                     }
                 }
                 __syncwarp();
@@ -773,12 +792,17 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                 // lanes 2k and 2k+1 hold the two halves of one stored row
 #pragma unroll
                 for (int pass = 0; pass < 2; ++pass) {
-                    const float v = acc[pass] + __shfl_xor_sync(0xFFFFFFFFu, acc[pass], 1);
+                    const float mine = (ptx::f32x2_sum(acc2[4 * pass]) + ptx::f32x2_sum(acc2[4 * pass + 1])) +
+                                       (ptx::f32x2_sum(acc2[4 * pass + 2]) + ptx::f32x2_sum(acc2[4 * pass + 3]));
+                    const float v = mine + __shfl_xor_sync(0xFFFFFFFFu, mine, 1);
                     const int j = j0 + ((t + pass * 128) >> 1);
                     if (!stop && tr == 0 && !(lane & 1) && j < n) g2out[j] = v;
                 }
             } else {
                 // lanes l and l + 16 hold two row groups of the same eight channels: one slice per warp
+                float acc[8];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) ptx::f32x2_unpack(acc2[i], acc[2 * i], acc[2 * i + 1]);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                     const float v = acc[e] + __shfl_xor_sync(0xFFFFFFFFu, acc[e], 16);
@@ -847,7 +871,7 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
         drain_phase(bar_drain, 0);
     }
     // the peer cannot watch the leader's barriers: after a wait gave up it lets its last loads land for 2 ms
-    if (rank == 1 && tid == 0 && *abort_flag)
+    if (rank == 1 && (tid == 0 || tid == 64) && *abort_flag)
         for (int i = 0; i < 2000; ++i) __nanosleep(1000);
     ptx::tc_fence_before_sync();
     __syncthreads();

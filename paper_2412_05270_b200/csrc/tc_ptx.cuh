@@ -245,6 +245,31 @@ __device__ __forceinline__ void prefetch_l2(const void* p)
     asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
 }
 
+// ---- packed fp32 pairs ----------------------------------------------------------------------
+// Two bf16 values of one 32-bit word as a pair of floats (low half first) in one 64-bit register.
+__device__ __forceinline__ uint64_t bf16x2_to_f32x2(uint32_t w)
+{
+    uint64_t r;
+    asm("{\n\t.reg .b32 lo, hi;\n\tshl.b32 lo, %1, 16;\n\tand.b32 hi, %1, 0xFFFF0000;\n\tmov.b64 %0, {lo, hi};\n\t}"
+        : "=l"(r) : "r"(w));
+    return r;
+}
+// acc += x * x on both halves with one instruction (two independent round-to-nearest fp32 FMAs).
+__device__ __forceinline__ void fma_sq_f32x2(uint64_t& acc, uint64_t x)
+{
+    asm("fma.rn.f32x2 %0, %1, %1, %0;" : "+l"(acc) : "l"(x));
+}
+__device__ __forceinline__ float f32x2_sum(uint64_t v)
+{
+    float lo, hi;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+    return lo + hi;
+}
+__device__ __forceinline__ void f32x2_unpack(uint64_t v, float& lo, float& hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+
 // ---- descriptors ----------------------------------------------------------------------------
 // Shared-memory matrix descriptor, 128-byte swizzle, tile base 1024-byte aligned.
 //   bits  0..13  start address >> 4        bits 16..29  leading-dimension byte offset >> 4
