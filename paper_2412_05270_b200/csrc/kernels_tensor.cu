@@ -293,7 +293,10 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
-    uint32_t it = 0;          // k-block counter across tiles: stage = it % stages, phase = (it / stages) & 1
+    // k-block counter across tiles; its stage (it % stages) and phase ((it / stages) & 1) are kept
+    // incrementally: a division per k-block is a large part of a single-thread role's instructions
+    uint32_t it = 0, stage = 0, phase = 0;
+    auto next_stage = [&]() { ++it; if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1; } };
     uint32_t tile_iter = 0;   // tiles done by this CTA: phase of the accumulator barrier
 
     for (int tile = tile_begin + blockIdx.x; tile < tile_end; tile += gridDim.x, ++tile_iter) {
@@ -324,8 +327,8 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                 if (staged) ptx::fence_tensormap_acquire(tmap_p);
                 // G is read once in this pass, every CTA of a matrix reads the same P: tell L2 which to keep
                 const uint64_t pol_g = ptx::policy_evict_first(), pol_p = ptx::policy_evict_last();
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                    const uint32_t s = it % stages, ph = (it / stages) & 1;
+                for (int kb = 0; kb < num_kb; ++kb, next_stage()) {
+                    const uint32_t s = stage, ph = phase;
                     if (!wait_phase(bar_empty + 8 * s, ph ^ 1, abort_flag, status)) break;
                     const uint32_t g_s = smem_base + s * stage_bytes;
                     ptx::mbar_arrive_expect_tx(bar_g_full + 8 * s,
@@ -347,8 +350,8 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
             if (lane == 0) {
                 const uint32_t idesc = ptx::instr_desc_bf16((uint32_t)r_slice, !tall);
                 int kb = 0;
-                for (; kb < num_kb; ++kb, ++it) {
-                    const uint32_t s = it % stages, ph = (it / stages) & 1;
+                for (; kb < num_kb; ++kb, next_stage()) {
+                    const uint32_t s = stage, ph = phase;
                     if (!wait_phase(bar_g_full + 8 * s, ph, abort_flag, status)) break;
                     if (!staged && !wait_phase(bar_p_full + 8 * s, ph, abort_flag, status)) break;
                     ptx::tc_fence_after_sync();
@@ -418,8 +421,8 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                         __nanosleep(100);
                 }
             }
-            for (int kb = 0; kb < num_kb && !staged; ++kb, ++it) {
-                const uint32_t s = it % stages, ph = (it / stages) & 1;
+            for (int kb = 0; kb < num_kb && !staged; ++kb, next_stage()) {
+                const uint32_t s = stage, ph = phase;
                 if (!__all_sync(0xFFFFFFFFu, wait_phase(bar_empty + 8 * s, ph ^ 1, abort_flag, status))) break;
                 const uint32_t p_s = smem_base + s * stage_bytes + p_off;
                 // two rows per pass (32 rows apart) so that four Philox chains are in flight per thread
@@ -456,8 +459,8 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
             const int parts = TC_NORM_THREADS / ccols;   // wide: threads sharing one chunk column
             const int cc = t % ccols, part = t / ccols;
             const int rows_pp = TC_BK / parts;
-            for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                const uint32_t s = it % stages, ph = (it / stages) & 1;
+            for (int kb = 0; kb < num_kb; ++kb, next_stage()) {
+                const uint32_t s = stage, ph = phase;
                 if (!__all_sync(0xFFFFFFFFu, wait_phase(bar_g_full + 8 * s, ph, abort_flag, status))) break;   // the warp stays together
                 const uint32_t g_s = smem_base + s * stage_bytes;
                 if (tall) {
