@@ -200,6 +200,7 @@ namespace {
 // caller stops issuing work and falls through to the barriers and the drain at the end of the kernel.
 __device__ __forceinline__ bool wait_phase(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status)
 {
+    if (ptx::mbar_try_wait(bar, parity)) return true;      // the common case costs one poll and no flag read
     if (*abort_flag) return false;
     for (uint32_t i = 0; i < TC_WAIT_CAP; ++i)
         if (ptx::mbar_try_wait(bar, parity)) return true;
