@@ -83,7 +83,7 @@ class ClockSampler:
     def __enter__(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "50",
                  "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -93,7 +93,7 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([x.strip() for x in line.split(",")])
+            self.rows.append((time.monotonic(), [x.strip() for x in line.split(",")]))
 
     def __exit__(self, *a):
         if self.proc:
@@ -103,10 +103,18 @@ class ClockSampler:
             except Exception:
                 self.proc.kill()
 
-    def summary(self):
+    def summary(self, t0=None, t1=None):
+        """Median SM clock and the throttle reasons seen between host times t0 and t1 (the timed region).
+        nvidia-smi needs 0.1-0.2 s to deliver its first sample, so the sampler is started before the
+        warm-up; if the region was too short to catch a sample, the samples since the start are used
+        and "window" says so."""
+        inside = [r for t, r in self.rows if t0 is None or (t0 <= t <= t1)]
+        window = "timed region"
+        if not inside:
+            inside, window = [r for _, r in self.rows], "warm-up and timed region"
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for r in inside:
             try:
                 sm.append(float(r[0])); mx.append(float(r[1]))
             except (ValueError, IndexError):
@@ -116,7 +124,7 @@ class ClockSampler:
                     reasons.add(name)
         sm.sort()
         return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "window": window}
 
 
 def cpu_baseline(wl: WL.Workload, budget_s: float = 12.0):
@@ -184,11 +192,12 @@ def run_ours(args, wl, rank, world, local_rank):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
-        opt.step(Ws, Gs, wl.lr, wl.wd, check=False)
-    barrier()
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with ClockSampler(local_rank) as clocks:
+        for _ in range(args.warmup):
+            opt.step(Ws, Gs, wl.lr, wl.wd, check=False)
+        barrier()
+        t_region0 = time.monotonic()
         start.record(stream)
         launches = 0
         for _ in range(args.steps):
@@ -196,6 +205,7 @@ def run_ours(args, wl, rank, world, local_rank):
             launches += opt.last_launches()      # P is regenerated only in steps that open an epoch
         stop.record(stream)
         barrier()
+        t_region1 = time.monotonic()
     ms_total = start.elapsed_time(stop)
     assert opt.status() == B.OK
     phases = [opt.timing(k) for k in range(min(args.steps, 64))]
@@ -270,7 +280,7 @@ def run_ours(args, wl, rank, world, local_rank):
                           "t_roofline_ms": 1e3 * t_roof, "frac": 1e3 * t_roof / ms_step,
                           "frac_vs_8TBs": 1e3 * max(two_pass / 8e12, flops / tc) / ms_step,
                           "phase_ms": {"projection": proj_ms, "finalize": fin_ms, "update": upd_ms}},
-        "clocks": clocks.summary(),
+        "clocks": clocks.summary(t_region0, t_region1),
         "gpu_launches": launches,
     }
     if not args.no_e2e:

@@ -60,9 +60,11 @@ __device__ __forceinline__ void fence_proxy_async_smem()
 {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
+// A tensor map that lives in global memory and was written by a host copy: the thread that is going to
+// use it makes that copy visible to the tensor-map proxy first (system scope, once per thread and map).
 __device__ __forceinline__ void fence_tensormap_acquire(const void* tmap)
 {
-    asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(tmap) : "memory");
+    asm volatile("fence.proxy.tensormap::generic.acquire.sys [%0], 128;" ::"l"(tmap) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before_sync()
 {
