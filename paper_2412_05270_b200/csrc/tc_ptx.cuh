@@ -1,5 +1,5 @@
 // Thin inline-PTX wrappers for the sm_100a features the tensor-core projection uses:
-// mbarrier, TMA tiled loads (no multicast), tcgen05 MMA / commit / TMEM allocation and loads,
+// mbarrier, TMA tiled loads (each into the shared memory of the CTA that issues it), tcgen05 MMA / commit / TMEM allocation and loads,
 // proxy fences.  Every wait is bounded by the caller.
 #pragma once
 #include <cuda_runtime.h>
@@ -180,7 +180,7 @@ __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr)
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // 2D tile load of a CTA pair: the data lands in this CTA's shared memory, the bytes are counted on
-// the mbarrier at `bar_cluster_addr`, which may belong to either CTA of the pair (no multicast).
+// the mbarrier at `bar_cluster_addr`, which may belong to either CTA of the pair.
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const void* tmap, int32_t x, int32_t y,
                                                  uint32_t bar_cluster_addr, uint64_t policy)
 {
