@@ -91,7 +91,7 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
             p.g2_slices = 1;
         }
         p.proj_tiles = (int64_t)p.tiles_n * p.tiles_k;
-        p.update_tiles = (rows * cols + UPDATE_TILE - 1) / UPDATE_TILE;
+        p.update_tiles = update_tile_count(rows, cols);
         plan.tiles[p.path] += p.proj_tiles;
         plan.tiles[3] += p.update_tiles;
     }

@@ -19,6 +19,22 @@ constexpr int SIMT_BN = 64;          // channels per CUDA-core tile
 constexpr int SIMT_BR = 64;          // rows of R per CUDA-core tile
 constexpr int SIMT_BK = 32;          // contraction chunk of the CUDA-core tile
 constexpr int UPDATE_TILE = 16384;   // elements one tile of the update pass covers
+// Matrices whose rows are whole 8-element vectors are updated in 2-D tiles of UPDATE_ROWS rows x one
+// column chunk (at most UPDATE_COLS columns: eight per thread), so a thread keeps its column scales in
+// registers and no index arithmetic is left per vector; the others go through flat tiles of UPDATE_TILE.
+constexpr int UPDATE_ROWS = 8;
+constexpr int UPDATE_COLS = 2048;
+__host__ __device__ inline int update_chunks(int cols) { return (cols + UPDATE_COLS - 1) / UPDATE_COLS; }
+__host__ __device__ inline int update_chunk_width(int cols)
+{
+    const int c = update_chunks(cols);
+    return ((cols + c - 1) / c + 7) & ~7;          // equal chunks, whole vectors
+}
+__host__ __device__ inline long long update_tile_count(long long rows, long long cols)
+{
+    return cols % 8 == 0 ? (rows + UPDATE_ROWS - 1) / UPDATE_ROWS * update_chunks((int)cols)
+                         : (rows * cols + UPDATE_TILE - 1) / UPDATE_TILE;
+}
 
 // Per-matrix record in device memory.  Pointers into the workspace are fixed at create
 // time; W, G and dW are refreshed whenever the caller passes different addresses.

@@ -463,6 +463,65 @@ update_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix,
         const float decay = sp.lr * sp.wd;
         const bool tall = d.tall != 0;
 
+        if ((cols & 7u) == 0) {
+            // 2-D tile: UPDATE_ROWS rows x one column chunk; this thread owns eight columns of it
+            const int chunks = update_chunks((int)cols), cw = update_chunk_width((int)cols);
+            const int rb = local / chunks, ct = local - rb * chunks;
+            const uint32_t c = (uint32_t)ct * (uint32_t)cw + threadIdx.x * 8u;
+            if (threadIdx.x * 8u >= (uint32_t)cw || c >= cols) continue;
+            const int r0 = rb * UPDATE_ROWS, nr = min(UPDATE_ROWS, d.rows - r0);
+            float sa[8];                               // step x scale of this thread's columns (wide)
+            if (!tall) {
+                const float4 s0 = __ldg(reinterpret_cast<const float4*>(s + c));
+                const float4 s1 = __ldg(reinterpret_cast<const float4*>(s + c + 4));
+                sa[0] = step * s0.x; sa[1] = step * s0.y; sa[2] = step * s0.z; sa[3] = step * s0.w;
+                sa[4] = step * s1.x; sa[5] = step * s1.y; sa[6] = step * s1.z; sa[7] = step * s1.w;
+            }
+            const int64_t base = (int64_t)r0 * cols + c;
+            auto finish = [&](int r, const float (&g)[8], const float (&w)[8]) {
+                const int64_t e = base + (int64_t)r * cols;
+                float dw[8], wn[8];
+                if (tall) {
+                    const float sv = step * __ldg(s + r0 + r);
+#pragma unroll
+                    for (int x = 0; x < 8; ++x) dw[x] = -__fmaf_rn(sv, g[x], __fmul_rn(decay, w[x]));
+                } else {
+#pragma unroll
+                    for (int x = 0; x < 8; ++x) dw[x] = -__fmaf_rn(sa[x], g[x], __fmul_rn(decay, w[x]));
+                }
+#pragma unroll
+                for (int x = 0; x < 8; ++x) wn[x] = __fadd_rn(w[x], dw[x]);
+                store8(W + e, wn);
+                if (d.dW) store8(d.dW + e, dw);
+            };
+            if (nr == UPDATE_ROWS) {
+                // whole tile: the loads of four rows are issued before the first use
+#pragma unroll
+                for (int rq = 0; rq < UPDATE_ROWS; rq += 4) {
+                    Raw8<T> gr[4], wr[4];
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        gr[v] = load_raw8_stream(G + base + (int64_t)(rq + v) * cols);
+                        wr[v] = load_raw8_stream(W + base + (int64_t)(rq + v) * cols);
+                    }
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        float g[8], w[8];
+                        unpack_raw8(gr[v], g); unpack_raw8(wr[v], w);
+                        finish(rq + v, g, w);
+                    }
+                }
+            } else {
+                for (int r = 0; r < nr; ++r) {
+                    float g[8], w[8];
+                    load8_aligned(G + base + (int64_t)r * cols, g);
+                    load8_aligned(W + base + (int64_t)r * cols, w);
+                    finish(r, g, w);
+                }
+            }
+            continue;
+        }
+
         constexpr int VECS = UPDATE_TILE / (UPDATE_THREADS * 8);   // vectors per thread per tile
         constexpr int BATCH = 4;                                   // vectors whose loads are issued together
         if (e0 + UPDATE_TILE <= total) {
