@@ -68,7 +68,7 @@ def whole_job_value(params_per_rank: int, world: int, ms_per_step: float) -> flo
 
 # DRAM bytes per parameter of update_kernel<bf16> from its ncu capture (profiles/update_kernel_*.md);
 # set to None when the kernel changes until the counters are taken again.
-UPDATE_TRAFFIC_BYTES_PER_PARAM = 5.88
+UPDATE_TRAFFIC_BYTES_PER_PARAM = 5.89
 
 
 class ClockSampler:
