@@ -279,6 +279,12 @@ int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_ma
         d.m_pad = (p.m + 63) / 64 * 64;
         d.gpad = p.gpad_bytes ? ctx->ws + p.off_gpad : nullptr;
         d.g_pitch = p.gpad_bytes ? (p.cols + 7) / 8 * 8 : p.cols;
+        if (p.cols % 8 == 0) {
+            const UpdateTiling ut = update_tiling(p.cols);
+            d.upd_chunks = ut.chunks; d.upd_width = ut.width; d.upd_groups = ut.groups;
+        } else {
+            d.upd_chunks = 0; d.upd_width = 0; d.upd_groups = 0;
+        }
         d.ext_p = nullptr;
         d.r_scale = (float)(1.0 / std::sqrt((double)cfg->rank));
         d.rows = p.rows; d.cols = p.cols; d.m = p.m; d.n = p.n; d.tall = p.tall; d.path = p.path;

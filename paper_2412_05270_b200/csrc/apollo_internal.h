@@ -19,21 +19,38 @@ constexpr int SIMT_BN = 64;          // channels per CUDA-core tile
 constexpr int SIMT_BR = 64;          // rows of R per CUDA-core tile
 constexpr int SIMT_BK = 32;          // contraction chunk of the CUDA-core tile
 constexpr int UPDATE_TILE = 16384;   // elements one tile of the update pass covers
-// Matrices whose rows are whole 8-element vectors are updated in 2-D tiles of UPDATE_ROWS rows x one
-// column chunk (at most UPDATE_COLS columns: eight per thread), so a thread keeps its column scales in
-// registers and no index arithmetic is left per vector; the others go through flat tiles of UPDATE_TILE.
+// Matrices whose rows are whole 8-element vectors are updated in 2-D tiles: the columns are cut into
+// equal chunks of at most UPDATE_COLS, a thread owns eight columns of a chunk (so it keeps its column
+// scales in registers and no index arithmetic is left per vector), and when a chunk needs fewer than
+// all the threads, several groups of UPDATE_ROWS rows are worked on side by side.  The other matrices
+// go through flat tiles of UPDATE_TILE elements.
 constexpr int UPDATE_ROWS = 8;
 constexpr int UPDATE_COLS = 2048;
-__host__ __device__ inline int update_chunks(int cols) { return (cols + UPDATE_COLS - 1) / UPDATE_COLS; }
-__host__ __device__ inline int update_chunk_width(int cols)
+constexpr int UPDATE_BLOCK = 256;      // threads of an update block
+struct UpdateTiling {
+    int chunks;       // column chunks
+    int width;        // columns of a chunk (multiple of 8; the last chunk may be narrower)
+    int groups;       // row groups side by side in one tile
+};
+// Among the smallest chunk counts, the one that keeps most threads busy.
+inline UpdateTiling update_tiling(int cols)
 {
-    const int c = update_chunks(cols);
-    return ((cols + c - 1) / c + 7) & ~7;          // equal chunks, whole vectors
+    UpdateTiling best{1, 8, 1};
+    int best_busy = -1;
+    const int cmin = (cols + UPDATE_COLS - 1) / UPDATE_COLS;
+    for (int c = cmin; c < cmin + 4; ++c) {
+        const int width = ((cols + c - 1) / c + 7) & ~7;
+        const int tpr = width / 8, groups = UPDATE_BLOCK / tpr, busy = tpr * groups;
+        if (busy > best_busy) { best_busy = busy; best = UpdateTiling{c, width, groups}; }
+    }
+    return best;
 }
-__host__ __device__ inline long long update_tile_count(long long rows, long long cols)
+inline long long update_tile_count(long long rows, long long cols)
 {
-    return cols % 8 == 0 ? (rows + UPDATE_ROWS - 1) / UPDATE_ROWS * update_chunks((int)cols)
-                         : (rows * cols + UPDATE_TILE - 1) / UPDATE_TILE;
+    if (cols % 8 != 0) return (rows * cols + UPDATE_TILE - 1) / UPDATE_TILE;
+    const UpdateTiling t = update_tiling((int)cols);
+    const long long tile_rows = (long long)UPDATE_ROWS * t.groups;
+    return (rows + tile_rows - 1) / tile_rows * t.chunks;
 }
 
 // Per-matrix record in device memory.  Pointers into the workspace are fixed at create
@@ -65,6 +82,7 @@ struct MatDesc {
     int32_t tiles_k;  // projection tiles along the other tiled axis (rows of G, or rows of R)
     int32_t m_pad;    // m rounded up to 64: row length of the staged P
     int32_t g_pitch;  // row pitch (elements) of the array the tensor path reads: cols, or cols rounded up to 8
+    int32_t upd_chunks, upd_width, upd_groups;   // 2-D tiling of the update pass (update_tiling(cols)); 0 chunks: flat tiles
     float r_scale;    // factor applied to the contraction: 1/sqrt(r) for generated standard normals, 1 for a supplied P
 };
 

@@ -88,6 +88,10 @@ extern "C" int apollo_mini_step_static(void* d_W, const void* d_G, int64_t rows,
     }
     const int64_t proj_tiles = (int64_t)d.tiles_n * d.tiles_k;
     const int64_t update_tiles = update_tile_count(rows, cols);
+    if (cols % 8 == 0) {
+        const UpdateTiling ut = update_tiling((int)cols);
+        d.upd_chunks = ut.chunks; d.upd_width = ut.width; d.upd_groups = ut.groups;
+    }
     const size_t bytes_s = align256(sizeof(float) * (size_t)d.n);
     const size_t bytes_part = align256(sizeof(float) * 2 * (size_t)d.slices * (size_t)d.n);
     if (OFF_ARRAYS + bytes_s + bytes_part > (size_t)APOLLO_STATIC_SCRATCH_BYTES || proj_tiles > INT32_MAX ||

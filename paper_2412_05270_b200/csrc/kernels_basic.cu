@@ -425,7 +425,7 @@ finalize_kernel(const MatDesc* __restrict__ descs, int first, StepParams sp)
 // pass over the flat rows*cols array in 16-byte vectors.  The scale index is the column
 // (wide) or the stored row (tall).
 // ----------------------------------------------------------------------------------------
-constexpr int UPDATE_THREADS = 256;
+constexpr int UPDATE_THREADS = UPDATE_BLOCK;
 
 __device__ __forceinline__ void store8(float* p, const float (&v)[8])
 {
@@ -463,13 +463,16 @@ update_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix,
         const float decay = sp.lr * sp.wd;
         const bool tall = d.tall != 0;
 
-        if ((cols & 7u) == 0) {
-            // 2-D tile: UPDATE_ROWS rows x one column chunk; this thread owns eight columns of it
-            const int chunks = update_chunks((int)cols), cw = update_chunk_width((int)cols);
+        if (d.upd_chunks > 0) {
+            // 2-D tile: `groups` groups of UPDATE_ROWS rows x one column chunk; this thread owns eight
+            // columns of the chunk in one of the groups
+            const int chunks = d.upd_chunks, cw = d.upd_width, tpr = cw >> 3;
             const int rb = local / chunks, ct = local - rb * chunks;
-            const uint32_t c = (uint32_t)ct * (uint32_t)cw + threadIdx.x * 8u;
-            if (threadIdx.x * 8u >= (uint32_t)cw || c >= cols) continue;
-            const int r0 = rb * UPDATE_ROWS, nr = min(UPDATE_ROWS, d.rows - r0);
+            const int grp = threadIdx.x / tpr, lt = threadIdx.x - grp * tpr;
+            const uint32_t c = (uint32_t)ct * (uint32_t)cw + (uint32_t)lt * 8u;
+            const int r0 = (rb * d.upd_groups + grp) * UPDATE_ROWS;
+            if (grp >= d.upd_groups || c >= cols || r0 >= d.rows) continue;
+            const int nr = min(UPDATE_ROWS, d.rows - r0);
             float sa[8];                               // step x scale of this thread's columns (wide)
             if (!tall) {
                 const float4 s0 = __ldg(reinterpret_cast<const float4*>(s + c));
