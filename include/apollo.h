@@ -105,6 +105,15 @@ APOLLO_API int apollo_workspace_bytes(const apollo_shape* shapes, int32_t n_matr
  * stream: the moments are zeroed (Appendix: "zero initialization") by the first
  * apollo_step on that step's stream.  The matrix index in the list is the `matrix index`
  * word of the Philox counter.  Must be called with the target device current.
+ *
+ * Environment switches of the tensor-core projection, read here and at every step (keep them
+ * unchanged for the life of a context); none of them changes the results beyond the order of
+ * floating-point sums:
+ *   APOLLO_TC_KERNEL=ring    the single-CTA kernel instead of the CTA-pair kernel
+ *   APOLLO_P_STAGING=0       generate the projection inside the kernel instead of staging it
+ *   APOLLO_P_STAGING_MB=n    staging budget in MB (default 512); below the size of all projections
+ *                            the slots are shared and every step refills them
+ *   APOLLO_TC_RSLICE, APOLLO_TC_NBLK   tile shape (rows of R per tile; 128-channel blocks, ring kernel)
  */
 APOLLO_API int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_matrices,
                   const apollo_config* cfg, void* d_workspace, size_t workspace_bytes);
