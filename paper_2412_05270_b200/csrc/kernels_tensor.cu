@@ -209,6 +209,21 @@ __device__ __forceinline__ bool wait_phase(uint32_t bar, uint32_t parity, volati
     return false;
 }
 
+// The same for waits that have slack (an epilogue waiting for its accumulator): sleeps between polls,
+// which costs nothing there and saves issue slots, i.e. power, on a board that runs at its power cap.
+__device__ __forceinline__ bool wait_phase_idle(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status)
+{
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    for (uint32_t i = 0; i < TC_WAIT_CAP; ++i) {
+        __nanosleep(200);
+        if (ptx::mbar_try_wait(bar, parity)) return true;
+    }
+    *abort_flag = 1;
+    atomicExch(status, STATUS_TIMEOUT);
+    return false;
+}
+
 // Bounded wait that neither reads nor sets the abort flag: lets copies and MMAs that are already in
 // flight finish before the CTA gives up its shared memory and TMEM.
 __device__ __forceinline__ void drain_phase(uint32_t bar, uint32_t parity)
@@ -822,7 +837,7 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             float* const Mbase = dp->M;
             float* const Vbase = dp->V;
             const float r_scale = __ldg(&dp->r_scale);
-            const bool acc_ok = __all_sync(0xFFFFFFFFu, wait_phase(bar_acc_full + 8 * buf, use & 1, abort_flag, status));   // tcgen05.ld needs the whole warp
+            const bool acc_ok = __all_sync(0xFFFFFFFFu, wait_phase_idle(bar_acc_full + 8 * buf, use & 1, abort_flag, status));   // tcgen05.ld needs the whole warp
             ptx::tc_fence_after_sync();
             float num = 0.f, den = 0.f;
             const int chunks = acc_ok ? r_slice / 16 : 0;
