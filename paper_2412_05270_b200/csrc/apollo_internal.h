@@ -24,7 +24,7 @@ constexpr int UPDATE_TILE = 16384;   // elements one tile of the update pass cov
 // scales in registers and no index arithmetic is left per vector), and when a chunk needs fewer than
 // all the threads, several groups of UPDATE_ROWS rows are worked on side by side.  The other matrices
 // go through flat tiles of UPDATE_TILE elements.
-constexpr int UPDATE_ROWS = 8;
+constexpr int UPDATE_ROWS = 16;
 constexpr int UPDATE_COLS = 2048;
 constexpr int UPDATE_BLOCK = 256;      // threads of an update block
 struct UpdateTiling {

@@ -481,6 +481,7 @@ update_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix,
                 sa[4] = step * s1.x; sa[5] = step * s1.y; sa[6] = step * s1.z; sa[7] = step * s1.w;
             }
             const int64_t base = (int64_t)r0 * cols + c;
+            float* const dWp = d.dW;
             auto finish = [&](int r, const float (&g)[8], const float (&w)[8]) {
                 const int64_t e = base + (int64_t)r * cols;
                 float dw[8], wn[8];
@@ -495,7 +496,7 @@ update_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix,
 #pragma unroll
                 for (int x = 0; x < 8; ++x) wn[x] = __fadd_rn(w[x], dw[x]);
                 store8(W + e, wn);
-                if (d.dW) store8(d.dW + e, dw);
+                if (dWp) store8(dWp + e, dw);
             };
             if (nr == UPDATE_ROWS) {
                 // whole tile: the loads of four rows are issued before the first use
