@@ -91,7 +91,7 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
             p.g2_slices = 1;
         }
         p.proj_tiles = (int64_t)p.tiles_n * p.tiles_k;
-        p.update_tiles = update_tile_count(rows, cols);
+        p.update_tiles = update_tile_count(rows, cols, p.tall != 0);
         plan.tiles[p.path] += p.proj_tiles;
         plan.tiles[3] += p.update_tiles;
     }
@@ -279,8 +279,9 @@ int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_ma
         d.m_pad = (p.m + 63) / 64 * 64;
         d.gpad = p.gpad_bytes ? ctx->ws + p.off_gpad : nullptr;
         d.g_pitch = p.gpad_bytes ? (p.cols + 7) / 8 * 8 : p.cols;
-        if (p.cols % 8 == 0) {
-            const UpdateTiling ut = update_tiling(p.cols);
+        d.upd_super = update_super_rows(p.rows, p.cols, p.tall != 0) ? 1 : 0;
+        if (p.cols % 8 == 0 || d.upd_super) {
+            const UpdateTiling ut = update_tiling(d.upd_super ? 8 * p.cols : p.cols);
             d.upd_chunks = ut.chunks; d.upd_width = ut.width; d.upd_groups = ut.groups;
         } else {
             d.upd_chunks = 0; d.upd_width = 0; d.upd_groups = 0;

@@ -23,7 +23,7 @@ constexpr int UPDATE_TILE = 16384;   // elements one tile of the update pass cov
 // equal chunks of at most UPDATE_COLS, a thread owns eight columns of a chunk (so it keeps its column
 // scales in registers and no index arithmetic is left per vector), and when a chunk needs fewer than
 // all the threads, several groups of UPDATE_ROWS rows are worked on side by side.  The other matrices
-// go through flat tiles of UPDATE_TILE elements.
+// go through flat tiles of UPDATE_TILE elements, or through the same 2-D tiles over super-rows (below).
 constexpr int UPDATE_ROWS = 16;
 constexpr int UPDATE_COLS = 2048;
 constexpr int UPDATE_BLOCK = 256;      // threads of an update block
@@ -45,8 +45,16 @@ inline UpdateTiling update_tiling(int cols)
     }
     return best;
 }
-inline long long update_tile_count(long long rows, long long cols)
+// A wide matrix whose rows are not whole vectors but whose row count is a multiple of 8 is tiled the
+// same way over "super-rows" of 8 stored rows: 8 * cols elements are whole vectors, every super-row
+// starts on a 16-byte boundary, and element c of a super-row belongs to column c mod cols in all of them.
+inline bool update_super_rows(long long rows, long long cols, bool tall)
 {
+    return cols % 8 != 0 && !tall && rows % 8 == 0 && cols <= (1ll << 27);
+}
+inline long long update_tile_count(long long rows, long long cols, bool tall)
+{
+    if (update_super_rows(rows, cols, tall)) { rows /= 8; cols *= 8; }
     if (cols % 8 != 0) return (rows * cols + UPDATE_TILE - 1) / UPDATE_TILE;
     const UpdateTiling t = update_tiling((int)cols);
     const long long tile_rows = (long long)UPDATE_ROWS * t.groups;
@@ -83,6 +91,7 @@ struct MatDesc {
     int32_t m_pad;    // m rounded up to 64: row length of the staged P
     int32_t g_pitch;  // row pitch (elements) of the array the tensor path reads: cols, or cols rounded up to 8
     int32_t upd_chunks, upd_width, upd_groups;   // 2-D tiling of the update pass (update_tiling(cols)); 0 chunks: flat tiles
+    int32_t upd_super;   // 1: the 2-D tiles run over super-rows of 8 stored rows (update_super_rows)
     float r_scale;    // factor applied to the contraction: 1/sqrt(r) for generated standard normals, 1 for a supplied P
 };
 

@@ -87,9 +87,10 @@ extern "C" int apollo_mini_step_static(void* d_W, const void* d_G, int64_t rows,
         d.slices = 1;
     }
     const int64_t proj_tiles = (int64_t)d.tiles_n * d.tiles_k;
-    const int64_t update_tiles = update_tile_count(rows, cols);
-    if (cols % 8 == 0) {
-        const UpdateTiling ut = update_tiling((int)cols);
+    const int64_t update_tiles = update_tile_count(rows, cols, d.tall != 0);
+    d.upd_super = update_super_rows(rows, cols, d.tall != 0) ? 1 : 0;
+    if (cols % 8 == 0 || d.upd_super) {
+        const UpdateTiling ut = update_tiling((int)(d.upd_super ? 8 * cols : cols));
         d.upd_chunks = ut.chunks; d.upd_width = ut.width; d.upd_groups = ut.groups;
     }
     const size_t bytes_s = align256(sizeof(float) * (size_t)d.n);

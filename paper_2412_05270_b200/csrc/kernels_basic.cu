@@ -467,23 +467,31 @@ update_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix,
             // 2-D tile: `groups` groups of UPDATE_ROWS rows x one column chunk; this thread owns eight
             // columns of the chunk in one of the groups
             const int chunks = d.upd_chunks, cw = d.upd_width, tpr = cw >> 3;
+            // over super-rows of 8 stored rows when the stored rows are not whole vectors
+            const bool sup = d.upd_super != 0;
+            const uint32_t ecols = sup ? cols * 8u : cols;
+            const int erows = sup ? d.rows >> 3 : d.rows;
             const int rb = local / chunks, ct = local - rb * chunks;
             const int grp = threadIdx.x / tpr, lt = threadIdx.x - grp * tpr;
             const uint32_t c = (uint32_t)ct * (uint32_t)cw + (uint32_t)lt * 8u;
             const int r0 = (rb * d.upd_groups + grp) * UPDATE_ROWS;
-            if (grp >= d.upd_groups || c >= cols || r0 >= d.rows) continue;
-            const int nr = min(UPDATE_ROWS, d.rows - r0);
+            if (grp >= d.upd_groups || c >= ecols || r0 >= erows) continue;
+            const int nr = min(UPDATE_ROWS, erows - r0);
             float sa[8];                               // step x scale of this thread's columns (wide)
-            if (!tall) {
+            if (sup) {
+                uint32_t col = c % cols;               // the same in every super-row
+#pragma unroll
+                for (int x = 0; x < 8; ++x) { sa[x] = step * __ldg(s + col); if (++col == cols) col = 0; }
+            } else if (!tall) {
                 const float4 s0 = __ldg(reinterpret_cast<const float4*>(s + c));
                 const float4 s1 = __ldg(reinterpret_cast<const float4*>(s + c + 4));
                 sa[0] = step * s0.x; sa[1] = step * s0.y; sa[2] = step * s0.z; sa[3] = step * s0.w;
                 sa[4] = step * s1.x; sa[5] = step * s1.y; sa[6] = step * s1.z; sa[7] = step * s1.w;
             }
-            const int64_t base = (int64_t)r0 * cols + c;
+            const int64_t base = (int64_t)r0 * ecols + c;
             float* const dWp = d.dW;
             auto finish = [&](int r, const float (&g)[8], const float (&w)[8]) {
-                const int64_t e = base + (int64_t)r * cols;
+                const int64_t e = base + (int64_t)r * ecols;
                 float dw[8], wn[8];
                 if (tall) {
                     const float sv = step * __ldg(s + r0 + r);
@@ -505,8 +513,8 @@ update_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix,
                     Raw8<T> gr[4], wr[4];
 #pragma unroll
                     for (int v = 0; v < 4; ++v) {
-                        gr[v] = load_raw8_stream(G + base + (int64_t)(rq + v) * cols);
-                        wr[v] = load_raw8_stream(W + base + (int64_t)(rq + v) * cols);
+                        gr[v] = load_raw8_stream(G + base + (int64_t)(rq + v) * ecols);
+                        wr[v] = load_raw8_stream(W + base + (int64_t)(rq + v) * ecols);
                     }
 #pragma unroll
                     for (int v = 0; v < 4; ++v) {
@@ -518,8 +526,8 @@ update_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix,
             } else {
                 for (int r = 0; r < nr; ++r) {
                     float g[8], w[8];
-                    load8_aligned(G + base + (int64_t)r * cols, g);
-                    load8_aligned(W + base + (int64_t)r * cols, w);
+                    load8_aligned(G + base + (int64_t)r * ecols, g);
+                    load8_aligned(W + base + (int64_t)r * ecols, w);
                     finish(r, g, w);
                 }
             }

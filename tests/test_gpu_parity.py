@@ -34,6 +34,14 @@ def test_cuda_core_path_small_shapes(dtype, rank, mode):
     run_parity(wl, flags=B.FLAG_NO_TENSOR_CORES, expect_path=B.PATH_SIMT)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_update_pass_over_groups_of_eight_rows_when_rows_are_not_whole_vectors(dtype):
+    # wide, cols % 8 != 0, rows % 8 == 0: the update pass tiles 8-row groups (one group, a ragged last
+    # tile of groups, several column chunks, columns that wrap inside a thread's eight elements)
+    wl = _wl([(8, 9), (16, 37), (40, 2053), (136, 4099), (264, 333)], 2, dtype=dtype, wd=0.05, steps=4, T=2)
+    run_parity(wl, flags=B.FLAG_NO_TENSOR_CORES, expect_path=B.PATH_SIMT)
+
+
 def test_cuda_core_path_rank_spanning_row_blocks_and_ragged_tiles():
     wl = _wl([(200, 333), (333, 200), (130, 130)], 130, dtype="bf16", steps=4, T=2)
     run_parity(wl, flags=B.FLAG_NO_TENSOR_CORES, expect_path=B.PATH_SIMT)
