@@ -935,27 +935,66 @@ __global__ void generate_p_kernel(const MatDesc* __restrict__ descs, int mat_beg
 }  // namespace
 
 // G with an odd row pitch -> copy with the pitch rounded up to 8 elements (TMA needs 16-byte rows).
-// One 16-byte store per thread and pass: its eight source elements are 2-byte loads, contiguous
-// across the warp, so every sector is fetched once; the padding columns are written as zero.
+// One 16-byte store per thread and pass.  A source row starts `mis` bytes (even, the same for the whole
+// row) past a 16-byte boundary of the array, so the eight elements of a store lie in two aligned
+// 16-byte words: both are loaded (the second is the neighbouring thread's first) and the result is cut
+// out with funnel shifts.  The padding columns are written as zero; the last vectors of the array, whose
+// second word would reach past its end, are gathered element by element.
 __global__ void repitch_kernel(const MatDesc* __restrict__ descs, int first)
 {
     const MatDesc* dp = descs + first + blockIdx.y;
     uint4* dst = static_cast<uint4*>(dp->gpad);
     if (!dst) return;
     const unsigned short* __restrict__ src = static_cast<const unsigned short*>(dp->G);
+    const char* __restrict__ src_b = static_cast<const char*>(dp->G);
     const int rows = __ldg(&dp->rows), cols = __ldg(&dp->cols), vecs = __ldg(&dp->g_pitch) / 8;
+    const int64_t total_bytes = (int64_t)rows * cols * 2;
     for (int row = blockIdx.x; row < rows; row += gridDim.x) {
-        const unsigned short* __restrict__ in = src + (int64_t)row * cols;
+        const int64_t rb = (int64_t)row * cols * 2;
+        const uint32_t mis = (uint32_t)(rb & 15), wsel = mis >> 2, sh = (mis & 2u) * 8u;
         for (int v = threadIdx.x; v < vecs; v += blockDim.x) {
             const int c = 8 * v;
-            uint32_t w[4];
+            const int64_t a = rb - mis + 16 * (int64_t)v;
+            uint32_t o[4];
+            if (a + 32 <= total_bytes) {
+                const uint4 lo = __ldg(reinterpret_cast<const uint4*>(src_b + a));
+                const uint4 hi = __ldg(reinterpret_cast<const uint4*>(src_b + a + 16));
+                const uint32_t w[8] = { lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w };
+                switch (wsel) {          // uniform over the row
+                case 0:
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const uint32_t lo = c + 2 * e < cols ? (uint32_t)__ldg(in + c + 2 * e) : 0u;
-                const uint32_t hi = c + 2 * e + 1 < cols ? (uint32_t)__ldg(in + c + 2 * e + 1) : 0u;
-                w[e] = lo | (hi << 16);
+                    for (int k = 0; k < 4; ++k) o[k] = __funnelshift_r(w[k], w[k + 1], sh);
+                    break;
+                case 1:
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) o[k] = __funnelshift_r(w[k + 1], w[k + 2], sh);
+                    break;
+                case 2:
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) o[k] = __funnelshift_r(w[k + 2], w[k + 3], sh);
+                    break;
+                default:
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) o[k] = __funnelshift_r(w[k + 3], w[k + 4], sh);
+                    break;
+                }
+                if (c + 8 > cols) {      // the row ends inside this vector: what follows belongs to the next row
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        if (c + 2 * k >= cols) o[k] = 0u;
+                        else if (c + 2 * k + 1 >= cols) o[k] &= 0xFFFFu;
+                    }
+                }
+            } else {
+                const unsigned short* __restrict__ in = src + (int64_t)row * cols;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const uint32_t e0 = c + 2 * k < cols ? (uint32_t)__ldg(in + c + 2 * k) : 0u;
+                    const uint32_t e1 = c + 2 * k + 1 < cols ? (uint32_t)__ldg(in + c + 2 * k + 1) : 0u;
+                    o[k] = e0 | (e1 << 16);
+                }
             }
-            dst[(int64_t)row * vecs + v] = make_uint4(w[0], w[1], w[2], w[3]);
+            dst[(int64_t)row * vecs + v] = make_uint4(o[0], o[1], o[2], o[3]);
         }
     }
 }
