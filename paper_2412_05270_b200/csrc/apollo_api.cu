@@ -144,7 +144,7 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
     plan.zero_begin = off;
     for (int i = 0; i < n_mat; ++i) {
         MatPlan& p = plan.mats[i];
-        const size_t state = ((cfg->flags & APOLLO_FLAG_BF16_STATES) ? 2 : sizeof(float)) * (size_t)r * (size_t)p.n;
+        const size_t state = ((cfg->flags & APOLLO_FLAG_BF16_STATES) ? 2 : sizeof(float)) * (size_t)r * (size_t)state_pitch(p.n, r);
         p.off_M = off; off = align_up(off + state);
         p.off_V = off; off = align_up(off + state);
         p.off_scal = off; off += ALIGN;     // scal[4] then prev at float index 8
@@ -289,6 +289,7 @@ int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_ma
         d.ext_p = nullptr;
         d.r_scale = (float)(1.0 / std::sqrt((double)cfg->rank));
         d.rows = p.rows; d.cols = p.cols; d.m = p.m; d.n = p.n; d.tall = p.tall; d.path = p.path;
+        d.ns = state_pitch(p.n, cfg->rank);
         d.slices = p.slices; d.g2_slices = p.g2_slices; d.matrix_id = i;
         d.tiles_n = p.tiles_n; d.tiles_k = p.tiles_k;
         for (int t = 0; t < 3; ++t)
@@ -504,15 +505,16 @@ int apollo_get_state(apollo_ctx* ctx, int32_t matrix, float* d_M, float* d_V, vo
 {
     if (!ctx || !d_M || !d_V || matrix < 0 || matrix >= ctx->n_mat) return APOLLO_ERR_INVALID_ARG;
     const MatDesc& d = ctx->h_descs[matrix];
-    const size_t count = (size_t)ctx->cfg.rank * (size_t)d.n;
+    const size_t r = (size_t)ctx->cfg.rank, n = (size_t)d.n, ns = (size_t)d.ns;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (ctx->cfg.flags & APOLLO_FLAG_BF16_STATES) {
-        launch_widen_bf16(d.M, d_M, count, stream);
-        launch_widen_bf16(d.V, d_V, count, stream);
+        launch_widen_bf16(d.M, d_M, r, n, ns, stream);
+        launch_widen_bf16(d.V, d_V, r, n, ns, stream);
         return cuda_ok(cudaGetLastError()) ? APOLLO_OK : APOLLO_ERR_CUDA;
     }
-    if (cudaMemcpyAsync(d_M, d.M, sizeof(float) * count, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) return APOLLO_ERR_CUDA;
-    if (cudaMemcpyAsync(d_V, d.V, sizeof(float) * count, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) return APOLLO_ERR_CUDA;
+    // the library's rows have pitch ns; the caller gets them dense
+    if (cudaMemcpy2DAsync(d_M, sizeof(float) * n, d.M, sizeof(float) * ns, sizeof(float) * n, r, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) return APOLLO_ERR_CUDA;
+    if (cudaMemcpy2DAsync(d_V, sizeof(float) * n, d.V, sizeof(float) * ns, sizeof(float) * n, r, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) return APOLLO_ERR_CUDA;
     return APOLLO_OK;
 }
 
@@ -558,16 +560,22 @@ static int state_copy(apollo_ctx* ctx, char* d_flat, bool to_flat, cudaStream_t 
     size_t at = 0;
     for (int i = 0; i < ctx->n_mat; ++i) {
         const MatDesc& d = ctx->h_descs[i];
-        const size_t bytes = state_elem_bytes(ctx) * (size_t)ctx->cfg.rank * (size_t)d.n;
-        void* parts[3] = { d.M, d.V, d.prev };
-        const size_t sizes[3] = { bytes, bytes, sizeof(float) };
-        for (int k = 0; k < 3; ++k) {
+        // M and V are dense (r x n) in the checkpoint and have row pitch ns in the workspace
+        const size_t row = state_elem_bytes(ctx) * (size_t)d.n, pitch = state_elem_bytes(ctx) * (size_t)d.ns;
+        const size_t r = (size_t)ctx->cfg.rank;
+        void* parts[2] = { d.M, d.V };
+        for (int k = 0; k < 2; ++k) {
             const cudaError_t e = to_flat
-                ? cudaMemcpyAsync(d_flat + at, parts[k], sizes[k], cudaMemcpyDeviceToDevice, stream)
-                : cudaMemcpyAsync(parts[k], d_flat + at, sizes[k], cudaMemcpyDeviceToDevice, stream);
+                ? cudaMemcpy2DAsync(d_flat + at, row, parts[k], pitch, row, r, cudaMemcpyDeviceToDevice, stream)
+                : cudaMemcpy2DAsync(parts[k], pitch, d_flat + at, row, row, r, cudaMemcpyDeviceToDevice, stream);
             if (!cuda_ok(e)) return APOLLO_ERR_CUDA;
-            at += sizes[k];
+            at += row * r;
         }
+        const cudaError_t e = to_flat
+            ? cudaMemcpyAsync(d_flat + at, d.prev, sizeof(float), cudaMemcpyDeviceToDevice, stream)
+            : cudaMemcpyAsync(d.prev, d_flat + at, sizeof(float), cudaMemcpyDeviceToDevice, stream);
+        if (!cuda_ok(e)) return APOLLO_ERR_CUDA;
+        at += sizeof(float);
     }
     return APOLLO_OK;
 }

@@ -61,13 +61,17 @@ inline long long update_tile_count(long long rows, long long cols, bool tall)
     return (rows + tile_rows - 1) / tile_rows * t.chunks;
 }
 
+// Row pitch of M and V.  The epilogues read and write a row of a moment 128 channels at a time; with
+// an odd n (5461 in the 1B-shaped list) those pieces straddle sectors and lines.
+inline int state_pitch(int n, int rank) { return rank > 1 ? (n + 63) / 64 * 64 : n; }
+
 // Per-matrix record in device memory.  Pointers into the workspace are fixed at create
 // time; W, G and dW are refreshed whenever the caller passes different addresses.
 struct MatDesc {
     void* W;
     const void* G;
     float* dW;        // optional fp32 capture of the update, or nullptr
-    float* M;         // r x n, row-major; fp32, or bfloat16 behind the same pointer when StepParams::state_bf16
+    float* M;         // r x n, row-major with row pitch ns; fp32, or bfloat16 behind the same pointer when StepParams::state_bf16
     float* V;         // r x n
     float* s;         // n scales of the last step
     float* part;      // projection partial sums, layout depends on the path (see kernels)
@@ -81,6 +85,7 @@ struct MatDesc {
     void* gpad;       // copy of G with a 16-byte row pitch when cols % 8 != 0 (tensor path), else nullptr
     int32_t rows, cols;
     int32_t m, n;     // m = min(rows, cols) = projected side; n = max = number of channels
+    int32_t ns;       // row pitch of M and V in elements: n, rounded up (state_pitch) so that every row starts a 256-byte line
     int32_t tall;     // 1 if rows > cols: channels are the stored rows
     int32_t path;
     int32_t slices;   // number of partial slices in `part`

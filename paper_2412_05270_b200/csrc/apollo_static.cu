@@ -75,6 +75,7 @@ extern "C" int apollo_mini_step_static(void* d_W, const void* d_G, int64_t rows,
     d.tall = rows > cols;
     d.m = (int32_t)(d.tall ? cols : rows);
     d.n = (int32_t)(d.tall ? rows : cols);
+    d.ns = d.n;
     d.path = PATH_STREAM;
     d.matrix_id = (int32_t)matrix;
     if (!d.tall) {

@@ -18,7 +18,7 @@ void launch_update(int dtype, const MatDesc* d_descs, const int* d_prefix, int n
 
 
 // bfloat16 -> float copy (observability of bfloat16 states).
-void launch_widen_bf16(const void* d_src, float* d_dst, size_t count, cudaStream_t stream);
+void launch_widen_bf16(const void* d_src, float* d_dst, size_t rows, size_t cols, size_t src_pitch, cudaStream_t stream);
 
 // Tensor-core projection (TMA + tcgen05 + TMEM).
 bool tensor_path_supports(int rows, int cols, int rank, int dtype);

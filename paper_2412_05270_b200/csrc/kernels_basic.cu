@@ -326,7 +326,7 @@ project_simt_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                 const int j = j0 + tx * 4 + y;
                 if (k < r && j < n) {
                     const float rv = acc[x][y] * r_scale;
-                    const int64_t at = (int64_t)k * n + j;
+                    const int64_t at = (int64_t)k * d.ns + j;
                     const bool sb = sp.state_bf16 != 0;
                     const float mv = sp.beta1 * state_load(d.M, at, sb) + (1.0f - sp.beta1) * rv;
                     const float vv = sp.beta2 * state_load(d.V, at, sb) + (1.0f - sp.beta2) * rv * rv;
@@ -622,16 +622,22 @@ update_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix,
     }
 }
 
-__global__ void widen_bf16_kernel(const unsigned short* __restrict__ src, float* __restrict__ dst, size_t count)
+__global__ void widen_bf16_kernel(const unsigned short* __restrict__ src, float* __restrict__ dst, size_t rows,
+                                  size_t cols, size_t src_pitch)
 {
-    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < count; i += (size_t)gridDim.x * blockDim.x)
-        dst[i] = bf16_bits_to_float((uint32_t)src[i]);
+    const size_t count = rows * cols;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < count; i += (size_t)gridDim.x * blockDim.x) {
+        const size_t r = i / cols;
+        dst[i] = bf16_bits_to_float((uint32_t)src[r * src_pitch + (i - r * cols)]);
+    }
 }
 
-void launch_widen_bf16(const void* d_src, float* d_dst, size_t count, cudaStream_t stream)
+// bfloat16 rows of pitch `src_pitch` elements -> dense fp32 rows
+void launch_widen_bf16(const void* d_src, float* d_dst, size_t rows, size_t cols, size_t src_pitch, cudaStream_t stream)
 {
-    if (count == 0) return;
-    widen_bf16_kernel<<<blocks_for((int64_t)count), 256, 0, stream>>>(static_cast<const unsigned short*>(d_src), d_dst, count);
+    if (rows * cols == 0) return;
+    widen_bf16_kernel<<<blocks_for((int64_t)(rows * cols)), 256, 0, stream>>>(static_cast<const unsigned short*>(d_src), d_dst, rows,
+                                                                            cols, src_pitch);
 }
 
 // ----------------------------------------------------------------------------------------

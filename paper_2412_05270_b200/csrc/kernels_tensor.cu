@@ -328,6 +328,7 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
         const void* tmap_p = dp->tmap_p;
         const float r_scale = __ldg(&dp->r_scale);
         float* const Mbase = dp->M;
+        const int64_t ns = __ldg(&dp->ns);
         float* const Vbase = dp->V;
         float* const part = dp->part;
         float* const g2out = dp->g2;
@@ -535,20 +536,20 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                 ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * r_slice + cchunk * 16), rv);
                 const int j = j0 + b * 128 + ch_in_blk;
                 if (j < n) {
-                    const int64_t at = (int64_t)(r0 + cchunk * 16) * n + j;
+                    const int64_t at = (int64_t)(r0 + cchunk * 16) * ns + j;
                     const bool sb = sp.state_bf16 != 0;
                     float mv[16], vv[16];
 #pragma unroll
                     for (int k = 0; k < 16; ++k) {
-                        mv[k] = state_load(Mbase, at + (int64_t)k * n, sb);
-                        vv[k] = state_load(Vbase, at + (int64_t)k * n, sb);
+                        mv[k] = state_load(Mbase, at + (int64_t)k * ns, sb);
+                        vv[k] = state_load(Vbase, at + (int64_t)k * ns, sb);
                     }
 #pragma unroll
                     for (int k = 0; k < 16; ++k) {
                         const float r = rv[k] * r_scale;
                         const float mn = sp.beta1 * mv[k] + (1.0f - sp.beta1) * r;
                         const float vn = sp.beta2 * vv[k] + (1.0f - sp.beta2) * r * r;
-                        state_store(Mbase, at + (int64_t)k * n, mn, sb); state_store(Vbase, at + (int64_t)k * n, vn, sb);
+                        state_store(Mbase, at + (int64_t)k * ns, mn, sb); state_store(Vbase, at + (int64_t)k * ns, vn, sb);
                         const float rt = __fdividef(mn * sp.inv_bc1, fast_sqrt(vn * sp.inv_bc2) + sp.eps);
                         num = fmaf(rt, rt, num);
                         den = fmaf(r, r, den);
@@ -835,6 +836,7 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             const int q = warp & 3, half = (warp - 8) >> 2;
             const int ch = q * 32 + lane, j = j0 + ch;
             float* const Mbase = dp->M;
+            const int64_t ns = __ldg(&dp->ns);
             float* const Vbase = dp->V;
             const float r_scale = __ldg(&dp->r_scale);
             const bool acc_ok = __all_sync(0xFFFFFFFFu, wait_phase_idle(bar_acc_full + 8 * buf, use & 1, abort_flag, status));   // tcgen05.ld needs the whole warp
@@ -845,20 +847,20 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                 float rv[16];
                 ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + buf * (uint32_t)r_slice + (uint32_t)(cchunk * 16), rv);
                 if (j < n) {
-                    const int64_t at = (int64_t)(r0 + cchunk * 16) * n + j;
+                    const int64_t at = (int64_t)(r0 + cchunk * 16) * ns + j;
                     const bool sb = sp.state_bf16 != 0;
                     float mv[16], vv[16];
 #pragma unroll
                     for (int k = 0; k < 16; ++k) {
-                        mv[k] = state_load(Mbase, at + (int64_t)k * n, sb);
-                        vv[k] = state_load(Vbase, at + (int64_t)k * n, sb);
+                        mv[k] = state_load(Mbase, at + (int64_t)k * ns, sb);
+                        vv[k] = state_load(Vbase, at + (int64_t)k * ns, sb);
                     }
 #pragma unroll
                     for (int k = 0; k < 16; ++k) {
                         const float r = rv[k] * r_scale;
                         const float mn = sp.beta1 * mv[k] + (1.0f - sp.beta1) * r;
                         const float vn = sp.beta2 * vv[k] + (1.0f - sp.beta2) * r * r;
-                        state_store(Mbase, at + (int64_t)k * n, mn, sb); state_store(Vbase, at + (int64_t)k * n, vn, sb);
+                        state_store(Mbase, at + (int64_t)k * ns, mn, sb); state_store(Vbase, at + (int64_t)k * ns, vn, sb);
                         const float rt = __fdividef(mn * sp.inv_bc1, fast_sqrt(vn * sp.inv_bc2) + sp.eps);
                         num = fmaf(rt, rt, num);
                         den = fmaf(r, r, den);
