@@ -128,6 +128,7 @@ struct TcTiling {
     int32_t smem_bytes;
     int32_t staged;    // 0: P generated in shared memory; 1: P loaded from the staging buffer
     int32_t pair;      // 1: the pair kernel (CTA pairs, cta_group::2); staged only
+    int32_t epi_prefetch; // pair kernel: the epilogue warps ask L2 for the moments one chunk ahead of their loads
 };
 
 // Device status word values.

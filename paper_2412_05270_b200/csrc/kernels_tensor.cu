@@ -65,6 +65,7 @@ TcTiling choose_tiling(int rank)
     }
     t.staged = tensor_path_staged() ? 1 : 0;
     t.pair = 0;
+    t.epi_prefetch = 0;
     // Staged P has two kernels: the pair kernel (default; faster on every list measured) and the
     // single-CTA ring kernel (APOLLO_TC_KERNEL=ring), which is also the one that can generate P itself.
     const char* kernel = std::getenv("APOLLO_TC_KERNEL");
@@ -76,6 +77,7 @@ TcTiling choose_tiling(int rank)
         t.stages = (TC_MAX_SMEM - 1536) / stage;
         if (t.stages > 8) t.stages = 8;
         t.smem_bytes = t.stages * stage + 1536;
+        if (const char* env = std::getenv("APOLLO_TC_EPI_PREFETCH")) t.epi_prefetch = env[0] != '0' ? 1 : 0;
         return t;
     }
     const int stage = t.nblk * TC_BLOCK_BYTES + t.r_slice * 128;
@@ -695,7 +697,9 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             if (lane == 0) {
                 const void* tmap = dp->tmap;
                 ptx::fence_tensormap_acquire(tmap);
-                const uint64_t pol_g = ptx::policy_evict_first();
+                // G is read once per row slice: with one slice it may leave L2 at once; with several, the pairs
+                // that work on the other slices of this channel tile at about the same time should find it there
+                const uint64_t pol_g = tiles_k > 1 ? ptx::policy_evict_normal() : ptx::policy_evict_first();
                 // the bytes of both CTAs are counted on the leader's barrier; the peer's may arrive
                 // there before the leader's expect_tx (the count is signed), never a phase early,
                 // because the peer's stage is only free once the leader's MMA has consumed it
@@ -839,11 +843,23 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             const int64_t ns = __ldg(&dp->ns);
             float* const Vbase = dp->V;
             const float r_scale = __ldg(&dp->r_scale);
+            // One chunk ahead of its loads, the warp asks L2 for the 32 lines of the chunk (lane l: row l of M,
+            // lane 16 + l: row l of V, the warp's 32 channels): the loads then pay an L2 round trip, and twice
+            // as many bytes of the moments are in flight per SM.  The first chunk is asked for before the
+            // wait for the accumulator.
+            const bool pf = tl.epi_prefetch != 0 && j0 + q * 32 < n;
+            const char* const pf_base = reinterpret_cast<const char*>(lane < 16 ? Mbase : Vbase);
+            const int64_t pf_esz = sp.state_bf16 != 0 ? 2 : 4;
+            auto ask = [&](int chunk) {
+                ptx::prefetch_l2(pf_base + ((int64_t)(r0 + chunk * 16 + (lane & 15)) * ns + j0 + q * 32) * pf_esz);
+            };
+            if (pf && half < r_slice / 16) ask(half);
             const bool acc_ok = __all_sync(0xFFFFFFFFu, wait_phase_idle(bar_acc_full + 8 * buf, use & 1, abort_flag, status));   // tcgen05.ld needs the whole warp
             ptx::tc_fence_after_sync();
             float num = 0.f, den = 0.f;
             const int chunks = acc_ok ? r_slice / 16 : 0;
             for (int cchunk = half; cchunk < chunks; cchunk += 2) {
+                if (pf && cchunk + 2 < chunks) ask(cchunk + 2);
                 float rv[16];
                 ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + buf * (uint32_t)r_slice + (uint32_t)(cchunk * 16), rv);
                 if (j < n) {
