@@ -114,6 +114,8 @@ APOLLO_API int apollo_workspace_bytes(const apollo_shape* shapes, int32_t n_matr
  *   APOLLO_P_STAGING_MB=n    staging budget in MB (default 512); below the size of all projections
  *                            the slots are shared and every step refills them
  *   APOLLO_TC_RSLICE, APOLLO_TC_NBLK   tile shape (rows of R per tile; 128-channel blocks, ring kernel)
+ *   APOLLO_TC_EPI_PREFETCH=d pair kernel: how many 16-row chunks ahead of its loads an epilogue warp asks L2
+ *                            for the moments (0..8, default 1; 0 = no prefetch)
  */
 APOLLO_API int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_matrices,
                   const apollo_config* cfg, void* d_workspace, size_t workspace_bytes);

@@ -65,7 +65,7 @@ TcTiling choose_tiling(int rank)
     }
     t.staged = tensor_path_staged() ? 1 : 0;
     t.pair = 0;
-    t.epi_prefetch = 0;
+    t.epi_prefetch = 1;
     // Staged P has two kernels: the pair kernel (default; faster on every list measured) and the
     // single-CTA ring kernel (APOLLO_TC_KERNEL=ring), which is also the one that can generate P itself.
     const char* kernel = std::getenv("APOLLO_TC_KERNEL");
@@ -77,7 +77,10 @@ TcTiling choose_tiling(int rank)
         t.stages = (TC_MAX_SMEM - 1536) / stage;
         if (t.stages > 8) t.stages = 8;
         t.smem_bytes = t.stages * stage + 1536;
-        if (const char* env = std::getenv("APOLLO_TC_EPI_PREFETCH")) t.epi_prefetch = env[0] != '0' ? 1 : 0;
+        if (const char* env = std::getenv("APOLLO_TC_EPI_PREFETCH")) {
+            const int v = std::atoi(env);
+            if (v >= 0 && v <= 8) t.epi_prefetch = v;
+        }
         return t;
     }
     const int stage = t.nblk * TC_BLOCK_BYTES + t.r_slice * 128;
@@ -853,13 +856,16 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             auto ask = [&](int chunk) {
                 ptx::prefetch_l2(pf_base + ((int64_t)(r0 + chunk * 16 + (lane & 15)) * ns + j0 + q * 32) * pf_esz);
             };
-            if (pf && half < r_slice / 16) ask(half);
+            const int pf_d = tl.epi_prefetch;                            // distance in chunks of this warp
+            if (pf)
+                for (int a = 0; a < pf_d; ++a)
+                    if (half + 2 * a < r_slice / 16) ask(half + 2 * a);
             const bool acc_ok = __all_sync(0xFFFFFFFFu, wait_phase_idle(bar_acc_full + 8 * buf, use & 1, abort_flag, status));   // tcgen05.ld needs the whole warp
             ptx::tc_fence_after_sync();
             float num = 0.f, den = 0.f;
             const int chunks = acc_ok ? r_slice / 16 : 0;
             for (int cchunk = half; cchunk < chunks; cchunk += 2) {
-                if (pf && cchunk + 2 < chunks) ask(cchunk + 2);
+                if (pf && cchunk + 2 * pf_d < chunks) ask(cchunk + 2 * pf_d);
                 float rv[16];
                 ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + buf * (uint32_t)r_slice + (uint32_t)(cchunk * 16), rv);
                 if (j < n) {

@@ -81,6 +81,8 @@ def test_tensor_core_path(rank, shapes):
     {"APOLLO_TC_KERNEL": "ring", "APOLLO_TC_RSLICE": "128", "APOLLO_TC_NBLK": "2"},
     {"APOLLO_P_STAGING": "0"},                              # P generated in shared memory by every CTA (ring kernel)
     {"APOLLO_P_STAGING": "0", "APOLLO_TC_RSLICE": "128", "APOLLO_TC_NBLK": "4"},
+    {"APOLLO_TC_EPI_PREFETCH": "0"},                        # no L2 prefetch of the moments in the epilogue
+    {"APOLLO_TC_EPI_PREFETCH": "8", "APOLLO_TC_RSLICE": "64"},   # prefetch distance beyond the chunks of a slice
 ])
 def test_tensor_core_path_selectable_modes(env, monkeypatch):
     """The environment switches of the tensor path give the same parity; where they leave the tiles and
