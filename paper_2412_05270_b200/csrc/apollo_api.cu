@@ -144,7 +144,7 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
     plan.zero_begin = off;
     for (int i = 0; i < n_mat; ++i) {
         MatPlan& p = plan.mats[i];
-        const size_t state = ((cfg->flags & APOLLO_FLAG_BF16_STATES) ? 2 : sizeof(float)) * (size_t)r * (size_t)state_pitch(p.n, r);
+        const size_t state = ((cfg->flags & APOLLO_FLAG_BF16_STATES) ? 2 : sizeof(float)) * (size_t)state_elements(p.n, r, p.path == PATH_TENSOR);
         p.off_M = off; off = align_up(off + state);
         p.off_V = off; off = align_up(off + state);
         p.off_scal = off; off += ALIGN;     // scal[4] then prev at float index 8
@@ -290,6 +290,7 @@ int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_ma
         d.r_scale = (float)(1.0 / std::sqrt((double)cfg->rank));
         d.rows = p.rows; d.cols = p.cols; d.m = p.m; d.n = p.n; d.tall = p.tall; d.path = p.path;
         d.ns = state_pitch(p.n, cfg->rank);
+        d.state_tiled = p.path == PATH_TENSOR ? 1 : 0;
         d.slices = p.slices; d.g2_slices = p.g2_slices; d.matrix_id = i;
         d.tiles_n = p.tiles_n; d.tiles_k = p.tiles_k;
         for (int t = 0; t < 3; ++t)
@@ -507,9 +508,11 @@ int apollo_get_state(apollo_ctx* ctx, int32_t matrix, float* d_M, float* d_V, vo
     const MatDesc& d = ctx->h_descs[matrix];
     const size_t r = (size_t)ctx->cfg.rank, n = (size_t)d.n, ns = (size_t)d.ns;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    if (ctx->cfg.flags & APOLLO_FLAG_BF16_STATES) {
-        launch_widen_bf16(d.M, d_M, r, n, ns, stream);
-        launch_widen_bf16(d.V, d_V, r, n, ns, stream);
+    const bool bf16 = (ctx->cfg.flags & APOLLO_FLAG_BF16_STATES) != 0;
+    if (bf16 || d.state_tiled) {
+        // the caller gets dense fp32 rows whatever the library's layout and storage type
+        launch_state_copy(d.M, d_M, (int)r, d.n, d.ns, d.state_tiled != 0, bf16 ? 2 : 4, 4, true, stream);
+        launch_state_copy(d.V, d_V, (int)r, d.n, d.ns, d.state_tiled != 0, bf16 ? 2 : 4, 4, true, stream);
         return cuda_ok(cudaGetLastError()) ? APOLLO_OK : APOLLO_ERR_CUDA;
     }
     // the library's rows have pitch ns; the caller gets them dense
@@ -556,7 +559,7 @@ int apollo_state_bytes(const apollo_ctx* ctx, size_t* out_bytes)
 
 static int state_copy(apollo_ctx* ctx, char* d_flat, bool to_flat, cudaStream_t stream)
 {
-    if (((uintptr_t)d_flat % 2) != 0) return APOLLO_ERR_ALIGN;
+    if (((uintptr_t)d_flat % state_elem_bytes(ctx)) != 0) return APOLLO_ERR_ALIGN;
     size_t at = 0;
     for (int i = 0; i < ctx->n_mat; ++i) {
         const MatDesc& d = ctx->h_descs[i];
@@ -565,10 +568,16 @@ static int state_copy(apollo_ctx* ctx, char* d_flat, bool to_flat, cudaStream_t 
         const size_t r = (size_t)ctx->cfg.rank;
         void* parts[2] = { d.M, d.V };
         for (int k = 0; k < 2; ++k) {
-            const cudaError_t e = to_flat
-                ? cudaMemcpy2DAsync(d_flat + at, row, parts[k], pitch, row, r, cudaMemcpyDeviceToDevice, stream)
-                : cudaMemcpy2DAsync(parts[k], pitch, d_flat + at, row, row, r, cudaMemcpyDeviceToDevice, stream);
-            if (!cuda_ok(e)) return APOLLO_ERR_CUDA;
+            if (d.state_tiled) {
+                const int esz = (int)state_elem_bytes(ctx);
+                launch_state_copy(parts[k], d_flat + at, (int)r, d.n, d.ns, true, esz, esz, to_flat, stream);
+                if (!cuda_ok(cudaGetLastError())) return APOLLO_ERR_CUDA;
+            } else {
+                const cudaError_t e = to_flat
+                    ? cudaMemcpy2DAsync(d_flat + at, row, parts[k], pitch, row, r, cudaMemcpyDeviceToDevice, stream)
+                    : cudaMemcpy2DAsync(parts[k], pitch, d_flat + at, row, row, r, cudaMemcpyDeviceToDevice, stream);
+                if (!cuda_ok(e)) return APOLLO_ERR_CUDA;
+            }
             at += row * r;
         }
         const cudaError_t e = to_flat

@@ -61,9 +61,19 @@ inline long long update_tile_count(long long rows, long long cols, bool tall)
     return (rows + tile_rows - 1) / tile_rows * t.chunks;
 }
 
-// Row pitch of M and V.  The epilogues read and write a row of a moment 128 channels at a time; with
-// an odd n (5461 in the 1B-shaped list) those pieces straddle sectors and lines.
+// Layout of M and V (r x n).  CUDA-core paths: row-major with the row pitch rounded up to 64 elements, so
+// that every row starts a 256-byte line.  Tensor path: channel blocks of 128, each block r x 128
+// row-major (block b holds channels 128 b ..): the 128 channels x r_slice rows that one CTA reads and
+// writes per tile are one contiguous piece of memory instead of r_slice pieces of 512 bytes n apart.
 inline int state_pitch(int n, int rank) { return rank > 1 ? (n + 63) / 64 * 64 : n; }
+inline long long state_elements(int n, int rank, bool tiled)
+{
+    return (long long)rank * (tiled ? (n + 127) / 128 * 128 : state_pitch(n, rank));
+}
+__host__ __device__ inline int64_t state_at(bool tiled, int64_t ns, int rank, int k, int j)
+{
+    return tiled ? ((int64_t)(j >> 7) * rank + k) * 128 + (j & 127) : (int64_t)k * ns + j;
+}
 
 // Per-matrix record in device memory.  Pointers into the workspace are fixed at create
 // time; W, G and dW are refreshed whenever the caller passes different addresses.
@@ -71,7 +81,7 @@ struct MatDesc {
     void* W;
     const void* G;
     float* dW;        // optional fp32 capture of the update, or nullptr
-    float* M;         // r x n, row-major with row pitch ns; fp32, or bfloat16 behind the same pointer when StepParams::state_bf16
+    float* M;         // r x n, element (k, j) at state_at(); fp32, or bfloat16 behind the same pointer when StepParams::state_bf16
     float* V;         // r x n
     float* s;         // n scales of the last step
     float* part;      // projection partial sums, layout depends on the path (see kernels)
@@ -85,7 +95,8 @@ struct MatDesc {
     void* gpad;       // copy of G with a 16-byte row pitch when cols % 8 != 0 (tensor path), else nullptr
     int32_t rows, cols;
     int32_t m, n;     // m = min(rows, cols) = projected side; n = max = number of channels
-    int32_t ns;       // row pitch of M and V in elements: n, rounded up (state_pitch) so that every row starts a 256-byte line
+    int32_t ns;       // row pitch of M and V in elements (state_pitch) when they are row-major
+    int32_t state_tiled; // 1: M and V are stored in channel blocks of 128 (tensor path), see state_at()
     int32_t tall;     // 1 if rows > cols: channels are the stored rows
     int32_t path;
     int32_t slices;   // number of partial slices in `part`

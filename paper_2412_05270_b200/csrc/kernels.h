@@ -18,7 +18,11 @@ void launch_update(int dtype, const MatDesc* d_descs, const int* d_prefix, int n
 
 
 // bfloat16 -> float copy (observability of bfloat16 states).
-void launch_widen_bf16(const void* d_src, float* d_dst, size_t rows, size_t cols, size_t src_pitch, cudaStream_t stream);
+// Copies a moment between the library's layout (state_at(): row-major with pitch ns, or channel blocks of
+// 128) and dense r x n rows; lib_esz / dense_esz are 2 (bfloat16) or 4 (fp32), a bfloat16 source is
+// widened when the destination is fp32.  to_dense = false copies dense -> library (same element size).
+void launch_state_copy(void* d_lib, void* d_dense, int rank, int n, int ns, bool tiled, int lib_esz, int dense_esz,
+                       bool to_dense, cudaStream_t stream);
 
 // Tensor-core projection (TMA + tcgen05 + TMEM).
 bool tensor_path_supports(int rows, int cols, int rank, int dtype);

@@ -622,22 +622,30 @@ update_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix,
     }
 }
 
-__global__ void widen_bf16_kernel(const unsigned short* __restrict__ src, float* __restrict__ dst, size_t rows,
-                                  size_t cols, size_t src_pitch)
+__global__ void state_copy_kernel(void* __restrict__ lib, void* __restrict__ dense, int rank, int n, int ns, bool tiled,
+                                  int lib_esz, int dense_esz, bool to_dense)
 {
-    const size_t count = rows * cols;
-    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < count; i += (size_t)gridDim.x * blockDim.x) {
-        const size_t r = i / cols;
-        dst[i] = bf16_bits_to_float((uint32_t)src[r * src_pitch + (i - r * cols)]);
+    const int64_t count = (int64_t)rank * n;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x) {
+        const int k = (int)(i / n), j = (int)(i - (int64_t)k * n);
+        const int64_t at = state_at(tiled, ns, rank, k, j);
+        if (to_dense) {
+            if (lib_esz == 4) static_cast<float*>(dense)[i] = static_cast<const float*>(lib)[at];
+            else if (dense_esz == 4) static_cast<float*>(dense)[i] = bf16_bits_to_float((uint32_t)static_cast<const unsigned short*>(lib)[at]);
+            else static_cast<unsigned short*>(dense)[i] = static_cast<const unsigned short*>(lib)[at];
+        } else {
+            if (lib_esz == 4) static_cast<float*>(lib)[at] = static_cast<const float*>(dense)[i];
+            else static_cast<unsigned short*>(lib)[at] = static_cast<const unsigned short*>(dense)[i];
+        }
     }
 }
 
-// bfloat16 rows of pitch `src_pitch` elements -> dense fp32 rows
-void launch_widen_bf16(const void* d_src, float* d_dst, size_t rows, size_t cols, size_t src_pitch, cudaStream_t stream)
+void launch_state_copy(void* d_lib, void* d_dense, int rank, int n, int ns, bool tiled, int lib_esz, int dense_esz,
+                       bool to_dense, cudaStream_t stream)
 {
-    if (rows * cols == 0) return;
-    widen_bf16_kernel<<<blocks_for((int64_t)(rows * cols)), 256, 0, stream>>>(static_cast<const unsigned short*>(d_src), d_dst, rows,
-                                                                            cols, src_pitch);
+    const int64_t count = (int64_t)rank * n;
+    if (count == 0) return;
+    state_copy_kernel<<<blocks_for(count), 256, 0, stream>>>(d_lib, d_dense, rank, n, ns, tiled, lib_esz, dense_esz, to_dense);
 }
 
 // ----------------------------------------------------------------------------------------

@@ -333,7 +333,6 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
         const void* tmap_p = dp->tmap_p;
         const float r_scale = __ldg(&dp->r_scale);
         float* const Mbase = dp->M;
-        const int64_t ns = __ldg(&dp->ns);
         float* const Vbase = dp->V;
         float* const part = dp->part;
         float* const g2out = dp->g2;
@@ -541,20 +540,20 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                 ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * r_slice + cchunk * 16), rv);
                 const int j = j0 + b * 128 + ch_in_blk;
                 if (j < n) {
-                    const int64_t at = (int64_t)(r0 + cchunk * 16) * ns + j;
+                    const int64_t at = state_at(true, 0, sp.rank, r0 + cchunk * 16, j);     // channel blocks of 128: rows are 128 elements apart
                     const bool sb = sp.state_bf16 != 0;
                     float mv[16], vv[16];
 #pragma unroll
                     for (int k = 0; k < 16; ++k) {
-                        mv[k] = state_load(Mbase, at + (int64_t)k * ns, sb);
-                        vv[k] = state_load(Vbase, at + (int64_t)k * ns, sb);
+                        mv[k] = state_load(Mbase, at + (int64_t)k * 128, sb);
+                        vv[k] = state_load(Vbase, at + (int64_t)k * 128, sb);
                     }
 #pragma unroll
                     for (int k = 0; k < 16; ++k) {
                         const float r = rv[k] * r_scale;
                         const float mn = sp.beta1 * mv[k] + (1.0f - sp.beta1) * r;
                         const float vn = sp.beta2 * vv[k] + (1.0f - sp.beta2) * r * r;
-                        state_store(Mbase, at + (int64_t)k * ns, mn, sb); state_store(Vbase, at + (int64_t)k * ns, vn, sb);
+                        state_store(Mbase, at + (int64_t)k * 128, mn, sb); state_store(Vbase, at + (int64_t)k * 128, vn, sb);
                         const float rt = __fdividef(mn * sp.inv_bc1, fast_sqrt(vn * sp.inv_bc2) + sp.eps);
                         num = fmaf(rt, rt, num);
                         den = fmaf(r, r, den);
@@ -843,18 +842,19 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             const int q = warp & 3, half = (warp - 8) >> 2;
             const int ch = q * 32 + lane, j = j0 + ch;
             float* const Mbase = dp->M;
-            const int64_t ns = __ldg(&dp->ns);
             float* const Vbase = dp->V;
             const float r_scale = __ldg(&dp->r_scale);
             // One chunk ahead of its loads, the warp asks L2 for the 32 lines of the chunk (lane l: row l of M,
             // lane 16 + l: row l of V, the warp's 32 channels): the loads then pay an L2 round trip, and twice
             // as many bytes of the moments are in flight per SM.  The first chunk is asked for before the
             // wait for the accumulator.
+            // M and V are stored in channel blocks of 128 (state_at): this CTA's block, rows 128 elements apart
+            const int64_t tile_el = (int64_t)(j0 >> 7) * sp.rank * 128;
             const bool pf = tl.epi_prefetch != 0 && j0 + q * 32 < n;
             const char* const pf_base = reinterpret_cast<const char*>(lane < 16 ? Mbase : Vbase);
             const int64_t pf_esz = sp.state_bf16 != 0 ? 2 : 4;
             auto ask = [&](int chunk) {
-                ptx::prefetch_l2(pf_base + ((int64_t)(r0 + chunk * 16 + (lane & 15)) * ns + j0 + q * 32) * pf_esz);
+                ptx::prefetch_l2(pf_base + (tile_el + (int64_t)(r0 + chunk * 16 + (lane & 15)) * 128 + q * 32) * pf_esz);
             };
             const int pf_d = tl.epi_prefetch;                            // distance in chunks of this warp
             if (pf)
@@ -869,20 +869,20 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                 float rv[16];
                 ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + buf * (uint32_t)r_slice + (uint32_t)(cchunk * 16), rv);
                 if (j < n) {
-                    const int64_t at = (int64_t)(r0 + cchunk * 16) * ns + j;
+                    const int64_t at = tile_el + (int64_t)(r0 + cchunk * 16) * 128 + ch;
                     const bool sb = sp.state_bf16 != 0;
                     float mv[16], vv[16];
 #pragma unroll
                     for (int k = 0; k < 16; ++k) {
-                        mv[k] = state_load(Mbase, at + (int64_t)k * ns, sb);
-                        vv[k] = state_load(Vbase, at + (int64_t)k * ns, sb);
+                        mv[k] = state_load(Mbase, at + (int64_t)k * 128, sb);
+                        vv[k] = state_load(Vbase, at + (int64_t)k * 128, sb);
                     }
 #pragma unroll
                     for (int k = 0; k < 16; ++k) {
                         const float r = rv[k] * r_scale;
                         const float mn = sp.beta1 * mv[k] + (1.0f - sp.beta1) * r;
                         const float vn = sp.beta2 * vv[k] + (1.0f - sp.beta2) * r * r;
-                        state_store(Mbase, at + (int64_t)k * ns, mn, sb); state_store(Vbase, at + (int64_t)k * ns, vn, sb);
+                        state_store(Mbase, at + (int64_t)k * 128, mn, sb); state_store(Vbase, at + (int64_t)k * 128, vn, sb);
                         const float rt = __fdividef(mn * sp.inv_bc1, fast_sqrt(vn * sp.inv_bc2) + sp.eps);
                         num = fmaf(rt, rt, num);
                         den = fmaf(r, r, den);
