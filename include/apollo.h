@@ -207,7 +207,9 @@ APOLLO_API int apollo_set_projection(apollo_ctx* ctx, int32_t matrix, const floa
  * state sizes: "2nr + 2"); P is not part of it because it is regenerated from (seed, matrix
  * index, floor(t / T)).  apollo_state_bytes gives the size of the flat DEVICE buffer:
  * per matrix in list order M (r x n entries), V (r x n entries), one float (previous norm);
- * entries are floats, or bfloat16 with APOLLO_FLAG_BF16_STATES.
+ * entries are floats, or bfloat16 with APOLLO_FLAG_BF16_STATES; the buffer is aligned to the entry
+ * size (APOLLO_ERR_ALIGN otherwise) and holds dense row-major matrices whatever layout the
+ * library keeps them in, so it can be read by a context that uses another projection kernel.
  * apollo_state_export copies the state out (after at least one step or an import);
  * apollo_state_import copies it in and sets the step counter; the context must have been
  * created with the same shapes and configuration (the seed and t are the caller's to keep:
