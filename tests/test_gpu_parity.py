@@ -229,6 +229,36 @@ def test_checkpoint_and_resume_continue_bit_for_bit(rank, mode, flags):
         fresh.state_export()                       # nothing has run yet
 
 
+@pytest.mark.parametrize("flags", [0, B.FLAG_BF16_STATES])
+def test_checkpoint_is_dense_whatever_layout_the_kernels_keep(flags):
+    """The tensor path keeps its moments in channel blocks, the CUDA-core path row by row with a padded
+    pitch; the checkpoint and apollo_get_state are dense in both, so a state written by one is read by
+    the other, entry for entry."""
+    shapes = [(200, 336), (336, 203), (64, 64), (128, 520)]     # n = 336, 336, 64, 520: ragged last blocks
+    wl = _wl(shapes, 32, dtype="bf16", T=2, steps=3, wd=0.01)
+    dev = torch.device("cuda")
+    tensor = B.Apollo(wl.shapes, B.config_for(wl, flags))
+    assert all(tensor.path(i) == B.PATH_TENSOR for i in range(len(shapes)))
+    W = [WL.make_weight(wl, i).to(dev) for i in range(len(shapes))]
+    for t in range(3):
+        tensor.step(W, [WL.make_grad(wl, i, t).to(dev) for i in range(len(shapes))], wl.lr, wl.wd)
+    blob = tensor.state_export()
+    cores = B.Apollo(wl.shapes, B.config_for(wl, flags | B.FLAG_NO_TENSOR_CORES))
+    assert all(cores.path(i) == B.PATH_SIMT for i in range(len(shapes)))
+    cores.state_import(blob.clone(), 3)
+    for i in range(len(shapes)):
+        (Ma, Va), (Mb, Vb) = tensor.state(i), cores.state(i)
+        assert torch.equal(Ma, Mb) and torch.equal(Va, Vb)
+        assert Ma.abs().max() > 0 and Va.abs().max() > 0
+    assert torch.equal(blob, cores.state_export())
+    # and back: a second tensor-path context resumes from the CUDA-core context's checkpoint
+    again = B.Apollo(wl.shapes, B.config_for(wl, flags))
+    again.state_import(cores.state_export(), 3)
+    for i in range(len(shapes)):
+        (Ma, Va), (Mb, Vb) = tensor.state(i), again.state(i)
+        assert torch.equal(Ma, Mb) and torch.equal(Va, Vb)
+
+
 @pytest.mark.parametrize("rank,mode,flags", [(32, "channel", 0), (1, "tensor", 0), (5, "channel", B.FLAG_NO_TENSOR_CORES)])
 def test_layer_wise_range_steps_equal_the_whole_list_step(rank, mode, flags):
     shapes = [(200, 336), (336, 200), (64, 64), (128, 520), (96, 203), (72, 64), (64, 72)]
