@@ -24,6 +24,7 @@ pytestmark = pytest.mark.gpu
     ((1100, 1300), "bf16", "tensor"),     # wide, several row slices and column tiles
     ((1300, 520), "bf16", "tensor"),      # tall
     ((257, 1029), "f32", "channel"),      # unaligned pitch, scalar loads
+    ((264, 1029), "bf16", "tensor"),      # unaligned pitch, rows a multiple of 8: update pass over groups of eight rows
 ])
 def test_two_consecutive_static_steps_match_the_context_step(shape, dtype, mode):
     dev = torch.device("cuda")
