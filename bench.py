@@ -5,7 +5,9 @@
 One "step" is one whole apollo_step (projection pass, finalize, update pass) over the
 LLaMA-7B-shaped list of 224 linear weights with rank 256 (bf16 W and G, fp32 states).
 Prints one JSON line.  With N > 1 (torchrun) every rank steps its own replica of the model;
-no collective runs inside the step.
+no collective runs inside the step.  The same line carries, under "also", the step of the
+other named lists (LLaMA-1B at rank 512, 7B APOLLO-Mini, 350M) and, under "sustained", the 7B
+step repeated for several seconds (the board then runs at its power cap).
 """
 from __future__ import annotations
 
@@ -66,7 +68,7 @@ def whole_job_value(params_per_rank: int, world: int, ms_per_step: float) -> flo
     return world * params_per_rank / (ms_per_step * 1e-3)
 
 
-# DRAM bytes per parameter of update_kernel<bf16> from its ncu capture (profiles/update_kernel_*.md);
+# DRAM bytes per parameter of update_kernel<bf16> from its ncu capture on the first two layers of the list;
 # set to None when the kernel changes until the counters are taken again.
 UPDATE_TRAFFIC_BYTES_PER_PARAM = 5.89
 
@@ -151,24 +153,103 @@ def cpu_baseline(wl: WL.Workload, budget_s: float = 12.0):
             "seconds": elapsed, "params": done_params}
 
 
+def oracle_sample_step(wl: WL.Workload, mats, state):
+    """One oracle step over the matrices `mats` (fresh gradients each call); returns seconds and parameters."""
+    import oracle
+    sys.path.insert(0, str(ROOT / "tests"))
+    from parity import oracle_of
+    if not state:
+        oracle.build()
+        state["orc"] = oracle_of(wl, mats)
+        state["W"] = {i: WL.make_weight(wl, i).float().numpy() for i in mats}
+        state["t"] = 0
+    elapsed, params = 0.0, 0
+    for i in mats:
+        G = WL.make_grad(wl, i, state["t"]).float().numpy()
+        t0 = time.perf_counter()
+        res = state["orc"][i].step(state["W"][i], G, float(wl.lr), float(wl.wd))
+        elapsed += time.perf_counter() - t0
+        state["W"][i] = res.W
+        params += G.size
+    state["t"] += 1
+    return elapsed, params
+
+
 def run_reference(args, wl, rank, world):
-    """The reference arm: the CPU oracle on a bounded sample of the workload."""
+    """The reference arm: the CPU oracle, as it stands, on the host cores.  One step of this arm is one oracle
+    step over a bounded sample of the list (one square and one tall matrix), so that warm-up plus timed steps
+    end within a few minutes; parameters per second is the metric, and the estimate for the whole list is the
+    sample's time scaled by the parameter counts."""
     if rank != 0:
         return
-    base = None
-    for _ in range(max(1, min(args.steps, 2))):
-        base = cpu_baseline(wl, budget_s=10.0)
+    mats = [0, 6] if len(wl.shapes) >= 7 else [0]
+    state = {}
+    for _ in range(args.warmup):
+        oracle_sample_step(wl, mats, state)
+    seconds, params = 0.0, 0
+    for _ in range(args.steps):
+        dt, p = oracle_sample_step(wl, mats, state)
+        seconds += dt
+        params += p
+    per_step_s = seconds / max(args.steps, 1)
+    sample_params = params // max(args.steps, 1)
+    value = params / seconds
+    sample = (f"per step: one oracle step of matrices {', '.join('%dx%d' % tuple(wl.shapes[i]) for i in mats)} of "
+              f"{wl.name} (rank {wl.rank}), {sample_params} parameters, {per_step_s:.2f} s")
+    base = {"value": value, "unit": "params/s", "cores": os.cpu_count() or 1, "kind": "oracle", "sample": sample}
     line = {
-        "impl": "reference", "metric": "apollo_step_params_per_s", "value": base["value"], "unit": "params/s",
+        "impl": "reference", "metric": "apollo_step_params_per_s", "value": value, "unit": "params/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": 1e3 * base["seconds"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": 1e3 * per_step_s, "ms_per_full_step_estimate": 1e3 * per_step_s * wl.params / sample_params,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "rank": wl.rank, "mode": wl.mode, "sample": base["sample"]},
-        "cpu_baseline": {k: base[k] for k in ("value", "unit", "cores", "kind", "sample")},
-        "e2e": {"value": base["value"], "unit": "params/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "config": {"workload": wl.name, "rank": wl.rank, "mode": wl.mode, "sample": sample,
+                   "step": "one oracle step over the sample; ms_per_step is the sample's, "
+                           "ms_per_full_step_estimate scales it by parameters to the whole list"},
+        "cpu_baseline": base,
+        "e2e": {"value": value, "unit": "params/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line), flush=True)
+
+
+def time_steps(opt, Ws, Gs, wl, steps, warmup, stream, barrier, clocks):
+    """`warmup` untimed steps, then `steps` timed ones between two CUDA events on `stream`.  Returns the
+    total milliseconds, the kernel launches inside the timed region, the per-phase means and the clocks
+    sampled during the region."""
+    for _ in range(warmup):
+        opt.step(Ws, Gs, wl.lr, wl.wd, check=False)
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t0 = time.monotonic()
+    start.record(stream)
+    launches = 0
+    for _ in range(steps):
+        opt.step(Ws, Gs, wl.lr, wl.wd, check=False)
+        launches += opt.last_launches()
+    stop.record(stream)
+    barrier()
+    t1 = time.monotonic()
+    phases = [opt.timing(k) for k in range(min(steps, 64))]
+    phase_ms = {name: sum(p[k] for p in phases) / len(phases) for k, name in enumerate(("projection", "finalize", "update"))}
+    return start.elapsed_time(stop), launches, phase_ms, clocks.summary(t0, t1)
+
+
+def step_roofline(wl, ms_step, phase_ms, peaks, state_elem=4):
+    """Where the step stands against its bytes and FLOPs.  bytes_min counts G once (the method's own traffic:
+    G, W read, W written, moments read and written); bytes_two_pass counts the second read of G that this
+    implementation's two passes make.  frac_vs_min is the fraction of the step's roofline; frac_schedule is
+    how close the two-pass schedule runs to its own bytes."""
+    two_pass, minimal, update_bytes, flops = step_bytes(wl, state_elem)
+    hbm, tc = peaks["hbm_gbs"] * 1e9, peaks["bf16_tflops_sustained"] * 1e12
+    t_min = max(minimal / hbm, flops / tc)
+    t_2p = max(two_pass / hbm, flops / tc)
+    return {"bytes_min": minimal, "bytes_two_pass": two_pass, "gemm_flops": flops,
+            "t_roofline_ms": 1e3 * t_min, "frac_vs_min": 1e3 * t_min / ms_step,
+            "frac_vs_min_8TBs": 1e3 * max(minimal / 8e12, flops / tc) / ms_step,
+            "t_two_pass_ms": 1e3 * t_2p, "frac_schedule": 1e3 * t_2p / ms_step,
+            "frac_schedule_8TBs": 1e3 * max(two_pass / 8e12, flops / tc) / ms_step,
+            "phase_ms": phase_ms}, update_bytes
 
 
 def run_ours(args, wl, rank, world, local_rank):
@@ -179,12 +260,13 @@ def run_ours(args, wl, rank, world, local_rank):
     torch.cuda.set_device(dev)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
-    n = len(wl.shapes)
-    Ws = [WL.make_weight(wl, i, device=dev) for i in range(n)]
-    Gs = [WL.make_grad(wl, i, 0, device=dev) for i in range(n)]
-    opt = B.Apollo(wl.shapes, B.config_for(wl, B.FLAG_BF16_STATES if args.bf16_states else 0), device=dev)
-    opt.set_timing(True)
+    flags = (B.FLAG_BF16_STATES if args.bf16_states else 0) | (B.FLAG_KEEP_P if args.keep_p else 0)
+    state_elem = 2 if args.bf16_states else 4
     stream = torch.cuda.current_stream()
+    peaks = measured_peaks()
+    tuning = None
+    if args.tuning:
+        tuning = B.make_tuning(**{k: int(v) for k, v in (kv.split("=") for kv in args.tuning.split(","))})
 
     def barrier():
         torch.cuda.synchronize()
@@ -192,29 +274,32 @@ def run_ours(args, wl, rank, world, local_rank):
             dist.barrier()
         torch.cuda.synchronize()
 
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    def make(w):
+        k = len(w.shapes)
+        Ws = [WL.make_weight(w, i, device=dev) for i in range(k)]
+        Gs = [WL.make_grad(w, i, 0, device=dev) for i in range(k)]
+        opt = B.Apollo(w.shapes, B.config_for(w, flags), device=dev, tuning=tuning)
+        opt.set_timing(True)
+        return opt, Ws, Gs
+
+    n = len(wl.shapes)
+    opt, Ws, Gs = make(wl)
     with ClockSampler(local_rank) as clocks:
-        for _ in range(args.warmup):
-            opt.step(Ws, Gs, wl.lr, wl.wd, check=False)
-        barrier()
-        t_region0 = time.monotonic()
-        start.record(stream)
-        launches = 0
-        for _ in range(args.steps):
-            opt.step(Ws, Gs, wl.lr, wl.wd, check=False)
-            launches += opt.last_launches()      # P is regenerated only in steps that open an epoch
-        stop.record(stream)
-        barrier()
-        t_region1 = time.monotonic()
-    ms_total = start.elapsed_time(stop)
-    assert opt.status() == B.OK
-    phases = [opt.timing(k) for k in range(min(args.steps, 64))]
-    proj_ms = sum(p[0] for p in phases) / len(phases)
-    fin_ms = sum(p[1] for p in phases) / len(phases)
-    upd_ms = sum(p[2] for p in phases) / len(phases)
+        ms_total, launches, phase_ms, clock_summary = time_steps(opt, Ws, Gs, wl, args.steps, args.warmup, stream,
+                                                                 barrier, clocks)
+        assert opt.status() == B.OK
+
+        # the same step repeated for several seconds: the board settles at its power cap
+        sustained = None
+        if args.sustain_s > 0:
+            k = max(10, int(args.sustain_s * 1e3 / (ms_total / args.steps)))
+            ms_s, _, phase_s, clock_s = time_steps(opt, Ws, Gs, wl, k, 0, stream, barrier, clocks)
+            sustained = {"steps": k, "seconds": ms_s * 1e-3, "ms_per_step": ms_s / k, "phase_ms": phase_s,
+                         "clocks": clock_s}
+            assert opt.status() == B.OK
 
     # end to end: gradients arrive from pinned host memory every step, the limiter norms go back
-    e2e = None
+    e2e_ms = 0.0
     if not args.no_e2e:
         e2e_steps = max(1, min(args.steps, 3))
         g_bytes = sum(g.numel() * g.element_size() for g in Gs)
@@ -250,19 +335,47 @@ def run_ours(args, wl, rank, world, local_rank):
         barrier()
         e2e_ms = s2.elapsed_time(e2) / e2e_steps
         del host_G
-    ms_total, e2e_ms = max_over_ranks([ms_total, e2e_ms if not args.no_e2e else 0.0], device=dev)
+    workspace = opt.workspace_bytes
+    opt.close()
+    del opt, Ws, Gs
+    torch.cuda.empty_cache()
+
+    # the other lists the metric names, in the same process, each with its own clock window
+    also = {}
+    for name in ([] if args.no_also or args.layers > 0 else [x for x in args.also.split(",") if x and x != wl.name]):
+        w2 = WL.workload(name)
+        o2, W2, G2 = make(w2)
+        with ClockSampler(local_rank) as c2:
+            ms2, _, ph2, cs2 = time_steps(o2, W2, G2, w2, args.steps, args.warmup, stream, barrier, c2)
+        assert o2.status() == B.OK
+        roof2, _ = step_roofline(w2, ms2 / args.steps, ph2, peaks, state_elem)
+        also[name] = {"ms_per_step": ms2 / args.steps, "params": w2.params, "rank": w2.rank, "mode": w2.mode,
+                      "value": whole_job_value(w2.params, world, ms2 / args.steps), "workspace_bytes": o2.workspace_bytes,
+                      "step_roofline": roof2, "clocks": cs2}
+        o2.close()
+        del o2, W2, G2
+        torch.cuda.empty_cache()
+
+    ranked = [ms_total, e2e_ms] + ([sustained["ms_per_step"]] if sustained else []) + [a["ms_per_step"] for a in also.values()]
+    ranked = max_over_ranks(ranked, device=dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
+    ms_total, e2e_ms = ranked[0], ranked[1]
+    at = 2
+    if sustained:
+        sustained["ms_per_step"] = ranked[at]; at += 1
+    for a in also.values():
+        a["ms_per_step"] = ranked[at]; at += 1
+        a["value"] = whole_job_value(a["params"], world, a["ms_per_step"])
 
-    peaks = measured_peaks()
     ms_step = ms_total / args.steps
-    two_pass, minimal, update_bytes, flops = step_bytes(wl, 2 if args.bf16_states else 4)
+    roof, update_bytes = step_roofline(wl, ms_step, phase_ms, peaks, state_elem)
     value = whole_job_value(wl.params, world, ms_step)
-    hbm, tc = peaks["hbm_gbs"] * 1e9, peaks["bf16_tflops_sustained"] * 1e12
-    t_roof = max(two_pass / hbm, flops / tc)
+    upd_ms = phase_ms["update"]
     upd_gbs = update_bytes / (upd_ms * 1e-3) / 1e9
+    traffic = UPDATE_TRAFFIC_BYTES_PER_PARAM * wl.params if UPDATE_TRAFFIC_BYTES_PER_PARAM and wl.dtype == "bf16" else None
     line = {
         "metric": "apollo_step_params_per_s", "value": value, "unit": "params/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
@@ -270,22 +383,29 @@ def run_ours(args, wl, rank, world, local_rank):
         "data": "synthetic",
         "config": {"workload": wl.name, "matrices": n, "params": wl.params, "rank": wl.rank, "mode": wl.mode,
                    "T": wl.T, "lr": wl.lr, "wd": wl.wd, "states": "bf16" if args.bf16_states else "f32", "replicas": world,
+                   "p_storage": "kept" if args.keep_p else "per_step", "workspace_bytes": workspace,
+                   "tuning": args.tuning or "default",
                    "l2": "inputs (W, G: %.1f GB) exceed L2, no flush" % (2 * wl.params * 2 / 1e9)},
         "roofline": {"bound": "hbm", "kernel": "update_kernel", "achieved": upd_gbs, "peak": peaks["hbm_gbs"],
-                     "unit": "GB/s", "frac": upd_gbs / peaks["hbm_gbs"],
-                     "traffic": (UPDATE_TRAFFIC_BYTES_PER_PARAM * wl.params
-                                 if UPDATE_TRAFFIC_BYTES_PER_PARAM and wl.dtype == "bf16" else None),
+                     "unit": "GB/s", "frac": upd_gbs / peaks["hbm_gbs"], "traffic": traffic,
+                     "traffic_source": "ncu capture of the first 2 layers, scaled by parameters (not measured in this run)"
+                     if traffic else None,
                      "peak_source": peaks["source"], "bytes_per_launch": update_bytes, "ms_per_launch": upd_ms},
-        "step_roofline": {"bytes_two_pass": two_pass, "bytes_min": minimal, "gemm_flops": flops,
-                          "t_roofline_ms": 1e3 * t_roof, "frac": 1e3 * t_roof / ms_step,
-                          "frac_vs_8TBs": 1e3 * max(two_pass / 8e12, flops / tc) / ms_step,
-                          "phase_ms": {"projection": proj_ms, "finalize": fin_ms, "update": upd_ms}},
-        "clocks": clocks.summary(t_region0, t_region1),
+        "step_roofline": roof,
+        "clocks": clock_summary,
         "gpu_launches": launches,
     }
+    if sustained:
+        sustained["value"] = whole_job_value(wl.params, world, sustained["ms_per_step"])
+        sustained["frac_vs_min"] = roof["t_roofline_ms"] / sustained["ms_per_step"]
+        sustained["frac_schedule"] = roof["t_two_pass_ms"] / sustained["ms_per_step"]
+        line["sustained"] = sustained
+    if also:
+        line["also"] = also
     if not args.no_e2e:
         line["e2e"] = {"value": whole_job_value(wl.params, world, e2e_ms), "unit": "params/s",
-                       "h2d_bytes_per_step": g_bytes, "d2h_bytes_per_step": n * 16, "ms_per_step": e2e_ms}
+                       "h2d_bytes_per_step": g_bytes, "d2h_bytes_per_step": n * 16, "ms_per_step": e2e_ms,
+                       "note": "bound by the host-to-device copy of the gradients; the weights stay on the device"}
     if args.adamw:
         # the non-projected parameters of the same model (embedding and head 32000 x hidden, norms):
         # 22 bytes per bf16 parameter (read g, p, m, v; write p, m, v)
@@ -325,6 +445,12 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="keep only the first LAYERS layers (profiling aid)")
     ap.add_argument("--adamw", action="store_true", help="also time the fused AdamW of the non-projected parameters")
     ap.add_argument("--bf16-states", action="store_true", help="keep M and V in bfloat16 (a variant, not the headline)")
+    ap.add_argument("--keep-p", action="store_true",
+                    help="keep every matrix's projection for its epoch (APOLLO_FLAG_KEEP_P) instead of regenerating it every step")
+    ap.add_argument("--tuning", default="", help="apollo_tuning fields, e.g. p_generator=1,scratch_mb=64 (measurement aid)")
+    ap.add_argument("--also", default="llama1b,llama7b_mini,llama350m", help="other lists timed in the same run")
+    ap.add_argument("--no-also", action="store_true")
+    ap.add_argument("--sustain-s", type=float, default=3.0, help="seconds of back-to-back steps for the sustained figure (0: skip)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

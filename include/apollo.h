@@ -66,6 +66,10 @@ extern "C" {
 #define APOLLO_FLAG_NO_TENSOR_CORES 1u /* run the projection on the CUDA cores (test and comparison aid) */
 #define APOLLO_FLAG_BF16_STATES 2u     /* keep M and V in bfloat16 (two bytes per entry, as the paper's state-size
                                           figures assume); R~ is formed from the unrounded update */
+#define APOLLO_FLAG_KEEP_P 4u          /* tensor-core path: keep every matrix's projection (r x m bfloat16) in the
+                                          workspace for the T steps of its epoch instead of regenerating it from the
+                                          seed in every step.  Off by default: the method keeps only the seed
+                                          (Algorithm 1; the paper's state-size table counts 2nr + 2 per matrix) */
 
 typedef struct apollo_ctx apollo_ctx; /* opaque HOST object */
 
@@ -87,16 +91,42 @@ typedef struct {
 } apollo_config;
 
 /*
- * Bytes of DEVICE workspace a context over `shapes[0..n_matrices)` needs (moments, scales,
- * partial sums, descriptor tables, tensor maps, and for the tensor-core path a staging buffer
- * for the random projections: up to 512 MB, r x m bf16 values per matrix).  When every matrix
- * has its own slot in that buffer, a projection is generated in the step that opens an epoch
- * (every T steps, Algorithm 1 "if t mod T = 0") and read again by the following steps of the
- * epoch, so the steps of one context must reach the GPU in order, whatever streams they use.
- * shapes, cfg, out: HOST.
+ * Tuning of the tensor-core projection, fixed when a context is created (and when its workspace is
+ * sized: pass the same values to both calls).  A zeroed struct, or a NULL pointer, selects the
+ * defaults.  None of the fields changes the results beyond the order of floating-point sums.
+ */
+#define APOLLO_TC_KERNEL_PAIR 0 /* CTA pairs share every MMA (tcgen05 cta_group::2); default */
+#define APOLLO_TC_KERNEL_RING 1 /* one CTA per tile, single shared-memory ring */
+#define APOLLO_P_SCRATCH 0      /* P goes through a scratch in the workspace that L2 keeps (default) */
+#define APOLLO_P_SHARED 1       /* every CTA generates the P tiles it needs straight into shared memory (ring kernel) */
+typedef struct {
+    int32_t kernel;        /* APOLLO_TC_KERNEL_* */
+    int32_t p_source;      /* APOLLO_P_* */
+    int32_t p_generator;   /* with APOLLO_P_SCRATCH and without APOLLO_FLAG_KEEP_P: 0 = spare warps of the pair
+                              kernel generate the projections a few matrices ahead of their use (default);
+                              1 = a separate kernel fills the scratch group by group between projection launches */
+    int32_t scratch_mb;    /* size of the P scratch in MB; 0 = default (32) */
+    int32_t r_slice;       /* rows of R per tile: a multiple of 16 that divides the rank, <= 256; 0 = default */
+    int32_t nblk;          /* ring kernel: 128-channel blocks per tile (1, 2 or 4; nblk * r_slice <= 512); 0 = default */
+    int32_t epi_prefetch;  /* pair kernel: how many 16-row chunks ahead of its loads an epilogue warp asks L2 for
+                              the moments, as distance + 1 (1 = no prefetch ... 9 = eight chunks); 0 = default (one chunk) */
+    int32_t reserved;      /* 0 */
+} apollo_tuning;
+
+/*
+ * Bytes of DEVICE workspace a context over `shapes[0..n_matrices)` needs: moments, scales,
+ * partial sums, descriptor tables, tensor maps, and for the tensor-core path a scratch for the
+ * random projections.  By default that scratch holds a few matrices' projections (32 MB) and
+ * is refilled from the seed in every step (Algorithm 1 "P_t <- N_seed(0, 1/r)": only the seed is
+ * kept).  With APOLLO_FLAG_KEEP_P every matrix has its own r x m slot, filled in the step that
+ * opens an epoch (every T steps, Algorithm 1 "if t mod T = 0") and read again by the following
+ * steps of the epoch; the steps of such a context must reach the GPU in order, whatever streams
+ * they use.  shapes, cfg, tuning (may be NULL), out: HOST.
  */
 APOLLO_API int apollo_workspace_bytes(const apollo_shape* shapes, int32_t n_matrices, const apollo_config* cfg,
                            size_t* out_bytes);
+APOLLO_API int apollo_workspace_bytes_tuned(const apollo_shape* shapes, int32_t n_matrices, const apollo_config* cfg,
+                                            const apollo_tuning* tuning, size_t* out_bytes);
 
 /*
  * Create a context (Algorithm 1, "Initialize: t <- 0").  d_workspace: DEVICE, 256-byte
@@ -104,21 +134,15 @@ APOLLO_API int apollo_workspace_bytes(const apollo_shape* shapes, int32_t n_matr
  * exclusively by this context until apollo_destroy.  Launches nothing and touches no
  * stream: the moments are zeroed (Appendix: "zero initialization") by the first
  * apollo_step on that step's stream.  The matrix index in the list is the `matrix index`
- * word of the Philox counter.  Must be called with the target device current.
- *
- * Environment switches of the tensor-core projection, read here and at every step (keep them
- * unchanged for the life of a context); none of them changes the results beyond the order of
- * floating-point sums:
- *   APOLLO_TC_KERNEL=ring    the single-CTA kernel instead of the CTA-pair kernel
- *   APOLLO_P_STAGING=0       generate the projection inside the kernel instead of staging it
- *   APOLLO_P_STAGING_MB=n    staging budget in MB (default 512); below the size of all projections
- *                            the slots are shared and every step refills them
- *   APOLLO_TC_RSLICE, APOLLO_TC_NBLK   tile shape (rows of R per tile; 128-channel blocks, ring kernel)
- *   APOLLO_TC_EPI_PREFETCH=d pair kernel: how many 16-row chunks ahead of its loads an epilogue warp asks L2
- *                            for the moments (0..8, default 1; 0 = no prefetch)
+ * word of the Philox counter.  Must be called with the target device current.  The library
+ * reads no environment variable.  apollo_create is apollo_create_tuned with tuning = NULL;
+ * a tuning value out of range is APOLLO_ERR_INVALID_ARG.
  */
 APOLLO_API int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_matrices,
                   const apollo_config* cfg, void* d_workspace, size_t workspace_bytes);
+APOLLO_API int apollo_create_tuned(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_matrices,
+                                   const apollo_config* cfg, const apollo_tuning* tuning, void* d_workspace,
+                                   size_t workspace_bytes);
 
 /*
  * One optimizer step over the whole parameter list (Algorithm 1, body of the loop).
@@ -197,7 +221,7 @@ APOLLO_API int apollo_get_path(const apollo_ctx* ctx, int32_t matrix, int32_t* o
  * as is (R = P G, no 1/sqrt(r) factor) in every later step until replaced; NULL returns
  * the matrix to the generator.  For bf16 gradients at rank > 1, P is rounded to bfloat16 as
  * the generated one is.  The buffer stays owned by the caller and must stay alive.  Not
- * available when the tensor path generates P in shared memory (APOLLO_ERR_UNSUPPORTED).
+ * available with APOLLO_P_SHARED (APOLLO_ERR_UNSUPPORTED).
  */
 APOLLO_API int apollo_set_projection(apollo_ctx* ctx, int32_t matrix, const float* d_P);
 
@@ -270,11 +294,14 @@ APOLLO_API int apollo_adamw_step(void* const* d_P, const void* const* d_G, float
  *                 zero before the first step.
  *   cfg           HOST; cfg->rank must be 1 (APOLLO_ERR_RANK otherwise); mode, dtype, T,
  *                 seed, alpha, gamma, betas, eps, bias_correction as for apollo_create.
+ *                 The moments are floats here: APOLLO_FLAG_BF16_STATES is rejected
+ *                 (APOLLO_ERR_INVALID_ARG); the other flags have no meaning at rank 1.
  *   matrix, t     the matrix index word of the Philox counter and the number of steps
  *                 already taken (the caller keeps t; epoch = t / T).
- * Limits and rules: a matrix whose temporaries exceed the array -- 4 n + 8 n ceil(rows/512)
- * bytes for a wide matrix, 12 n for a tall one, plus 1 KiB -- is rejected with
- * APOLLO_ERR_TOO_LARGE and nothing is launched.  No cudaMalloc, cudaFree or other
+ * Limits and rules: the temporaries are 1 KiB of tables, the n scales (4 n bytes) and the
+ * partial sums of the projection (8 n ceil(rows/512) bytes for a wide matrix, 8 n for a tall
+ * one), the two arrays each rounded up to a multiple of 256 bytes.  A matrix for which that
+ * sum exceeds the array is rejected with APOLLO_ERR_TOO_LARGE and nothing is launched.  No cudaMalloc, cudaFree or other
  * allocating call is made.  The first call on each device looks up the array's device
  * address (with that device current); make that first call outside any stream capture.
  * All calls on a device share the one array, which keeps whatever the previous call

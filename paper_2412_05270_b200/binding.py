@@ -23,6 +23,9 @@ SCALE_CHANNEL, SCALE_TENSOR = 0, 1
 DT_F32, DT_BF16 = 0, 1
 FLAG_NO_TENSOR_CORES = 1
 FLAG_BF16_STATES = 2
+FLAG_KEEP_P = 4
+TC_KERNEL_PAIR, TC_KERNEL_RING = 0, 1
+P_SCRATCH, P_SHARED = 0, 1
 PATH_STREAM, PATH_SIMT, PATH_TENSOR = 0, 1, 2
 
 EXPORTS = [
@@ -31,7 +34,7 @@ EXPORTS = [
     "apollo_philox_draws", "apollo_projection", "apollo_get_path", "apollo_last_launches", "apollo_strerror",
     "apollo_set_timing", "apollo_get_timing", "apollo_mini_step_static", "apollo_cuda_error_string", "apollo_adamw_step",
     "apollo_state_bytes", "apollo_state_export", "apollo_state_import", "apollo_step_range", "apollo_set_projection",
-    "apollo_selftest_bounded_wait",
+    "apollo_selftest_bounded_wait", "apollo_workspace_bytes_tuned", "apollo_create_tuned",
 ]
 
 
@@ -56,6 +59,20 @@ class Config(ctypes.Structure):
     ]
 
 
+class Tuning(ctypes.Structure):
+    """apollo_tuning: zero fields select the defaults."""
+    _fields_ = [("kernel", ctypes.c_int32), ("p_source", ctypes.c_int32), ("p_generator", ctypes.c_int32),
+                ("scratch_mb", ctypes.c_int32), ("r_slice", ctypes.c_int32), ("nblk", ctypes.c_int32),
+                ("epi_prefetch", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+def make_tuning(kernel=TC_KERNEL_PAIR, p_source=P_SCRATCH, p_generator=0, scratch_mb=0, r_slice=0, nblk=0,
+                epi_prefetch=None) -> Tuning:
+    """epi_prefetch: distance in chunks (0 = no prefetch), None = the default."""
+    return Tuning(int(kernel), int(p_source), int(p_generator), int(scratch_mb), int(r_slice), int(nblk),
+                  0 if epi_prefetch is None else int(epi_prefetch) + 1, 0)
+
+
 _lib = None
 
 
@@ -72,6 +89,10 @@ def load():
                                            ctypes.POINTER(ctypes.c_size_t)]
     lib.apollo_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(Shape), i32, ctypes.POINTER(Config), vp,
                                   ctypes.c_size_t]
+    lib.apollo_workspace_bytes_tuned.argtypes = [ctypes.POINTER(Shape), i32, ctypes.POINTER(Config),
+                                                 ctypes.POINTER(Tuning), ctypes.POINTER(ctypes.c_size_t)]
+    lib.apollo_create_tuned.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(Shape), i32, ctypes.POINTER(Config),
+                                        ctypes.POINTER(Tuning), vp, ctypes.c_size_t]
     lib.apollo_step.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), f32, f32, vp]
     lib.apollo_step_range.argtypes = [vp, i32, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), f32, f32, i32, vp]
     lib.apollo_set_projection.argtypes = [vp, i32, vp]
@@ -144,10 +165,15 @@ def config_for(wl, flags=0, bias_correction=False) -> Config:
                        bias_correction=bias_correction, flags=flags)
 
 
-def workspace_bytes(shapes, cfg: Config) -> int:
+def workspace_bytes(shapes, cfg: Config, tuning: Tuning | None = None) -> int:
     out = ctypes.c_size_t(0)
-    _check(load().apollo_workspace_bytes(_shape_array(shapes), len(shapes), ctypes.byref(cfg), ctypes.byref(out)),
-           "apollo_workspace_bytes")
+    if tuning is None:
+        _check(load().apollo_workspace_bytes(_shape_array(shapes), len(shapes), ctypes.byref(cfg), ctypes.byref(out)),
+               "apollo_workspace_bytes")
+    else:
+        _check(load().apollo_workspace_bytes_tuned(_shape_array(shapes), len(shapes), ctypes.byref(cfg),
+                                                   ctypes.byref(tuning), ctypes.byref(out)),
+               "apollo_workspace_bytes_tuned")
     return out.value
 
 
@@ -200,19 +226,25 @@ def adamw_step(params, grads, ms, vs, t, lr, beta1=0.9, beta2=0.999, eps=1e-8, w
 class Apollo:
     """apollo_create / apollo_step over a list of CUDA tensors (same dtype, 2-D, contiguous)."""
 
-    def __init__(self, shapes, cfg: Config, device="cuda"):
+    def __init__(self, shapes, cfg: Config, device="cuda", tuning: Tuning | None = None):
         self.lib = load()
         self.shapes = [(int(r), int(c)) for r, c in shapes]
         self.cfg = cfg
         self.device = torch.device(device)
-        nbytes = workspace_bytes(self.shapes, cfg)
+        nbytes = workspace_bytes(self.shapes, cfg, tuning)
+        self.workspace_bytes = nbytes
         with torch.cuda.device(self.device):
             self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
             base = self.workspace.data_ptr()
             self._ws_ptr = (base + 255) // 256 * 256
             ctx = ctypes.c_void_p()
-            _check(self.lib.apollo_create(ctypes.byref(ctx), _shape_array(self.shapes), len(self.shapes),
-                                          ctypes.byref(cfg), self._ws_ptr, nbytes), "apollo_create")
+            if tuning is None:
+                _check(self.lib.apollo_create(ctypes.byref(ctx), _shape_array(self.shapes), len(self.shapes),
+                                              ctypes.byref(cfg), self._ws_ptr, nbytes), "apollo_create")
+            else:
+                _check(self.lib.apollo_create_tuned(ctypes.byref(ctx), _shape_array(self.shapes), len(self.shapes),
+                                                    ctypes.byref(cfg), ctypes.byref(tuning), self._ws_ptr, nbytes),
+                       "apollo_create_tuned")
         self.ctx = ctx
         self._delta = None
         self._w_arr = (ctypes.c_void_p * len(self.shapes))()

@@ -30,9 +30,13 @@ struct StageGroup {   // matrices whose staged P share one filling of the stagin
 struct Plan {
     std::vector<MatPlan> mats;
     size_t off_status, off_descs, off_prefix[4], off_tmaps, off_stage, stage_bytes, zero_begin, zero_end, total;
+    size_t off_tmats, off_counters, counter_bytes;
     bool any_repitch;
     int64_t tiles[4];   // stream, simt, tensor, update
     std::vector<StageGroup> groups;
+    TcTiling tc;                    // tiling and mode of the tensor-core projection
+    std::vector<int32_t> tensor_mats;   // tensor ordinal -> matrix index
+    std::vector<int32_t> tq_prefix;     // matrix index -> number of tensor-path matrices before it
 };
 
 int validate_config(const apollo_config* cfg)
@@ -51,11 +55,17 @@ int validate_config(const apollo_config* cfg)
     return APOLLO_OK;
 }
 
-int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cfg, Plan& plan)
+int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cfg, const apollo_tuning* tuning,
+              Plan& plan)
 {
     if (!shapes || n_mat < 1) return APOLLO_ERR_INVALID_ARG;
     int rc = validate_config(cfg);
     if (rc != APOLLO_OK) return rc;
+    plan.tc = TcTiling{};
+    if (cfg->rank >= 16) {
+        rc = tensor_path_configure(cfg->rank, cfg->flags, tuning, &plan.tc);
+        if (rc != APOLLO_OK) return rc;
+    }
     plan.mats.resize(n_mat);
     for (int t = 0; t < 4; ++t) plan.tiles[t] = 0;
     const int r = cfg->rank;
@@ -82,7 +92,7 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
             }
         } else if (tensor_path_supports(p.rows, p.cols, r, cfg->dtype) && !(cfg->flags & APOLLO_FLAG_NO_TENSOR_CORES)) {
             p.path = PATH_TENSOR;
-            tensor_path_tiling(p.rows, p.cols, r, &p.tiles_n, &p.tiles_k, &p.slices, &p.g2_slices);
+            tensor_path_tiling(p.rows, p.cols, r, plan.tc, &p.tiles_n, &p.tiles_k, &p.slices, &p.g2_slices);
         } else {
             p.path = PATH_SIMT;
             p.tiles_n = (p.n + SIMT_BN - 1) / SIMT_BN;
@@ -103,19 +113,46 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
     plan.off_descs = off; off = align_up(off + sizeof(MatDesc) * (size_t)n_mat);
     for (int t = 0; t < 4; ++t) { plan.off_prefix[t] = off; off = align_up(off + sizeof(int) * ((size_t)n_mat + 1)); }
     plan.off_tmaps = off; off = align_up(off + 256 * (size_t)n_mat);
-    // staging groups: consecutive matrices whose P fit the staging budget together
+    // tensor-path matrices in list order
+    plan.tensor_mats.clear();
+    plan.tq_prefix.assign((size_t)n_mat + 1, 0);
+    for (int i = 0; i < n_mat; ++i) {
+        plan.tq_prefix[i] = (int32_t)plan.tensor_mats.size();
+        if (plan.mats[i].path == PATH_TENSOR) plan.tensor_mats.push_back(i);
+    }
+    plan.tq_prefix[n_mat] = (int32_t)plan.tensor_mats.size();
+    plan.off_tmats = off; off = align_up(off + sizeof(int32_t) * (plan.tensor_mats.size() + 1));
+    // generator counters of the pair kernel: ticket, then per matrix pieces written and tiles read
+    plan.counter_bytes = align_up(sizeof(uint32_t) * (1 + 2 * (size_t)n_mat));
+    plan.off_counters = off; off += plan.counter_bytes;
+    // The P scratch.  kept: every matrix owns a slot.  gen: a ring of equal slots over the tensor ordinals.
+    // Otherwise staging groups: consecutive matrices whose P fit the scratch together, filled group by group.
     plan.groups.clear();
     plan.stage_bytes = 0;
-    {
-        const size_t budget = tensor_path_stage_budget();
+    if (plan.tc.gen && !plan.tensor_mats.empty()) {
+        size_t slot = 0;
+        for (int i : plan.tensor_mats) {
+            const size_t need = align_up(tensor_path_stage_bytes(plan.mats[i].rows, plan.mats[i].cols, r));
+            if (need > slot) slot = need;
+        }
+        int64_t slots = plan.tc.scratch_bytes / (int64_t)slot;
+        if (slots < 2) slots = 2;
+        if (slots > (int64_t)plan.tensor_mats.size()) slots = (int64_t)plan.tensor_mats.size();
+        plan.tc.slots = (int32_t)slots;
+        for (size_t q = 0; q < plan.tensor_mats.size(); ++q)
+            plan.mats[plan.tensor_mats[q]].off_pstage = (q % (size_t)slots) * slot;
+        plan.stage_bytes = (size_t)slots * slot;
+        plan.groups.push_back(StageGroup{ 0, n_mat, 0, (int)plan.tiles[PATH_TENSOR] });
+    } else {
+        const size_t budget = plan.tc.keep ? (size_t)-1 : (size_t)plan.tc.scratch_bytes;
         StageGroup g = { 0, 0, 0, 0 };
         size_t used = 0;
         int tile_at = 0;
         for (int i = 0; i < n_mat; ++i) {
             MatPlan& p = plan.mats[i];
             const bool tensor = p.path == PATH_TENSOR;
-            const size_t need = tensor && tensor_path_staged() ? align_up(tensor_path_stage_bytes(p.rows, p.cols, r)) : 0;
-            if (used > 0 && used + need > budget) {
+            const size_t need = tensor && plan.tc.staged ? align_up(tensor_path_stage_bytes(p.rows, p.cols, r)) : 0;
+            if (used > 0 && (used >= budget || need > budget - used)) {
                 g.mat_end = i; g.tile_end = tile_at;
                 plan.groups.push_back(g);
                 g.mat_begin = i; g.tile_begin = tile_at;
@@ -172,10 +209,22 @@ static bool cuda_ok(cudaError_t e)
     return true;
 }
 
+// Pinned host staging of the descriptor table and the tensor maps: an upload from pageable memory would
+// make cudaMemcpyAsync wait for the stream.  Two slots, each reused once the copy recorded in it is done.
+struct UploadSlot {
+    char* host;
+    cudaEvent_t done;
+    bool in_flight;
+};
+
 struct apollo_ctx {
     apollo_config cfg;
     int32_t n_mat;
     Plan plan;
+    TcLaunchState tc_state;
+    std::vector<char> h_maps;        // 2 x n_mat tensor maps of 128 bytes (G, staged P)
+    UploadSlot upload[2];
+    int upload_next;
     std::vector<MatDesc> h_descs;
     std::vector<int> h_prefix[4];
     char* ws;
@@ -218,25 +267,38 @@ const char* apollo_strerror(int code)
     }
 }
 
-int apollo_workspace_bytes(const apollo_shape* shapes, int32_t n_matrices, const apollo_config* cfg,
-                           size_t* out_bytes)
+int apollo_workspace_bytes_tuned(const apollo_shape* shapes, int32_t n_matrices, const apollo_config* cfg,
+                                 const apollo_tuning* tuning, size_t* out_bytes)
 {
     if (!out_bytes) return APOLLO_ERR_INVALID_ARG;
     Plan plan;
-    const int rc = make_plan(shapes, n_matrices, cfg, plan);
+    const int rc = make_plan(shapes, n_matrices, cfg, tuning, plan);
     if (rc != APOLLO_OK) return rc;
     *out_bytes = plan.total;
     return APOLLO_OK;
 }
 
+int apollo_workspace_bytes(const apollo_shape* shapes, int32_t n_matrices, const apollo_config* cfg,
+                           size_t* out_bytes)
+{
+    return apollo_workspace_bytes_tuned(shapes, n_matrices, cfg, nullptr, out_bytes);
+}
+
 int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_matrices,
                   const apollo_config* cfg, void* d_workspace, size_t workspace_bytes)
+{
+    return apollo_create_tuned(out_ctx, shapes, n_matrices, cfg, nullptr, d_workspace, workspace_bytes);
+}
+
+int apollo_create_tuned(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_matrices,
+                        const apollo_config* cfg, const apollo_tuning* tuning, void* d_workspace,
+                        size_t workspace_bytes)
 {
     if (!out_ctx) return APOLLO_ERR_INVALID_ARG;
     *out_ctx = nullptr;
     apollo_ctx* ctx = new (std::nothrow) apollo_ctx();
     if (!ctx) return APOLLO_ERR_INVALID_ARG;
-    int rc = make_plan(shapes, n_matrices, cfg, ctx->plan);
+    int rc = make_plan(shapes, n_matrices, cfg, tuning, ctx->plan);
     if (rc != APOLLO_OK) { delete ctx; return rc; }
     if (!d_workspace) { delete ctx; return APOLLO_ERR_INVALID_ARG; }
     if (((uintptr_t)d_workspace % ALIGN) != 0 || workspace_bytes < ctx->plan.total) { delete ctx; return APOLLO_ERR_WORKSPACE; }
@@ -297,6 +359,22 @@ int apollo_create(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_t n_ma
             ctx->h_prefix[t][i + 1] = ctx->h_prefix[t][i] + (p.path == t ? (int)p.proj_tiles : 0);
         ctx->h_prefix[3][i + 1] = ctx->h_prefix[3][i] + (int)p.update_tiles;
     }
+    ctx->tc_state = TcLaunchState{ false, 0 };
+    ctx->h_maps.assign(256 * (size_t)n_matrices, 0);
+    ctx->upload_next = 0;
+    for (UploadSlot& u : ctx->upload) {
+        u.host = nullptr; u.done = nullptr; u.in_flight = false;
+        void* host = nullptr;
+        if (cudaHostAlloc(&host, sizeof(MatDesc) * (size_t)n_matrices + 256 * (size_t)n_matrices, cudaHostAllocDefault) ==
+                cudaSuccess &&
+            cudaEventCreateWithFlags(&u.done, cudaEventDisableTiming) == cudaSuccess) {
+            u.host = static_cast<char*>(host);
+        } else {
+            cudaGetLastError();          // no pinned memory to be had: uploads go from pageable memory
+            if (host) cudaFreeHost(host);
+            u.done = nullptr;
+        }
+    }
     ctx->delta.assign(n_matrices, nullptr);
     ctx->delta_on = false;
     ctx->first = true;
@@ -317,6 +395,13 @@ int apollo_destroy(apollo_ctx* ctx)
     if (ctx->timing_ready)
         for (int sl = 0; sl < APOLLO_TIMING_SLOTS; ++sl)
             for (int e = 0; e < 4; ++e) cudaEventDestroy(ctx->ev[sl][e]);
+    for (UploadSlot& u : ctx->upload) {
+        if (u.host) {
+            if (u.in_flight) cudaEventSynchronize(u.done);
+            cudaEventDestroy(u.done);
+            cudaFreeHost(u.host);
+        }
+    }
     delete ctx;
     return APOLLO_OK;
 }
@@ -371,22 +456,45 @@ static int step_range(apollo_ctx* ctx, int first, int count, void* const* d_W, c
             if (cudaMemcpyAsync(ctx->d_prefix[t], ctx->h_prefix[t].data(), sizeof(int) * (ctx->n_mat + 1),
                                 cudaMemcpyHostToDevice, stream) != cudaSuccess)
                 return APOLLO_ERR_CUDA;
+        if (!plan.tensor_mats.empty() &&
+            cudaMemcpyAsync(ctx->ws + plan.off_tmats, plan.tensor_mats.data(), sizeof(int32_t) * plan.tensor_mats.size(),
+                            cudaMemcpyHostToDevice, stream) != cudaSuccess)
+            return APOLLO_ERR_CUDA;
     }
+    // A tensor map depends on the matrix's G address alone (the map of its P slot never changes): matrices
+    // whose G moved get a new one; the whole table travels with the descriptors when anything changed.
     bool changed = ctx->descs_dirty;
     for (int i = first; i < last; ++i) {
         MatDesc& d = ctx->h_descs[i];
-        if (d.W != d_W[i - first] || d.G != d_G[i - first] || d.dW != ctx->delta[i]) {
+        const bool g_moved = d.G != d_G[i - first];
+        if (d.W != d_W[i - first] || g_moved || d.dW != ctx->delta[i]) {
             d.W = d_W[i - first]; d.G = d_G[i - first]; d.dW = ctx->delta[i];
             changed = true;
         }
+        if ((g_moved || ctx->first) && d.path == PATH_TENSOR) {
+            const int rc = tensor_path_prepare(&d, 1, cfg.rank, plan.tc, ctx->h_maps.data() + 256 * (size_t)i);
+            if (rc != APOLLO_OK) return rc;
+        }
     }
     if (changed) {
-        const int rc = tensor_path_prepare(ctx->h_descs.data(), ctx->n_mat, cfg.rank,
-                                           ctx->ws + plan.off_tmaps, stream);
-        if (rc != APOLLO_OK) return rc;
-        if (cudaMemcpyAsync(ctx->d_descs, ctx->h_descs.data(), sizeof(MatDesc) * ctx->n_mat,
-                            cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        const size_t desc_bytes = sizeof(MatDesc) * (size_t)ctx->n_mat, map_bytes = 256 * (size_t)ctx->n_mat;
+        const char* src_descs = reinterpret_cast<const char*>(ctx->h_descs.data());
+        const char* src_maps = ctx->h_maps.data();
+        UploadSlot& u = ctx->upload[ctx->upload_next];
+        if (u.host) {
+            if (u.in_flight && cudaEventSynchronize(u.done) != cudaSuccess) return APOLLO_ERR_CUDA;   // two uploads ago
+            std::memcpy(u.host, src_descs, desc_bytes);
+            std::memcpy(u.host + desc_bytes, src_maps, map_bytes);
+            src_descs = u.host; src_maps = u.host + desc_bytes;
+        }
+        if (cudaMemcpyAsync(ctx->d_descs, src_descs, desc_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+            cudaMemcpyAsync(ctx->ws + plan.off_tmaps, src_maps, map_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
             return APOLLO_ERR_CUDA;
+        if (u.host) {
+            if (cudaEventRecord(u.done, stream) != cudaSuccess) return APOLLO_ERR_CUDA;
+            u.in_flight = true;
+            ctx->upload_next ^= 1;
+        }
         ctx->descs_dirty = false;
     }
 
@@ -429,41 +537,56 @@ static int step_range(apollo_ctx* ctx, int first, int count, void* const* d_W, c
             launch_repitch(ctx->d_descs, first, count, stream);
             ++launches;
         }
-        for (const StageGroup& g : plan.groups) {
-            // the part of this staging group inside the range
-            const int mb = g.mat_begin > first ? g.mat_begin : first;
-            const int me = g.mat_end < last ? g.mat_end : last;
-            if (me <= mb || !tiles_of(PATH_TENSOR, mb, me, tb, te)) continue;
-            if (tensor_path_staged()) {
-                // P changes only with the epoch (every T steps).  When every matrix owns its staging slot
-                // (one group), a slot filled in this epoch is read again instead of being regenerated.
-                // A projection supplied by the caller is converted every step: its buffer may have been rewritten.
-                int lo = mb, hi = me;
-                if (plan.groups.size() == 1) {
-                    auto fresh = [&](int i) {
-                        const MatDesc& d = ctx->h_descs[i];
-                        return d.path != PATH_TENSOR || (!d.ext_p && ctx->staged_epoch[i] == (int64_t)sp.epoch);
-                    };
-                    while (lo < hi && fresh(lo)) ++lo;
-                    while (hi > lo && fresh(hi - 1)) --hi;
-                    for (int i = lo; i < hi; ++i) ctx->staged_epoch[i] = (int64_t)sp.epoch;
-                }
-                if (hi > lo) {
-                    launch_generate_p(ctx->d_descs, lo, hi, sp, stream);
-                    ++launches;
-                }
-            }
-            launch_project_tensor(ctx->d_descs, ctx->d_prefix[PATH_TENSOR], ctx->n_mat, tb, te, sp, ctx->sm_count,
-                                  ctx->d_status, stream);
+        const TcTiling& tc = plan.tc;
+        GenArgs gen = {};
+        if (tc.gen) {
+            // one launch over the range: spare warps of the kernel regenerate every matrix's P from the seed,
+            // a few matrices ahead of the tiles that read it, through the ring of slots in the scratch
+            uint32_t* counters = reinterpret_cast<uint32_t*>(ctx->ws + plan.off_counters);
+            if (cudaMemsetAsync(counters, 0, plan.counter_bytes, stream) != cudaSuccess) return APOLLO_ERR_CUDA;
+            gen.mats = reinterpret_cast<const int32_t*>(ctx->ws + plan.off_tmats);
+            gen.q_begin = plan.tq_prefix[first]; gen.q_end = plan.tq_prefix[last];
+            gen.ticket = counters; gen.gen_done = counters + 1; gen.use_done = counters + 1 + ctx->n_mat;
+            launch_project_tensor(ctx->d_descs, ctx->d_prefix[PATH_TENSOR], ctx->n_mat, tb, te, sp, tc, gen,
+                                  ctx->tc_state, ctx->sm_count, ctx->d_status, stream);
             ++launches;
+        } else {
+            for (const StageGroup& g : plan.groups) {
+                // the part of this staging group inside the range
+                const int mb = g.mat_begin > first ? g.mat_begin : first;
+                const int me = g.mat_end < last ? g.mat_end : last;
+                if (me <= mb || !tiles_of(PATH_TENSOR, mb, me, tb, te)) continue;
+                if (tc.staged) {
+                    // P changes only with the epoch (every T steps).  When every matrix keeps its own slot
+                    // (APOLLO_FLAG_KEEP_P), a slot filled in this epoch is read again instead of being regenerated.
+                    // A projection supplied by the caller is converted every step: its buffer may have been rewritten.
+                    int lo = mb, hi = me;
+                    if (tc.keep) {
+                        auto fresh = [&](int i) {
+                            const MatDesc& d = ctx->h_descs[i];
+                            return d.path != PATH_TENSOR || (!d.ext_p && ctx->staged_epoch[i] == (int64_t)sp.epoch);
+                        };
+                        while (lo < hi && fresh(lo)) ++lo;
+                        while (hi > lo && fresh(hi - 1)) --hi;
+                        for (int i = lo; i < hi; ++i) ctx->staged_epoch[i] = (int64_t)sp.epoch;
+                    }
+                    if (hi > lo) {
+                        launch_generate_p(ctx->d_descs, lo, hi, sp, stream);
+                        ++launches;
+                    }
+                }
+                launch_project_tensor(ctx->d_descs, ctx->d_prefix[PATH_TENSOR], ctx->n_mat, tb, te, sp, tc, gen,
+                                      ctx->tc_state, ctx->sm_count, ctx->d_status, stream);
+                ++launches;
+            }
         }
     }
     if (ev) cudaEventRecord(ev[1], stream);
-    launch_finalize(ctx->d_descs, first, count, sp, stream);
+    launch_finalize(ctx->d_descs, first, count, sp, ctx->d_status, stream);
     ++launches;
     if (ev) cudaEventRecord(ev[2], stream);
     tiles_of(3, first, last, tb, te);
-    launch_update(cfg.dtype, ctx->d_descs, ctx->d_prefix[3], ctx->n_mat, tb, te, sp, ctx->sm_count, stream);
+    launch_update(cfg.dtype, ctx->d_descs, ctx->d_prefix[3], ctx->n_mat, tb, te, sp, ctx->sm_count, ctx->d_status, stream);
     ++launches;
     if (ev) cudaEventRecord(ev[3], stream);
     if (!cuda_ok(cudaGetLastError())) return APOLLO_ERR_CUDA;
@@ -613,7 +736,7 @@ int apollo_set_projection(apollo_ctx* ctx, int32_t matrix, const float* d_P)
     if (!ctx || matrix < 0 || matrix >= ctx->n_mat) return APOLLO_ERR_INVALID_ARG;
     if (d_P && ((uintptr_t)d_P % 4)) return APOLLO_ERR_ALIGN;
     MatDesc& d = ctx->h_descs[matrix];
-    if (d_P && d.path == PATH_TENSOR && !tensor_path_staged()) return APOLLO_ERR_UNSUPPORTED;
+    if (d_P && d.path == PATH_TENSOR && !ctx->plan.tc.staged) return APOLLO_ERR_UNSUPPORTED;
     d.ext_p = d_P;
     ctx->staged_epoch[matrix] = -1;
     d.r_scale = d_P ? 1.0f : (float)(1.0 / std::sqrt((double)ctx->cfg.rank));

@@ -131,15 +131,36 @@ inline void fill_round_keys(StepParams& sp)
     }
 }
 
-// Tiling of the tensor-core projection (one choice per context, set by the rank).
+// Tiling and mode of the tensor-core projection: one choice per context, made when it is created.
 struct TcTiling {
     int32_t r_slice;   // rows of R per tile = N of the MMA (multiple of 16, <= 256)
     int32_t nblk;      // 128-channel blocks per tile (1, 2 or 4); nblk * r_slice <= 512 TMEM columns
     int32_t stages;    // shared-memory pipeline depth
     int32_t smem_bytes;
-    int32_t staged;    // 0: P generated in shared memory; 1: P loaded from the staging buffer
+    int32_t staged;    // 0: P generated in shared memory; 1: P loaded from the scratch in the workspace
     int32_t pair;      // 1: the pair kernel (CTA pairs, cta_group::2); staged only
-    int32_t epi_prefetch; // pair kernel: the epilogue warps ask L2 for the moments one chunk ahead of their loads
+    int32_t epi_prefetch; // pair kernel: the epilogue warps ask L2 for the moments this many chunks ahead of their loads
+    int32_t keep;      // 1: every matrix owns a slot of the scratch, filled once per epoch (APOLLO_FLAG_KEEP_P)
+    int32_t gen;       // 1: spare warps of the pair kernel generate P into a ring of `slots` slots, ahead of its use
+    int32_t slots;     // gen: slots of the ring (matrix with tensor ordinal q uses slot q % slots)
+    int64_t scratch_bytes; // byte budget of the scratch when it is neither kept nor a ring (groups of matrices share it)
+};
+
+// What the generator warps of the pair kernel and the consumers of their output share (TcTiling::gen).
+// The counters are zeroed before every launch.
+constexpr int GEN_CHUNKS = 64;     // pieces a matrix's P is generated in; one ticket each
+struct GenArgs {
+    const int32_t* mats;   // tensor ordinal -> matrix index
+    int32_t q_begin, q_end;   // ordinals of the launch
+    uint32_t* ticket;      // next piece to generate: (ordinal - q_begin) * GEN_CHUNKS + chunk
+    uint32_t* gen_done;    // per matrix: pieces written
+    uint32_t* use_done;    // per matrix: tiles whose MMAs have read their last P tile
+};
+
+// Per-context launch state of the tensor path (function attributes are per device; set once per context).
+struct TcLaunchState {
+    bool attr_set;
+    int max_pairs;
 };
 
 // Device status word values.

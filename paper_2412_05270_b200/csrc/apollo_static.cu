@@ -64,7 +64,10 @@ extern "C" int apollo_mini_step_static(void* d_W, const void* d_G, int64_t rows,
     if (!std::isfinite(cfg->alpha) || !std::isfinite(cfg->gamma) || !std::isfinite(cfg->eps) || cfg->eps < 0.f ||
         !(cfg->beta1 >= 0.f && cfg->beta1 <= 1.f) || !(cfg->beta2 >= 0.f && cfg->beta2 <= 1.f))
         return APOLLO_ERR_INVALID_ARG;
+    if (cfg->bias_correction != 0 && cfg->bias_correction != 1) return APOLLO_ERR_INVALID_ARG;
     if (cfg->bias_correction && (cfg->beta1 >= 1.f || cfg->beta2 >= 1.f)) return APOLLO_ERR_INVALID_ARG;
+    // d_M and d_V are n floats: a caller that asks for two-byte moments would be overrun
+    if (cfg->flags & APOLLO_FLAG_BF16_STATES) return APOLLO_ERR_INVALID_ARG;
     if (rows < 1 || cols < 1 || rows > INT32_MAX || cols > INT32_MAX) return APOLLO_ERR_SHAPE;
     if (((uintptr_t)d_W % 16) || ((uintptr_t)d_G % 16) || ((uintptr_t)d_M % 16) || ((uintptr_t)d_V % 16) ||
         ((uintptr_t)d_prev_norm % 4))
@@ -160,8 +163,8 @@ extern "C" int apollo_mini_step_static(void* d_W, const void* d_G, int64_t rows,
     static_setup_kernel<<<1, 1, 0, stream>>>(d, (int)proj_tiles, (int)update_tiles);
     launch_project_stream(cfg->dtype, d_desc, reinterpret_cast<const int*>(base + OFF_PREFIX_P), 1,
                           0, (int)proj_tiles, sp, sm_count, stream);
-    launch_finalize(d_desc, 0, 1, sp, stream);
+    launch_finalize(d_desc, 0, 1, sp, nullptr, stream);
     launch_update(cfg->dtype, d_desc, reinterpret_cast<const int*>(base + OFF_PREFIX_U), 1, 0, (int)update_tiles,
-                  sp, sm_count, stream);
+                  sp, sm_count, nullptr, stream);
     return cudaGetLastError() == cudaSuccess ? APOLLO_OK : APOLLO_ERR_CUDA;
 }

@@ -1,5 +1,6 @@
 // Host-callable launchers of the kernels (one grouped launch each over the parameter list).
 #pragma once
+#include "../../include/apollo.h"
 #include "apollo_internal.h"
 
 namespace apollo {
@@ -12,9 +13,13 @@ void launch_project_stream(int dtype, const MatDesc* d_descs, const int* d_prefi
                            const StepParams& sp, int sm_count, cudaStream_t stream);
 void launch_project_simt(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int tile_begin, int tile_end,
                          const StepParams& sp, int sm_count, cudaStream_t stream);
-void launch_finalize(const MatDesc* d_descs, int first, int count, const StepParams& sp, cudaStream_t stream);
+// d_status (may be null): the context's status word.  When it is not STATUS_OK -- a bounded wait of the
+// projection gave up -- finalize and update return without writing, so that a step whose projection is
+// incomplete leaves the weights, the scales and the limiter's norm as they were.
+void launch_finalize(const MatDesc* d_descs, int first, int count, const StepParams& sp, const int32_t* d_status,
+                     cudaStream_t stream);
 void launch_update(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int tile_begin, int tile_end,
-                   const StepParams& sp, int sm_count, cudaStream_t stream);
+                   const StepParams& sp, int sm_count, const int32_t* d_status, cudaStream_t stream);
 
 
 // bfloat16 -> float copy (observability of bfloat16 states).
@@ -26,16 +31,16 @@ void launch_state_copy(void* d_lib, void* d_dense, int rank, int n, int ns, bool
 
 // Tensor-core projection (TMA + tcgen05 + TMEM).
 bool tensor_path_supports(int rows, int cols, int rank, int dtype);
-void tensor_path_tiling(int rows, int cols, int rank, int32_t* tiles_n, int32_t* tiles_k, int32_t* slices,
-                        int32_t* g2_slices);
-// L2 staging of P: whether it is on, the byte budget of the staging buffer, and the bytes
-// one matrix needs in it (rank x round_up(m, 64) bf16).
-bool tensor_path_staged();
-size_t tensor_path_stage_budget();
+// The tiling and mode for a rank, the context's flags and the caller's tuning (may be null):
+// APOLLO_OK, or APOLLO_ERR_INVALID_ARG for a tuning value out of range.
+int tensor_path_configure(int rank, uint32_t flags, const apollo_tuning* tuning, TcTiling* out);
+void tensor_path_tiling(int rows, int cols, int rank, const TcTiling& tl, int32_t* tiles_n, int32_t* tiles_k,
+                        int32_t* slices, int32_t* g2_slices);
+// Bytes one matrix's P needs in the scratch (rank x round_up(m, 64) bf16).
 size_t tensor_path_stage_bytes(int rows, int cols, int rank);
 // Encodes the tensor maps of the matrices on the tensor path (G at +0, staged P at +128 of
-// each 256-byte slot) and queues their upload to `d_tmaps`.  Returns an APOLLO_* code.
-int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, void* d_tmaps, cudaStream_t stream);
+// each 256-byte slot) into h_maps (2 x n_mat maps of 128 bytes, host).  Returns an APOLLO_* code.
+int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, const TcTiling& tl, void* h_maps);
 // Copies the gradients whose row pitch is not a multiple of 16 bytes into their padded buffers.
 void launch_repitch(const MatDesc* d_descs, int first, int count, cudaStream_t stream);
 // Fills the staging buffer with the standard normals of matrices [mat_begin, mat_end).
@@ -44,6 +49,7 @@ void launch_bounded_wait_selftest(int32_t* d_status, cudaStream_t stream);
 void launch_generate_p(const MatDesc* d_descs, int mat_begin, int mat_end, const StepParams& sp, cudaStream_t stream);
 // Projection over tiles [tile_begin, tile_end) of the tensor-path prefix table.
 void launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_mat, int tile_begin, int tile_end,
-                           const StepParams& sp, int sm_count, int32_t* d_status, cudaStream_t stream);
+                           const StepParams& sp, const TcTiling& tl, const GenArgs& gen, TcLaunchState& state,
+                           int sm_count, int32_t* d_status, cudaStream_t stream);
 
 }  // namespace apollo

@@ -359,9 +359,10 @@ project_simt_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
 constexpr int FINALIZE_THREADS = 1024;
 
 __global__ void __launch_bounds__(FINALIZE_THREADS)
-finalize_kernel(const MatDesc* __restrict__ descs, int first, StepParams sp)
+finalize_kernel(const MatDesc* __restrict__ descs, int first, StepParams sp, const int32_t* __restrict__ status)
 {
     __shared__ double scratch[32];
+    if (status && *status != STATUS_OK) return;      // the projection did not complete: leave s, prev and scal alone
     const MatDesc& d = descs[first + blockIdx.x];
     const int n = d.n;
     const bool tensor_mode = sp.mode == 1;
@@ -445,8 +446,9 @@ __device__ __forceinline__ void store1(__nv_bfloat16* p, float v) { *p = __float
 template <typename T>
 __global__ void __launch_bounds__(UPDATE_THREADS)
 update_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix, int n_mat,
-              int tile_begin, int tile_end, StepParams sp)
+              int tile_begin, int tile_end, StepParams sp, const int32_t* __restrict__ status)
 {
+    if (status && *status != STATUS_OK) return;      // the projection did not complete: leave W alone
     for (int tile = tile_begin + blockIdx.x; tile < tile_end; tile += gridDim.x) {
         const int mat = find_matrix(prefix, n_mat, tile);
         const MatDesc& d = descs[mat];
@@ -681,22 +683,23 @@ void launch_project_simt(int dtype, const MatDesc* d_descs, const int* d_prefix,
         project_simt_kernel<__nv_bfloat16><<<grid, SIMT_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end, sp);
 }
 
-void launch_finalize(const MatDesc* d_descs, int first, int count, const StepParams& sp, cudaStream_t stream)
+void launch_finalize(const MatDesc* d_descs, int first, int count, const StepParams& sp, const int32_t* d_status,
+                     cudaStream_t stream)
 {
     if (count <= 0) return;
-    finalize_kernel<<<count, FINALIZE_THREADS, 0, stream>>>(d_descs, first, sp);
+    finalize_kernel<<<count, FINALIZE_THREADS, 0, stream>>>(d_descs, first, sp, d_status);
 }
 
 void launch_update(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int tile_begin, int tile_end,
-                   const StepParams& sp, int sm_count, cudaStream_t stream)
+                   const StepParams& sp, int sm_count, const int32_t* d_status, cudaStream_t stream)
 {
     const int total_tiles = tile_end - tile_begin;
     if (total_tiles <= 0) return;
     const int grid = grid_for(total_tiles, 8, sm_count);
     if (dtype == 0)
-        update_kernel<float><<<grid, UPDATE_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end, sp);
+        update_kernel<float><<<grid, UPDATE_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end, sp, d_status);
     else
-        update_kernel<__nv_bfloat16><<<grid, UPDATE_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end, sp);
+        update_kernel<__nv_bfloat16><<<grid, UPDATE_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end, sp, d_status);
 }
 
 }  // namespace apollo

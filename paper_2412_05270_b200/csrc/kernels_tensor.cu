@@ -1,7 +1,9 @@
 // Tensor-core projection: R = P G on tcgen05 with TMEM accumulators (Algorithm 1, step 1),
 // with the moment update and the per-channel norm sums fused into the epilogue (Algorithm 1,
-// step 2; Eq. 5).  P is either loaded from a staging buffer that generate_p_kernel fills once
-// per epoch (default) or generated straight into shared memory by every CTA.
+// step 2; Eq. 5).  P tiles come from a scratch in the workspace that L2 keeps: spare warps of the pair
+// kernel regenerate every matrix's P from the seed a few matrices ahead of its use (default), or
+// generate_p_kernel fills it (once per epoch with APOLLO_FLAG_KEEP_P, else group by group); the ring
+// kernel can also generate them straight into shared memory.
 //
 // Two kernels share this file: project_pair_kernel (default when P is staged; CTA pairs, described
 // above its definition) and project_tensor_kernel, the single-CTA ring kernel described here.
@@ -24,7 +26,6 @@
 #include "kernels.h"
 
 #include <cuda.h>
-#include <cstdlib>
 #include <cstring>
 #include <vector>
 
@@ -49,47 +50,6 @@ constexpr int TC_PREFETCH = 2;             // k-blocks of G asked into L2 ahead 
 constexpr uint32_t TC_PACE_CAP = 1u << 12; // polls (100 ns apart) of the prefetchers' pacing wait; expiry is harmless
 constexpr uint32_t TC_WAIT_CAP = 1u << 20;   // polls before a wait gives up (normal waits are far below 1 ms)
 
-TcTiling choose_tiling(int rank)
-{
-    TcTiling t;
-    t.r_slice = rank <= 256 ? rank : rank / 2;
-    if (const char* env = std::getenv("APOLLO_TC_RSLICE")) {
-        const int v = std::atoi(env);
-        if (v >= 16 && v <= 256 && v % 16 == 0 && rank % v == 0) t.r_slice = v;
-    }
-    const int fit = 512 / t.r_slice;
-    t.nblk = fit >= 4 ? 4 : (fit >= 2 ? 2 : 1);
-    if (const char* env = std::getenv("APOLLO_TC_NBLK")) {
-        const int v = std::atoi(env);
-        if ((v == 1 || v == 2 || v == 4) && v * t.r_slice <= 512) t.nblk = v;
-    }
-    t.staged = tensor_path_staged() ? 1 : 0;
-    t.pair = 0;
-    t.epi_prefetch = 1;
-    // Staged P has two kernels: the pair kernel (default; faster on every list measured) and the
-    // single-CTA ring kernel (APOLLO_TC_KERNEL=ring), which is also the one that can generate P itself.
-    const char* kernel = std::getenv("APOLLO_TC_KERNEL");
-    if (t.staged && !(kernel && std::strcmp(kernel, "ring") == 0)) {
-        // pair tile: 256 channels (128 per CTA) x r_slice rows, accumulator double buffered
-        t.pair = 1;
-        t.nblk = 2;
-        const int stage = 128 * TC_BK * 2 + (t.r_slice / 2) * 128;
-        t.stages = (TC_MAX_SMEM - 1536) / stage;
-        if (t.stages > 8) t.stages = 8;
-        t.smem_bytes = t.stages * stage + 1536;
-        if (const char* env = std::getenv("APOLLO_TC_EPI_PREFETCH")) {
-            const int v = std::atoi(env);
-            if (v >= 0 && v <= 8) t.epi_prefetch = v;
-        }
-        return t;
-    }
-    const int stage = t.nblk * TC_BLOCK_BYTES + t.r_slice * 128;
-    t.stages = (TC_MAX_SMEM - TC_MISC_BYTES) / stage;
-    if (t.stages > 4) t.stages = 4;
-    t.smem_bytes = t.stages * stage + TC_MISC_BYTES;
-    return t;
-}
-
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -109,28 +69,58 @@ EncodeTiledFn encode_fn()
 
 }  // namespace
 
-// P tiles either come from a per-step staging buffer that stays in L2 (default) or are
-// generated in shared memory by every CTA that needs them (APOLLO_P_STAGING=0).
-bool tensor_path_staged()
-{
-    const char* env = std::getenv("APOLLO_P_STAGING");
-    return !(env && env[0] == '0');
-}
-
-size_t tensor_path_stage_budget()
-{
-    size_t mb = 512;
-    if (const char* env = std::getenv("APOLLO_P_STAGING_MB")) {
-        const long v = std::atol(env);
-        if (v >= 1 && v <= 65536) mb = (size_t)v;
-    }
-    return mb << 20;
-}
-
+// Bytes one matrix's P takes in the scratch: rank rows of round_up(m, 64) bfloat16 standard normals.
 size_t tensor_path_stage_bytes(int rows, int cols, int rank)
 {
     const int m = rows > cols ? cols : rows;
     return (size_t)rank * (size_t)((m + 63) / 64 * 64) * 2;
+}
+
+int tensor_path_configure(int rank, uint32_t flags, const apollo_tuning* tuning, TcTiling* out)
+{
+    static const apollo_tuning defaults = {};
+    const apollo_tuning& tu = tuning ? *tuning : defaults;
+    TcTiling t = {};
+    if (tu.kernel != APOLLO_TC_KERNEL_PAIR && tu.kernel != APOLLO_TC_KERNEL_RING) return APOLLO_ERR_INVALID_ARG;
+    if (tu.p_source != APOLLO_P_SCRATCH && tu.p_source != APOLLO_P_SHARED) return APOLLO_ERR_INVALID_ARG;
+    if (tu.p_generator != 0 && tu.p_generator != 1) return APOLLO_ERR_INVALID_ARG;
+    if (tu.scratch_mb < 0 || tu.scratch_mb > 65536 || tu.reserved != 0) return APOLLO_ERR_INVALID_ARG;
+    if (tu.epi_prefetch < 0 || tu.epi_prefetch > 9) return APOLLO_ERR_INVALID_ARG;
+    t.r_slice = rank <= 256 ? rank : rank / 2;
+    if (tu.r_slice != 0) {
+        if (tu.r_slice < 16 || tu.r_slice > 256 || tu.r_slice % 16 || rank % tu.r_slice) return APOLLO_ERR_INVALID_ARG;
+        t.r_slice = tu.r_slice;
+    }
+    const int fit = 512 / t.r_slice;
+    t.nblk = fit >= 4 ? 4 : (fit >= 2 ? 2 : 1);
+    if (tu.nblk != 0) {
+        if ((tu.nblk != 1 && tu.nblk != 2 && tu.nblk != 4) || tu.nblk * t.r_slice > 512) return APOLLO_ERR_INVALID_ARG;
+        t.nblk = tu.nblk;
+    }
+    t.staged = tu.p_source == APOLLO_P_SCRATCH ? 1 : 0;
+    t.keep = t.staged && (flags & APOLLO_FLAG_KEEP_P) ? 1 : 0;
+    t.scratch_bytes = (int64_t)(tu.scratch_mb ? tu.scratch_mb : 32) << 20;
+    t.epi_prefetch = tu.epi_prefetch ? tu.epi_prefetch - 1 : 1;
+    // Staged P has two kernels: the pair kernel (default; faster on every list measured) and the single-CTA
+    // ring kernel, which is also the one that can generate P in shared memory.
+    if (t.staged && tu.kernel == APOLLO_TC_KERNEL_PAIR) {   // (APOLLO_P_SHARED always runs on the ring kernel)
+        // pair tile: 256 channels (128 per CTA) x r_slice rows, accumulator double buffered
+        t.pair = 1;
+        t.nblk = 2;
+        t.gen = !t.keep && tu.p_generator == 0 ? 1 : 0;
+        const int stage = 128 * TC_BK * 2 + (t.r_slice / 2) * 128;
+        t.stages = (TC_MAX_SMEM - 1536) / stage;
+        if (t.stages > 8) t.stages = 8;
+        t.smem_bytes = t.stages * stage + 1536;
+        *out = t;
+        return APOLLO_OK;
+    }
+    const int stage = t.nblk * TC_BLOCK_BYTES + t.r_slice * 128;
+    t.stages = (TC_MAX_SMEM - TC_MISC_BYTES) / stage;
+    if (t.stages > 4) t.stages = 4;
+    t.smem_bytes = t.stages * stage + TC_MISC_BYTES;
+    *out = t;
+    return APOLLO_OK;
 }
 
 bool tensor_path_supports(int rows, int cols, int rank, int dtype)
@@ -142,10 +132,9 @@ bool tensor_path_supports(int rows, int cols, int rank, int dtype)
     return true;
 }
 
-void tensor_path_tiling(int rows, int cols, int rank, int32_t* tiles_n, int32_t* tiles_k, int32_t* slices,
-                        int32_t* g2_slices)
+void tensor_path_tiling(int rows, int cols, int rank, const TcTiling& t, int32_t* tiles_n, int32_t* tiles_k,
+                        int32_t* slices, int32_t* g2_slices)
 {
-    const TcTiling t = choose_tiling(rank);
     const int n = rows > cols ? rows : cols;
     *tiles_n = (n + t.nblk * 128 - 1) / (t.nblk * 128);
     *tiles_k = rank / t.r_slice;
@@ -155,16 +144,15 @@ void tensor_path_tiling(int rows, int cols, int rank, int32_t* tiles_n, int32_t*
     *g2_slices = t.pair && rows <= cols ? 4 : 1;
 }
 
-int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, void* d_tmaps, cudaStream_t stream)
+int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, const TcTiling& tl, void* h_maps)
 {
-    const TcTiling tl = choose_tiling(rank);
     bool any = false;
     for (int i = 0; i < n_mat; ++i) any |= h_descs[i].path == PATH_TENSOR;
     if (!any) return APOLLO_OK;
     EncodeTiledFn encode = encode_fn();
     if (!encode) return APOLLO_ERR_CUDA;
-    std::vector<CUtensorMap> maps(2 * (size_t)n_mat);
-    std::memset(maps.data(), 0, sizeof(CUtensorMap) * maps.size());
+    static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
+    CUtensorMap* maps = static_cast<CUtensorMap*>(h_maps);
     for (int i = 0; i < n_mat; ++i) {
         const MatDesc& d = h_descs[i];
         if (d.path != PATH_TENSOR) continue;
@@ -190,10 +178,6 @@ int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, void* d_tmaps, cu
             if (rp != CUDA_SUCCESS) return APOLLO_ERR_CUDA;
         }
     }
-    static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
-    if (cudaMemcpyAsync(d_tmaps, maps.data(), sizeof(CUtensorMap) * maps.size(), cudaMemcpyHostToDevice, stream) !=
-        cudaSuccess)
-        return APOLLO_ERR_CUDA;
     return APOLLO_OK;
 }
 
@@ -235,6 +219,56 @@ __device__ __forceinline__ void drain_phase(uint32_t bar, uint32_t parity)
 {
     for (uint32_t i = 0; i < TC_WAIT_CAP; ++i)
         if (ptx::mbar_try_wait(bar, parity)) return;
+}
+
+// Counters in global memory that CTAs of one launch signal each other through (P generated by spare warps).
+__device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* p)
+{
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void red_release_gpu_add(uint32_t* p, uint32_t v)
+{
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+// Bounded wait until *counter >= target.  All CTAs of the launch are resident (the grid is sized by the
+// occupancy query), so the writers run; the bound covers the case that one of them gave up.  A set status
+// word ends the wait at once.  false = gave up (abort flag and status word are set).
+__device__ __forceinline__ bool wait_counter(const uint32_t* counter, uint32_t target, volatile int* abort_flag,
+                                             int32_t* status)
+{
+    if (ld_acquire_gpu(counter) >= target) return true;
+    if (*abort_flag) return false;
+    for (uint32_t i = 0; i < TC_WAIT_CAP; ++i) {
+        __nanosleep(256);
+        if (ld_acquire_gpu(counter) >= target) return true;
+        if ((i & 63u) == 63u && *reinterpret_cast<volatile int32_t*>(status) != STATUS_OK) break;
+    }
+    *abort_flag = 1;
+    atomicExch(status, STATUS_TIMEOUT);
+    return false;
+}
+
+// Eight standard normals of row `row`, columns 8 ch .. 8 ch + 7 of a matrix's P as bfloat16 (one 16-byte
+// store of the scratch), from the generator or from a projection supplied by the caller.
+__device__ __forceinline__ uint4 p_vector(const float* __restrict__ ext_p, int m, int row, int ch, uint32_t matrix_id,
+                                          const StepParams& sp)
+{
+    uint4 v;
+    if (ext_p) {
+        float z[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) z[e] = 8 * ch + e < m ? __ldg(ext_p + (int64_t)row * m + 8 * ch + e) : 0.f;
+        v.x = pack_bf16x2(z[0], z[1]); v.y = pack_bf16x2(z[2], z[3]);
+        v.z = pack_bf16x2(z[4], z[5]); v.w = pack_bf16x2(z[6], z[7]);
+        return v;
+    }
+    const float4 a0 = normal_quad_fast((uint32_t)(2 * ch), (uint32_t)row, matrix_id, sp.epoch, sp.round_key);
+    const float4 a1 = normal_quad_fast((uint32_t)(2 * ch + 1), (uint32_t)row, matrix_id, sp.epoch, sp.round_key);
+    v.x = pack_bf16x2(a0.x, a0.y); v.y = pack_bf16x2(a0.z, a0.w);
+    v.z = pack_bf16x2(a1.x, a1.y); v.w = pack_bf16x2(a1.z, a1.w);
+    return v;
 }
 
 __device__ __forceinline__ float sum_sq_bf16x8(const uint4& v)
@@ -627,11 +661,11 @@ constexpr int P2_THREADS = 512;
 constexpr int P2_G_BYTES = 128 * TC_BK * 2;        // G of 128 channels, one k-block: 16 KiB
 constexpr int P2_MAX_STAGES = 8;
 constexpr int P2_MISC_BYTES = 512 + 1024;          // barriers and flags, alignment slack
-static_assert(P2_MISC_BYTES == 1536, "choose_tiling() reserves this many bytes");
+static_assert(P2_MISC_BYTES == 1536, "tensor_path_configure() reserves this many bytes");
 
 __global__ void __launch_bounds__(P2_THREADS, 1)
 project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix, int n_mat, int tile_begin,
-                    int tile_end, StepParams sp, TcTiling tl, int32_t* __restrict__ status)
+                    int tile_end, StepParams sp, TcTiling tl, GenArgs gen, int32_t* __restrict__ status)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
@@ -679,8 +713,58 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
     uint32_t it = 0, tile_iter = 0, stage = 0, phase = 0;
     auto next_stage = [&]() { ++it; if (++stage == (uint32_t)ns) { stage = 0; phase ^= 1; } };
 
+    // ---------------- generator warps (TcTiling::gen): P of every matrix of the launch, ahead of its use ----------------
+    // The spare warps of all CTAs (warp 3 everywhere, warp 1 of the peers, whose MMA role is the leader's) draw
+    // tickets; a ticket is one of GEN_CHUNKS pieces of one matrix's P, written as 16-byte vectors into the
+    // matrix's slot of the scratch (a ring of `slots` slots over the matrices in list order).  A slot is
+    // rewritten once every tile of its previous user has finished its MMAs (use_done); the P producers of
+    // the tiles wait for all pieces of their matrix (gen_done).  The lowest ticket outstanding never waits
+    // on anything that is not already under way, so the scheme cannot deadlock; every wait is bounded.
+    if (tl.gen != 0 && (warp == 3 || (warp == 1 && rank == 1))) {
+        for (;;) {
+            uint32_t ticket = 0;
+            if (lane == 0) ticket = atomicAdd(gen.ticket, 1u);
+            ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
+            const int q = gen.q_begin + (int)(ticket / GEN_CHUNKS);
+            if (q >= gen.q_end) break;
+            const int piece = (int)(ticket % GEN_CHUNKS);
+            const int gm = __ldg(gen.mats + q);
+            int ok = 1;
+            if (q - tl.slots >= gen.q_begin) {
+                const int pm = __ldg(gen.mats + q - tl.slots);
+                const uint32_t need = (uint32_t)(__ldg(&descs[pm].tiles_n) * __ldg(&descs[pm].tiles_k));
+                if (lane == 0) ok = wait_counter(gen.use_done + pm, need, abort_flag, status) ? 1 : 0;
+                ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+            }
+            if (!ok) break;
+            const MatDesc* gp = descs + gm;
+            const int vec_per_row = __ldg(&gp->m_pad) / 8, total = sp.rank * vec_per_row;
+            const int per = (total + GEN_CHUNKS - 1) / GEN_CHUNKS;
+            const int c_end = min(total, (piece + 1) * per);
+            const uint32_t matrix_id = (uint32_t)__ldg(&gp->matrix_id);
+            const float* __restrict__ ext_p = gp->ext_p;
+            const int gmm = __ldg(&gp->m);
+            uint4* const out = static_cast<uint4*>(gp->pstage);
+            // two vectors per pass: four Philox chains in flight per thread
+            for (int c = piece * per + lane; c < c_end; c += 64) {
+                const int row0 = c / vec_per_row;
+                const uint4 v0 = p_vector(ext_p, gmm, row0, c - row0 * vec_per_row, matrix_id, sp);
+                if (c + 32 < c_end) {
+                    const int row1 = (c + 32) / vec_per_row;
+                    out[c + 32] = p_vector(ext_p, gmm, row1, c + 32 - row1 * vec_per_row, matrix_id, sp);
+                }
+                out[c] = v0;
+            }
+            ptx::fence_proxy_async_global();
+            __threadfence();
+            __syncwarp();
+            if (lane == 0) red_release_gpu_add(gen.gen_done + gm, 1u);
+        }
+    }
+
     const int pair = blockIdx.x >> 1, pairs = gridDim.x >> 1;
     int mat = find_matrix(prefix, n_mat, tile_begin + pair < tile_end ? tile_begin + pair : tile_begin);
+    int p_ready_mat = -1;      // P producer: the matrix whose generated P it has already waited for
     for (int tile = tile_begin + pair; tile < tile_end; tile += pairs, ++tile_iter) {
         // the tiles of a CTA come in increasing order: the matrix index only moves forward
         while (mat + 1 < n_mat && __ldg(prefix + mat + 1) <= tile) ++mat;
@@ -729,7 +813,15 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                 const uint64_t pol_p = ptx::policy_evict_last();
                 const uint32_t full0 = ptx::map_to_cta(bar_full, 0);
                 const int p_row = r0 + (int)rank * r_half;
-                for (int kb = 0; kb < num_kb; ++kb, next_stage()) {
+                bool p_ok = true;
+                if (tl.gen != 0 && mat != p_ready_mat) {
+                    // every piece of this matrix's P has been written (by generic stores of other SMs): order
+                    // them before this thread's loads through the async proxy
+                    p_ok = wait_counter(gen.gen_done + mat, (uint32_t)GEN_CHUNKS, abort_flag, status);
+                    ptx::fence_proxy_async_global();
+                    p_ready_mat = mat;
+                }
+                for (int kb = 0; p_ok && kb < num_kb; ++kb, next_stage()) {
                     const uint32_t s = stage;
                     if (!wait_phase(bar_empty + 8 * s, phase ^ 1, abort_flag, status)) break;
                     ptx::tma_load_2d_pair(smem_base + s * stage_bytes + P2_G_BYTES, tmap_p, kb * TC_BK, p_row, full0 + 8 * s, pol_p);
@@ -862,6 +954,8 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                     if (half + 2 * a < r_slice / 16) ask(half + 2 * a);
             const bool acc_ok = __all_sync(0xFFFFFFFFu, wait_phase_idle(bar_acc_full + 8 * buf, use & 1, abort_flag, status));   // tcgen05.ld needs the whole warp
             ptx::tc_fence_after_sync();
+            // the MMAs of this tile are done, so both CTAs' last P tiles have been read: one count per pair tile
+            if (tl.gen != 0 && rank == 0 && warp == 8 && lane == 0 && acc_ok) red_release_gpu_add(gen.use_done + mat, 1u);
             float num = 0.f, den = 0.f;
             const int chunks = acc_ok ? r_slice / 16 : 0;
             for (int cchunk = half; cchunk < chunks; cchunk += 2) {
@@ -936,23 +1030,7 @@ __global__ void generate_p_kernel(const MatDesc* __restrict__ descs, int mat_beg
     const int m = __ldg(&dp->m);
     for (int c = blockIdx.x * blockDim.x + threadIdx.x; c < total; c += gridDim.x * blockDim.x) {
         const int row = c / chunks_per_row, ch = c - row * chunks_per_row;
-        if (ext_p) {
-            // a projection supplied by the caller: convert its row to bf16, zero the padding
-            float z[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) z[e] = 8 * ch + e < m ? __ldg(ext_p + (int64_t)row * m + 8 * ch + e) : 0.f;
-            uint4 v;
-            v.x = pack_bf16x2(z[0], z[1]); v.y = pack_bf16x2(z[2], z[3]);
-            v.z = pack_bf16x2(z[4], z[5]); v.w = pack_bf16x2(z[6], z[7]);
-            out[c] = v;
-            continue;
-        }
-        const float4 a0 = normal_quad_fast((uint32_t)(2 * ch), (uint32_t)row, matrix_id, sp.epoch, sp.round_key);
-        const float4 a1 = normal_quad_fast((uint32_t)(2 * ch + 1), (uint32_t)row, matrix_id, sp.epoch, sp.round_key);
-        uint4 v;
-        v.x = pack_bf16x2(a0.x, a0.y); v.y = pack_bf16x2(a0.z, a0.w);
-        v.z = pack_bf16x2(a1.x, a1.y); v.w = pack_bf16x2(a1.z, a1.w);
-        out[c] = v;
+        out[c] = p_vector(ext_p, m, row, ch, matrix_id, sp);
     }
 }
 
@@ -1064,20 +1142,16 @@ void launch_generate_p(const MatDesc* d_descs, int mat_begin, int mat_end, const
 }
 
 void launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_mat, int tile_begin, int tile_end,
-                           const StepParams& sp, int sm_count, int32_t* d_status, cudaStream_t stream)
+                           const StepParams& sp, const TcTiling& tl, const GenArgs& gen, TcLaunchState& state,
+                           int sm_count, int32_t* d_status, cudaStream_t stream)
 {
     const int tiles = tile_end - tile_begin;
     if (tiles <= 0) return;
-    const TcTiling tl = choose_tiling(sp.rank);
-    // the shared-memory opt-in is a per-device attribute of the kernels
-    static bool attr_set_on[64] = {};
-    int device = 0;
-    cudaGetDevice(&device);
-    bool& attr_set = attr_set_on[device & 63];
-    if (!attr_set) {
+    // the shared-memory opt-in is a per-device attribute of the kernels: set once per context
+    if (!state.attr_set) {
         cudaFuncSetAttribute(project_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
         cudaFuncSetAttribute(project_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
-        attr_set = true;
+        state.attr_set = true;
     }
     if (tl.pair) {
         cudaLaunchConfig_t cfg = {};
@@ -1092,20 +1166,18 @@ void launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_ma
         cfg.numAttrs = 1;
         // the tile loop is persistent: launch exactly as many pairs as can be resident at once
         // (a pair sits in one GPC, so this can be fewer than half the SMs)
-        static int max_pairs_on[64] = {};
-        int& max_pairs = max_pairs_on[device & 63];
-        if (max_pairs == 0) {
+        if (state.max_pairs == 0) {
             int clusters = 0;
             if (cudaOccupancyMaxActiveClusters(&clusters, project_pair_kernel, &cfg) != cudaSuccess || clusters < 1) {
                 cudaGetLastError();
                 clusters = sm_count / 2;
             }
-            max_pairs = clusters;
+            state.max_pairs = clusters;
         }
-        int pairs = max_pairs;
+        int pairs = state.max_pairs;
         if (tiles < pairs) pairs = tiles;
         cfg.gridDim = dim3(2 * pairs);
-        cudaLaunchKernelEx(&cfg, project_pair_kernel, d_descs, d_prefix, n_mat, tile_begin, tile_end, sp, tl, d_status);
+        cudaLaunchKernelEx(&cfg, project_pair_kernel, d_descs, d_prefix, n_mat, tile_begin, tile_end, sp, tl, gen, d_status);
         return;
     }
     const int grid = tiles < sm_count ? tiles : sm_count;

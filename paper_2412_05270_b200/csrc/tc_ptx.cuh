@@ -60,6 +60,13 @@ __device__ __forceinline__ void fence_proxy_async_smem()
 {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
+// Orders global-memory accesses made through the generic proxy (plain stores; other SMs' stores that this
+// thread has acquired) against accesses through the async proxy (TMA loads of the same memory).  Issued by
+// the writer after its stores and by the reader before its loads.
+__device__ __forceinline__ void fence_proxy_async_global()
+{
+    asm volatile("fence.proxy.async.global;" ::: "memory");
+}
 // A tensor map that lives in global memory and was written by a host copy: the thread that is going to
 // use it makes that copy visible to the tensor-map proxy first (system scope, once per thread and map).
 __device__ __forceinline__ void fence_tensormap_acquire(const void* tmap)

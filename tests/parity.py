@@ -3,6 +3,18 @@ seeded inputs and compares them under the stated bounds.
 
 Bounds: Philox draws bit-exact; per element |dW_gpu - dW_oracle| <= 2e-3 max|dW_oracle| + 1e-6;
 scales within 1e-3 relative; stored W equal to round(W_old + dW_gpu) exactly.
+
+The scale bound is stated against the projection in the precision of the GEMM operands: for
+bfloat16 gradients at rank > 1 the oracle rounds the standard normals behind P to bfloat16, as
+the tensor cores see them (against an unrounded P the scales move by up to 2.6e-3, which the
+1e-3 bound does not allow).
+
+Below rank 16 a channel's "norm" is the norm of very few numbers (one signed number at rank 1)
+and can come out far below its typical size; such a channel's scale is a ratio of two nearly
+cancelled sums and has no 1e-3 relative meaning in fp32.  Those channels are exempt from the
+scale bound (never from the dW bound); the exempt fraction is returned in `worst["exempt"]`
+and must stay below EXEMPT_MAX_LOW_RANK (or two channels, for matrices of fewer than 40).
+From rank 16 on no channel is exempt.
 """
 from __future__ import annotations
 
@@ -14,6 +26,9 @@ from paper_2412_05270_b200 import binding as B
 from paper_2412_05270_b200 import workloads as WL
 
 DW_REL, DW_ABS, SCALE_REL = 2e-3, 1e-6, 1e-3
+EXEMPT_BELOW = 0.02          # a channel is ill-conditioned when |R_j| or |R~_j| is under 2 % of the median
+EXEMPT_RANK = 16             # ranks from here on: no exemption
+EXEMPT_MAX_LOW_RANK = 0.05   # largest exempt fraction accepted below EXEMPT_RANK (rank 1: about 2 %)
 
 
 def config_of(wl: WL.Workload, flags=0, bias_correction=False) -> B.Config:
@@ -40,7 +55,7 @@ def oracle_of(wl: WL.Workload, mats=None, bias_correction=False, state_bf16=Fals
 
 
 def run_parity(wl: WL.Workload, steps=None, flags=0, bias_correction=False, check_mats=None, expect_path=None,
-               grad_fn=None, gen_device="cpu"):
+               grad_fn=None, gen_device="cpu", tuning=None):
     """Steps the whole list on the GPU and the matrices in `check_mats` on the oracle.
 
     With gen_device="cuda" the inputs are drawn on the GPU (large lists) and only the checked
@@ -49,7 +64,7 @@ def run_parity(wl: WL.Workload, steps=None, flags=0, bias_correction=False, chec
     n = len(wl.shapes)
     check_mats = list(range(n)) if check_mats is None else list(check_mats)
     dev = torch.device("cuda")
-    opt = B.Apollo(wl.shapes, config_of(wl, flags, bias_correction))
+    opt = B.Apollo(wl.shapes, config_of(wl, flags, bias_correction), tuning=tuning)
     if expect_path is not None:
         for i in check_mats:
             assert opt.path(i) == expect_path, (i, opt.path(i))
@@ -59,7 +74,7 @@ def run_parity(wl: WL.Workload, steps=None, flags=0, bias_correction=False, chec
     opt.set_delta_out(deltas)
     orc = oracle_of(wl, check_mats, bias_correction, state_bf16=bool(flags & B.FLAG_BF16_STATES))
     Wo = {i: Wg[i].float().cpu().numpy() for i in check_mats}
-    worst = {"dw": 0.0, "s": 0.0}
+    worst = {"dw": 0.0, "s": 0.0, "exempt": 0.0}
     for t in range(steps):
         Gg = [(grad_fn(wl, i, t) if grad_fn else WL.make_grad(wl, i, t, device=gen_device)).to(dev)
               for i in range(n)]
@@ -74,17 +89,16 @@ def run_parity(wl: WL.Workload, steps=None, flags=0, bias_correction=False, chec
             assert err <= bound, f"step {t} matrix {i}: |dW error| {err:.3e} > {bound:.3e}"
             worst["dw"] = max(worst["dw"], err / bound)
             s_gpu = opt.scales(i).cpu().numpy().astype(np.float64)
-            # A channel whose projected column (or its normalised moment) is far below the
-            # typical size is the difference of large terms: its scale has no 1e-3 relative
-            # meaning in fp32 (this happens at rank 1, where a "norm" is one signed number).
-            # Those channels are held to the dW bound above only.
             rn = np.linalg.norm(res.R, axis=0)
             tn = res.s * rn
-            good = (rn >= 0.02 * np.median(rn)) & (tn >= 0.02 * np.median(tn))
-            if wl.mode == "tensor":
-                good[:] = True
+            good = np.ones(rn.shape, dtype=bool)
+            if wl.mode != "tensor" and wl.rank < EXEMPT_RANK:
+                good = (rn >= EXEMPT_BELOW * np.median(rn)) & (tn >= EXEMPT_BELOW * np.median(tn))
+            exempt = 1.0 - float(good.mean())
+            assert (~good).sum() <= max(2, EXEMPT_MAX_LOW_RANK * good.size), \
+                f"step {t} matrix {i}: {exempt:.3f} of the channels exempt"
+            worst["exempt"] = max(worst["exempt"], exempt)
             rel = np.abs(s_gpu - res.s) / (np.abs(res.s) + 1e-30)
-            assert good.mean() > 0.7
             assert np.all(rel[good] <= SCALE_REL), f"step {t} matrix {i}: scale rel error {rel[good].max():.3e}"
             worst["s"] = max(worst["s"], float(rel[good].max()))
             lim = opt.limiter(i).cpu().numpy()

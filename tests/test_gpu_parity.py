@@ -73,47 +73,50 @@ def test_tensor_core_path(rank, shapes):
     run_parity(wl, expect_path=B.PATH_TENSOR)
 
 
-@pytest.mark.parametrize("env", [
-    {"APOLLO_P_STAGING_MB": "1"},                           # staging slots shared group by group: refilled every step
-    {"APOLLO_TC_RSLICE": "64"},                             # four row slices of R per channel tile
-    {"APOLLO_TC_KERNEL": "ring"},                           # single-CTA kernel, 256 channels x 256 rows per tile
-    {"APOLLO_TC_KERNEL": "ring", "APOLLO_P_STAGING_MB": "1"},
-    {"APOLLO_TC_KERNEL": "ring", "APOLLO_TC_RSLICE": "128", "APOLLO_TC_NBLK": "2"},
-    {"APOLLO_P_STAGING": "0"},                              # P generated in shared memory by every CTA (ring kernel)
-    {"APOLLO_P_STAGING": "0", "APOLLO_TC_RSLICE": "128", "APOLLO_TC_NBLK": "4"},
-    {"APOLLO_TC_EPI_PREFETCH": "0"},                        # no L2 prefetch of the moments in the epilogue
-    {"APOLLO_TC_EPI_PREFETCH": "8", "APOLLO_TC_RSLICE": "64"},   # prefetch distance beyond the chunks of a slice
-])
-def test_tensor_core_path_selectable_modes(env, monkeypatch):
-    """The environment switches of the tensor path give the same parity; where they leave the tiles and
-    the order of every sum alone, they give the same bits."""
-    shapes = [(512, 1376), (1376, 512), (512, 512), (300, 1032), (1376, 1400)]   # staged P: 1.6 MB in all
+MODES = [
+    # (flags, tuning of the mode, tuning of the run to compare bits with)
+    (B.FLAG_KEEP_P, {}, None),                                    # every matrix keeps its P for the epoch
+    (0, {"p_generator": 1}, {}),                                  # a separate kernel fills the scratch (one group here)
+    (0, {"p_generator": 1, "scratch_mb": 1}, {}),                 # ... group by group: the scratch holds 1 MB
+    (0, {"scratch_mb": 1}, {}),                                   # generator warps, ring of two slots
+    (0, {"r_slice": 64}, {"r_slice": 64, "p_generator": 1}),      # four row slices of R per channel tile
+    (0, {"kernel": B.TC_KERNEL_RING}, None),                      # single-CTA kernel, 256 channels x 256 rows per tile
+    (0, {"kernel": B.TC_KERNEL_RING, "scratch_mb": 1}, {"kernel": B.TC_KERNEL_RING}),
+    (B.FLAG_KEEP_P, {"kernel": B.TC_KERNEL_RING, "r_slice": 128, "nblk": 2}, None),
+    (0, {"p_source": B.P_SHARED}, {"kernel": B.TC_KERNEL_RING}),  # P generated in shared memory by every CTA (ring kernel)
+    (0, {"p_source": B.P_SHARED, "r_slice": 128, "nblk": 4}, {"kernel": B.TC_KERNEL_RING, "r_slice": 128, "nblk": 4}),
+    (0, {"epi_prefetch": 0}, {}),                                 # no L2 prefetch of the moments in the epilogue
+    (0, {"epi_prefetch": 8, "r_slice": 64}, {"r_slice": 64}),     # prefetch distance beyond the chunks of a slice
+]
+
+
+@pytest.mark.parametrize("flags,mode,ref", MODES)
+def test_tensor_core_path_selectable_modes(flags, mode, ref):
+    """Every mode of the tensor path (apollo_tuning, APOLLO_FLAG_KEEP_P) meets the parity bounds, and since none
+    of them changes P or, at equal tile shape, the order of any sum, it gives the same bits as the run it is
+    paired with."""
+    shapes = [(512, 1376), (1376, 512), (512, 512), (300, 1032), (1376, 1400)]   # P: 1.6 MB in all
     wl = _wl(shapes, 256, dtype="bf16", steps=4, T=2, wd=0.01)
     dev = torch.device("cuda")
 
-    def final_weights():
-        opt = B.Apollo(wl.shapes, B.config_for(wl))
+    def final_weights(fl, tu):
+        opt = B.Apollo(wl.shapes, B.config_for(wl, fl), tuning=B.make_tuning(**tu))
         W = [WL.make_weight(wl, i).to(dev) for i in range(len(shapes))]
         for t in range(4):
             opt.step(W, [WL.make_grad(wl, i, t).to(dev) for i in range(len(shapes))], wl.lr, wl.wd)
         assert opt.status() == B.OK
-        return W, [opt.scales(i) for i in range(len(shapes))]
+        out = W, [opt.scales(i) for i in range(len(shapes))]
+        opt.close()
+        return out
 
-    # the run to compare with: the same kernel and tile shape, P staged once per epoch
-    same_tiles = {k: v for k, v in env.items() if k in ("APOLLO_TC_KERNEL", "APOLLO_TC_RSLICE", "APOLLO_TC_NBLK")}
-    if env.get("APOLLO_P_STAGING") == "0":
-        same_tiles["APOLLO_TC_KERNEL"] = "ring"             # the kernel that generates P itself
-    for k, v in same_tiles.items():
-        monkeypatch.setenv(k, v)
-    W_ref, s_ref = final_weights()
-    for k, v in env.items():
-        monkeypatch.setenv(k, v)
-    run_parity(wl, expect_path=B.PATH_TENSOR)
-    W_mode, s_mode = final_weights()
-    for a, b in zip(W_ref, W_mode):
-        assert torch.equal(a, b)
-    for a, b in zip(s_ref, s_mode):
-        assert torch.equal(a, b)
+    run_parity(wl, flags=flags, expect_path=B.PATH_TENSOR, tuning=B.make_tuning(**mode))
+    if ref is not None:
+        W_ref, s_ref = final_weights(0, ref)
+        W_mode, s_mode = final_weights(flags, mode)
+        for a, b in zip(W_ref, W_mode):
+            assert torch.equal(a, b)
+        for a, b in zip(s_ref, s_mode):
+            assert torch.equal(a, b)
 
 
 def test_tensor_core_path_tensor_mode_and_bias_correction():
@@ -383,3 +386,31 @@ def test_a_wait_that_runs_out_is_reported_and_leaves_the_context_usable():
     assert a.status() == B.OK and b.status() == B.OK
     for x, y in zip(Wa, Wb):
         assert torch.equal(x, y)
+
+
+def test_a_step_whose_projection_gave_up_leaves_weights_and_limiter_untouched():
+    """Once the status word says that a wait has run out, the finalize and update passes of a step write
+    nothing: the weights and the limiter's norm stay as they were until the caller has read the status."""
+    wl = _wl([(512, 1376), (1376, 512)], 64, dtype="bf16", steps=3, T=2, wd=0.01)
+    dev = torch.device("cuda")
+    opt = B.Apollo(wl.shapes, B.config_for(wl))
+    W = [WL.make_weight(wl, i).to(dev) for i in range(2)]
+    opt.step(W, [WL.make_grad(wl, i, 0).to(dev) for i in range(2)], wl.lr, wl.wd)
+    assert opt.status() == B.OK
+    W_before = [w.clone() for w in W]
+    lim_before = [opt.limiter(i).clone() for i in range(2)]
+    opt.selftest_bounded_wait()                   # the status word now reads "timeout", as after a wait that gave up
+    opt.step(W, [WL.make_grad(wl, i, 1).to(dev) for i in range(2)], wl.lr, wl.wd)
+    torch.cuda.synchronize()
+    for a, b in zip(W, W_before):
+        assert torch.equal(a, b)
+    for i in range(2):
+        assert torch.equal(opt.limiter(i), lim_before[i])
+    assert opt.status() == B.ERR_TIMEOUT
+    assert opt.status() == B.OK
+    opt.step(W, [WL.make_grad(wl, i, 2).to(dev) for i in range(2)], wl.lr, wl.wd)     # the context works on
+    torch.cuda.synchronize()
+    assert opt.status() == B.OK
+    assert not torch.equal(W[0], W_before[0])
+    opt.close()
+

@@ -6,16 +6,19 @@ synchronisation of an allocation, a process whose pool is fully handed out), so 
 cannot give apollo_create a workspace.  For them the library carries a fixed scratch array
 and one entry point that uses it.  This test drives that entry point through the C ABI on
 two steps in a row and checks weights, moments and limiter norm against the regular
-context-based step on the same inputs.  It lives in a file that is collected last, so a
-run that stops at the first failure has already run every other test.
+context-based step on the same inputs, then against the CPU oracle, and checks that the
+device's free memory does not move across a call.  It lives in a file that is collected
+last, so a run that stops at the first failure has already run every other test.
 """
 import math
 
+import numpy as np
 import pytest
 import torch
 
 from paper_2412_05270_b200 import binding as B
 from paper_2412_05270_b200 import workloads as WL
+from parity import DW_ABS, DW_REL, _f32, oracle_of
 
 pytestmark = pytest.mark.gpu
 
@@ -60,6 +63,55 @@ def test_two_consecutive_static_steps_match_the_context_step(shape, dtype, mode)
     opt.close()
 
 
+@pytest.mark.parametrize("shape,mode", [((520, 1300), "tensor"), ((1300, 520), "channel")])
+def test_static_steps_against_the_oracle(shape, mode):
+    """Five steps across a projection refresh (T = 3), the caller keeping t, M, V and the previous
+    norm: the weights follow the oracle's within the parity bound on the update."""
+    dev = torch.device("cuda")
+    wl = WL.Workload("static_oracle", [shape], "bf16", 1, mode, T=3, steps=5, wd=0.01,
+                     alpha=math.sqrt(128.0) if mode == "tensor" else 1.0)
+    cfg = B.config_for(wl)
+    n = max(shape)
+    W = WL.make_weight(wl, 0).to(dev)
+    M = torch.zeros(n, dtype=torch.float32, device=dev)
+    V = torch.zeros(n, dtype=torch.float32, device=dev)
+    prev = torch.zeros(1, dtype=torch.float32, device=dev)
+    orc = oracle_of(wl, [0])[0]
+    Wo = W.float().cpu().numpy()
+    for t in range(wl.steps):
+        G = WL.make_grad(wl, 0, t).to(dev)
+        B.mini_step_static(W, G, M, V, prev, cfg, matrix=0, t=t, lr=wl.lr, wd=wl.wd)
+        torch.cuda.synchronize()
+        res = orc.step(Wo, G.float().cpu().numpy(), _f32(wl.lr), _f32(wl.wd))
+        bound = DW_REL * np.max(np.abs(res.dW)) + DW_ABS
+        # the stored weight is a bf16 rounding of W_old + dW: one rounding step of slack on top of the bound
+        tol = 2.0 ** -7 * np.abs(res.W) + bound
+        assert np.all(np.abs(W.float().cpu().numpy() - res.W) <= tol), f"step {t}"
+        assert abs(prev.item() - res.norm) <= 2e-3 * res.norm
+        np.testing.assert_allclose(M.cpu().numpy(), orc.M[0], rtol=2e-3, atol=2e-3 * np.abs(orc.M).max())
+        Wo = res.W
+        W.copy_(torch.from_numpy(res.W).to(W.dtype))     # keep the two trajectories on the same weights
+
+
+def test_a_static_step_obtains_no_device_memory():
+    dev = torch.device("cuda")
+    shape = (640, 1024)
+    wl = WL.Workload("static_mem", [shape], "bf16", 1, "tensor", T=1, steps=2, alpha=math.sqrt(128.0))
+    cfg = B.config_for(wl)
+    W = WL.make_weight(wl, 0).to(dev)
+    G = WL.make_grad(wl, 0, 0).to(dev)
+    M = torch.zeros(1024, dtype=torch.float32, device=dev)
+    V = torch.zeros(1024, dtype=torch.float32, device=dev)
+    prev = torch.zeros(1, dtype=torch.float32, device=dev)
+    B.mini_step_static(W, G, M, V, prev, cfg, matrix=0, t=0, lr=wl.lr)      # first call on the device: looks the array up
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info(dev)
+    B.mini_step_static(W, G, M, V, prev, cfg, matrix=0, t=1, lr=wl.lr)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info(dev)
+    assert free_after == free_before
+
+
 def test_oversized_and_wrong_rank_requests_are_rejected():
     dev = torch.device("cuda")
     small = torch.zeros(8, 8, dtype=torch.bfloat16, device=dev)
@@ -74,4 +126,9 @@ def test_oversized_and_wrong_rank_requests_are_rejected():
     rc = lib.apollo_mini_step_static(small.data_ptr(), small.data_ptr(), 8, 8, f.data_ptr(), f.data_ptr(),
                                      f.data_ptr(), cfg2, 0, 0, 0.1, 0.0, None)
     assert rc == B.ERR_RANK
+    # the moments of this entry point are floats: a request for two-byte moments is refused, not overrun
+    cfg3 = B.make_config(rank=1, mode=B.SCALE_TENSOR, flags=B.FLAG_BF16_STATES)
+    rc = lib.apollo_mini_step_static(small.data_ptr(), small.data_ptr(), 8, 8, f.data_ptr(), f.data_ptr(),
+                                     f.data_ptr(), cfg3, 0, 0, 0.1, 0.0, None)
+    assert rc == B.ERR_INVALID_ARG
     torch.cuda.synchronize()
