@@ -53,6 +53,8 @@ extern "C" {
 #define APOLLO_ERR_TIMEOUT (-7)     /* a bounded device-side wait expired (reported by apollo_status) */
 #define APOLLO_ERR_UNSUPPORTED (-8) /* the device is not an sm_100 part */
 #define APOLLO_ERR_TOO_LARGE (-9)   /* the matrix does not fit the built-in scratch of apollo_mini_step_static */
+#define APOLLO_ERR_INTERNAL (-10)   /* debug build of the library (-DAPOLLO_DEBUG) only: an index check inside a kernel
+                                       failed; the access was skipped (reported by apollo_status) */
 
 #define APOLLO_MAX_RANK 512
 
@@ -193,8 +195,13 @@ APOLLO_API int apollo_get_state(apollo_ctx* ctx, int32_t matrix, float* d_M, flo
 APOLLO_API int apollo_set_delta_out(apollo_ctx* ctx, float* const* d_dW);
 
 /*
- * Synchronises `cuda_stream` and returns the device status word: APOLLO_OK, or
- * APOLLO_ERR_TIMEOUT if a bounded wait inside a kernel expired since the last call.
+ * Synchronises `cuda_stream` and returns the device status word, clearing it: APOLLO_OK, or
+ * APOLLO_ERR_TIMEOUT if a bounded wait inside a projection kernel expired since the last call
+ * (APOLLO_ERR_INTERNAL: see above).  While the word is set, the finalize and update passes of
+ * every step write nothing: the step whose projection gave up, and the steps issued after it
+ * until this call, leave the weights, the scales and the limiter's norm as they were.  The
+ * moments of that step are partly updated; resume from a checkpoint (apollo_state_import) to
+ * continue exactly.
  */
 APOLLO_API int apollo_status(apollo_ctx* ctx, void* cuda_stream);
 

@@ -13,11 +13,13 @@ import torch
 
 _PKG = Path(__file__).resolve().parent
 LIB_PATH = _PKG / "libapollo.so"
+DEBUG_LIB_PATH = _PKG / "libapollo_debug.so"     # built with -DAPOLLO_DEBUG: index checks inside every kernel
 
 OK = 0
 ERR_INVALID_ARG, ERR_SHAPE, ERR_RANK, ERR_ALIGN, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED = (
     -1, -2, -3, -4, -5, -6, -7, -8)
 ERR_TOO_LARGE = -9
+ERR_INTERNAL = -10
 STATIC_SCRATCH_BYTES = 8 << 20
 SCALE_CHANNEL, SCALE_TENSOR = 0, 1
 DT_F32, DT_BF16 = 0, 1
@@ -76,14 +78,31 @@ def make_tuning(kernel=TC_KERNEL_PAIR, p_source=P_SCRATCH, p_generator=0, scratc
 _lib = None
 
 
+_libs = {}
+
+
+def use_library(path=None):
+    """Route all later calls of this module through the library at `path` (None: libapollo.so); the test of
+    the bounds-checking build switches to libapollo_debug.so and back.  Contexts keep the library they were
+    created with."""
+    global _lib
+    _lib = None if path is None else _load_from(Path(path))
+
+
 def load():
     """Load libapollo.so; raises if it has not been built (there is no fallback)."""
     global _lib
-    if _lib is not None:
-        return _lib
-    if not LIB_PATH.exists():
-        raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2412_05270_b200.build` (nvcc, sm_100a)")
-    lib = ctypes.CDLL(str(LIB_PATH))
+    if _lib is None:
+        _lib = _load_from(LIB_PATH)
+    return _lib
+
+
+def _load_from(path: Path):
+    if path in _libs:
+        return _libs[path]
+    if not path.exists():
+        raise ImportError(f"{path} is missing: run `python -m paper_2412_05270_b200.build` (nvcc, sm_100a)")
+    lib = ctypes.CDLL(str(path))
     vp, i32, u32, u64, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint32, ctypes.c_uint64, ctypes.c_float
     lib.apollo_workspace_bytes.argtypes = [ctypes.POINTER(Shape), i32, ctypes.POINTER(Config),
                                            ctypes.POINTER(ctypes.c_size_t)]
@@ -125,7 +144,7 @@ def load():
     for name in EXPORTS:
         if name not in ("apollo_strerror", "apollo_cuda_error_string"):
             getattr(lib, name).restype = ctypes.c_int
-    _lib = lib
+    _libs[path] = lib
     return lib
 
 

@@ -8,6 +8,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libapollo.so"
+LIB_DEBUG = PKG / "libapollo_debug.so"      # the same sources with -DAPOLLO_DEBUG: index checks inside the kernels
 SOURCES = ["apollo_api.cu", "kernels_basic.cu", "kernels_tensor.cu", "apollo_static.cu", "kernels_adamw.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -15,25 +16,30 @@ NVCC_FLAGS = [
 ]
 
 
-def _stale() -> bool:
-    if not LIB.exists():
+def _stale(lib: Path = LIB) -> bool:
+    if not lib.exists():
         return True
-    built = LIB.stat().st_mtime
+    built = lib.stat().st_mtime
     deps = list(CSRC.glob("*")) + [PKG.parent / "include" / "apollo.h", Path(__file__)]
     return any(p.stat().st_mtime > built for p in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> Path:
-    if not force and not _stale():
-        return LIB
+def build_library(force: bool = False, verbose: bool = False, debug: bool = False) -> Path:
+    """Compiles the library in-tree.  debug=True builds libapollo_debug.so: every kernel checks the index
+    range of its global loads and stores and reports a violation through the context's status word
+    (apollo_status returns APOLLO_ERR_INTERNAL) instead of making the access."""
+    lib = LIB_DEBUG if debug else LIB
+    if not force and not _stale(lib):
+        return lib
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     objs = []
-    obj_dir = PKG / "_build"
-    obj_dir.mkdir(exist_ok=True)
+    obj_dir = PKG / ("_build/debug" if debug else "_build")
+    obj_dir.mkdir(parents=True, exist_ok=True)
+    flags = NVCC_FLAGS + (["-DAPOLLO_DEBUG"] if debug else [])
     procs = []
     for src in SOURCES:
         obj = obj_dir / (src + ".o")
-        cmd = [nvcc, *NVCC_FLAGS, "-c", str(CSRC / src), "-o", str(obj)]
+        cmd = [nvcc, *flags, "-c", str(CSRC / src), "-o", str(obj)]
         if verbose:
             cmd.insert(1, "-Xptxas=-v")
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
@@ -44,12 +50,12 @@ def build_library(force: bool = False, verbose: bool = False) -> Path:
             print(out)
         if p.returncode != 0:
             raise RuntimeError(f"nvcc failed on {src}")
-    tmp = LIB.with_suffix(f".{os.getpid()}.tmp")
+    tmp = lib.with_suffix(f".{os.getpid()}.tmp")
     subprocess.run([nvcc, "-shared", "-o", str(tmp), *objs, "-Xcompiler", "-fvisibility=hidden"], check=True)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
     import sys
-    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

@@ -2,6 +2,8 @@
 // launch sequence of one step (Algorithm 1): projection pass -> finalize -> update pass.
 #include "../../include/apollo.h"
 
+#include <nvtx3/nvToolsExt.h>
+
 #include <cmath>
 #include <cstring>
 #include <new>
@@ -16,6 +18,14 @@ namespace {
 
 constexpr size_t ALIGN = 256;
 inline size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
+
+// An NVTX range on the calling thread, closed at the latest when the object goes out of scope.
+struct NvtxRange {
+    bool open;
+    explicit NvtxRange(const char* name) : open(true) { nvtxRangePushA(name); }
+    void close() { if (open) { nvtxRangePop(); open = false; } }
+    ~NvtxRange() { close(); }
+};
 
 struct MatPlan {
     int32_t rows, cols, m, n, tall, path, slices, g2_slices, tiles_n, tiles_k;
@@ -263,6 +273,7 @@ const char* apollo_strerror(int code)
         case APOLLO_ERR_TIMEOUT: return "bounded device-side wait expired";
         case APOLLO_ERR_UNSUPPORTED: return "device is not an sm_100 GPU";
         case APOLLO_ERR_TOO_LARGE: return "matrix exceeds the built-in scratch of apollo_mini_step_static";
+        case APOLLO_ERR_INTERNAL: return "an index check inside a kernel failed (debug build)";
         default: return "unknown error";
     }
 }
@@ -514,9 +525,12 @@ static int step_range(apollo_ctx* ctx, int first, int count, void* const* d_W, c
         sp.inv_bc2 = (float)(1.0 / (1.0 - std::pow((double)cfg.beta2, (double)(ctx->t + 1))));
     }
 
+    // NVTX ranges around the three phases (host side of the launches): a timeline tool shows them, and
+    // without one attached each call is a pointer test
     int launches = 0;
     cudaEvent_t* ev = (ctx->timing_on && whole) ? ctx->ev[ctx->t % APOLLO_TIMING_SLOTS] : nullptr;
     if (ev) cudaEventRecord(ev[0], stream);
+    NvtxRange range_projection("apollo.projection");
     auto tiles_of = [&](int path, int a, int b, int& tb, int& te) {
         tb = ctx->h_prefix[path][a]; te = ctx->h_prefix[path][b];
         return te > tb;
@@ -524,12 +538,12 @@ static int step_range(apollo_ctx* ctx, int first, int count, void* const* d_W, c
     int tb = 0, te = 0;
     if (tiles_of(PATH_STREAM, first, last, tb, te)) {
         launch_project_stream(cfg.dtype, ctx->d_descs, ctx->d_prefix[PATH_STREAM], ctx->n_mat, tb, te, sp,
-                              ctx->sm_count, stream);
+                              ctx->sm_count, ctx->d_status, stream);
         ++launches;
     }
     if (tiles_of(PATH_SIMT, first, last, tb, te)) {
         launch_project_simt(cfg.dtype, ctx->d_descs, ctx->d_prefix[PATH_SIMT], ctx->n_mat, tb, te, sp, ctx->sm_count,
-                            stream);
+                            ctx->d_status, stream);
         ++launches;
     }
     if (tiles_of(PATH_TENSOR, first, last, tb, te)) {
@@ -581,13 +595,18 @@ static int step_range(apollo_ctx* ctx, int first, int count, void* const* d_W, c
             }
         }
     }
+    range_projection.close();
     if (ev) cudaEventRecord(ev[1], stream);
+    NvtxRange range_finalize("apollo.finalize");
     launch_finalize(ctx->d_descs, first, count, sp, ctx->d_status, stream);
     ++launches;
+    range_finalize.close();
     if (ev) cudaEventRecord(ev[2], stream);
+    NvtxRange range_update("apollo.update");
     tiles_of(3, first, last, tb, te);
     launch_update(cfg.dtype, ctx->d_descs, ctx->d_prefix[3], ctx->n_mat, tb, te, sp, ctx->sm_count, ctx->d_status, stream);
     ++launches;
+    range_update.close();
     if (ev) cudaEventRecord(ev[3], stream);
     if (!cuda_ok(cudaGetLastError())) return APOLLO_ERR_CUDA;
     ctx->first = false;
@@ -661,7 +680,7 @@ int apollo_status(apollo_ctx* ctx, void* cuda_stream)
     if (cudaMemcpy(&word, ctx->d_status, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return APOLLO_ERR_CUDA;
     if (word != STATUS_OK) {
         cudaMemset(ctx->d_status, 0, sizeof(word));
-        return APOLLO_ERR_TIMEOUT;
+        return word == STATUS_BOUNDS ? APOLLO_ERR_INTERNAL : APOLLO_ERR_TIMEOUT;
     }
     return APOLLO_OK;
 }

@@ -65,8 +65,8 @@ inline long long update_tile_count(long long rows, long long cols, bool tall)
 // that every row starts a 256-byte line.  Tensor path: channel blocks of 128, each block r x 128
 // row-major (block b holds channels 128 b ..): the 128 channels x r_slice rows that one CTA reads and
 // writes per tile are one contiguous piece of memory instead of r_slice pieces of 512 bytes n apart.
-inline int state_pitch(int n, int rank) { return rank > 1 ? (n + 63) / 64 * 64 : n; }
-inline long long state_elements(int n, int rank, bool tiled)
+__host__ __device__ inline int state_pitch(int n, int rank) { return rank > 1 ? (n + 63) / 64 * 64 : n; }
+__host__ __device__ inline long long state_elements(int n, int rank, bool tiled)
 {
     return (long long)rank * (tiled ? (n + 127) / 128 * 128 : state_pitch(n, rank));
 }
@@ -166,5 +166,6 @@ struct TcLaunchState {
 // Device status word values.
 constexpr int32_t STATUS_OK = 0;
 constexpr int32_t STATUS_TIMEOUT = 1;
+constexpr int32_t STATUS_BOUNDS = 2;    // debug build only: an index check inside a kernel failed (the access was skipped)
 
 }  // namespace apollo

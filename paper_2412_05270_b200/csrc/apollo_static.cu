@@ -162,7 +162,7 @@ extern "C" int apollo_mini_step_static(void* d_W, const void* d_G, int64_t rows,
     const MatDesc* d_desc = reinterpret_cast<const MatDesc*>(base + OFF_DESC);
     static_setup_kernel<<<1, 1, 0, stream>>>(d, (int)proj_tiles, (int)update_tiles);
     launch_project_stream(cfg->dtype, d_desc, reinterpret_cast<const int*>(base + OFF_PREFIX_P), 1,
-                          0, (int)proj_tiles, sp, sm_count, stream);
+                          0, (int)proj_tiles, sp, sm_count, nullptr, stream);
     launch_finalize(d_desc, 0, 1, sp, nullptr, stream);
     launch_update(cfg->dtype, d_desc, reinterpret_cast<const int*>(base + OFF_PREFIX_U), 1, 0, (int)update_tiles,
                   sp, sm_count, nullptr, stream);

@@ -9,6 +9,22 @@
 
 namespace apollo {
 
+// Debug build (-DAPOLLO_DEBUG): every kernel checks the index range of its global loads and stores against
+// the extent of the array before the access; a range that is not inside sets the status word to STATUS_BOUNDS
+// and the access is skipped (the kernel goes on and ends normally).  In the release build the macro is `true`.
+#ifdef APOLLO_DEBUG
+__device__ __forceinline__ bool dbg_in_range(int64_t first, int64_t last, int64_t extent, int32_t* status)
+{
+    if (first >= 0 && last >= first && last < extent) return true;
+    if (status) atomicExch(status, STATUS_BOUNDS);
+    return false;
+}
+#define APOLLO_DBG_RANGE(first, last, extent, status) \
+    apollo::dbg_in_range((int64_t)(first), (int64_t)(last), (int64_t)(extent), (status))
+#else
+#define APOLLO_DBG_RANGE(first, last, extent, status) true
+#endif
+
 // prefix[i] = first tile of matrix i, prefix[n_mat] = total.  Returns the matrix that owns
 // `tile` (the last i with prefix[i] <= tile; matrices without tiles are skipped).
 __device__ __forceinline__ int find_matrix(const int* __restrict__ prefix, int n_mat, int tile)

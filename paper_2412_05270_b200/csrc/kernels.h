@@ -10,16 +10,17 @@ void launch_philox_draws(uint32_t key0, uint32_t key1, uint32_t matrix, uint32_t
 void launch_projection(uint32_t key0, uint32_t key1, uint32_t matrix, uint32_t epoch, int r, int m,
                        float* d_out, cudaStream_t stream);
 void launch_project_stream(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int tile_begin, int tile_end,
-                           const StepParams& sp, int sm_count, cudaStream_t stream);
+                           const StepParams& sp, int sm_count, int32_t* d_status, cudaStream_t stream);
 void launch_project_simt(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int tile_begin, int tile_end,
-                         const StepParams& sp, int sm_count, cudaStream_t stream);
+                         const StepParams& sp, int sm_count, int32_t* d_status, cudaStream_t stream);
 // d_status (may be null): the context's status word.  When it is not STATUS_OK -- a bounded wait of the
 // projection gave up -- finalize and update return without writing, so that a step whose projection is
-// incomplete leaves the weights, the scales and the limiter's norm as they were.
-void launch_finalize(const MatDesc* d_descs, int first, int count, const StepParams& sp, const int32_t* d_status,
+// incomplete leaves the weights, the scales and the limiter's norm as they were.  Kernels built with
+// -DAPOLLO_DEBUG also report a failed index check there (STATUS_BOUNDS).
+void launch_finalize(const MatDesc* d_descs, int first, int count, const StepParams& sp, int32_t* d_status,
                      cudaStream_t stream);
 void launch_update(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int tile_begin, int tile_end,
-                   const StepParams& sp, int sm_count, const int32_t* d_status, cudaStream_t stream);
+                   const StepParams& sp, int sm_count, int32_t* d_status, cudaStream_t stream);
 
 
 // bfloat16 -> float copy (observability of bfloat16 states).

@@ -77,7 +77,7 @@ constexpr int STREAM_TALL_CHUNK = 2048;   // entries of P staged per pass over a
 template <typename T>
 __global__ void __launch_bounds__(STREAM_THREADS, 3)     // three blocks per SM: at most 85 registers
 project_stream_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix, int n_mat,
-                      int tile_begin, int tile_end, StepParams sp)
+                      int tile_begin, int tile_end, StepParams sp, int32_t* __restrict__ status)
 {
     __shared__ float Ps[STREAM_TALL_CHUNK];
     __shared__ float red[2][8][STREAM_COLS];
@@ -90,6 +90,8 @@ project_stream_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
         const T* __restrict__ G = static_cast<const T*>(d.G);
         const int cols = d.cols;
         const bool vec_ok = (cols % 8) == 0;
+        const int64_t g_extent = (int64_t)d.rows * cols;      // (index checks of the debug build)
+        (void)g_extent; (void)status;
 
         if (!d.tall) {
             const int tn = local % d.tiles_n, tk = local / d.tiles_n;
@@ -120,6 +122,7 @@ project_stream_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                 if (vec_ok) {
                     // eight rows per pass: all eight 16-byte loads are issued before the first use
                     for (; ii + 56 < rows_here; ii += 64) {
+                        if (!APOLLO_DBG_RANGE((int64_t)(i0 + ii) * cols + j0, (int64_t)(i0 + ii + 56) * cols + j0 + 7, g_extent, status)) continue;
                         Raw8<T> raw[8];
 #pragma unroll
                         for (int u = 0; u < 8; ++u) raw[u] = load_raw8_stream(G + (int64_t)(i0 + ii + 8 * u) * cols + j0);
@@ -136,6 +139,7 @@ project_stream_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                 for (; ii < rows_here; ii += 8) {
                     float g[8];
                     const T* src = G + (int64_t)(i0 + ii) * cols + j0;
+                    if (!APOLLO_DBG_RANGE(src - G, src - G + count - 1, g_extent, status)) continue;
                     if (vec_ok) load8_aligned(src, g); else load8_guarded(src, count, g);
                     const float p = Ps[ii];
 #pragma unroll
@@ -151,7 +155,8 @@ project_stream_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
 #pragma unroll
                 for (int w = 0; w < 8; ++w) { r += red[0][w][tid]; g2 += red[1][w][tid]; }
                 float2* out = reinterpret_cast<float2*>(d.part) + ((int64_t)tk * d.n + j);
-                *out = make_float2(r * d.r_scale, g2);
+                if (APOLLO_DBG_RANGE((int64_t)tk * d.n + j, (int64_t)tk * d.n + j, (int64_t)d.slices * d.n, status))
+                    *out = make_float2(r * d.r_scale, g2);
             }
         } else {
             // channels are the stored rows; the contraction runs along the contiguous side
@@ -183,6 +188,7 @@ project_stream_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
 #pragma unroll
                     for (int e = 0; e < 8; ++e) p[e] = Ps[x + e];   // entries past `chunk` meet zero-filled g
                     if (vec_ok && rows_left >= 8) {
+                        if (!APOLLO_DBG_RANGE((int64_t)j_base * cols + c0 + x, (int64_t)(j_base + 7) * cols + c0 + x + 7, g_extent, status)) continue;
                         // all eight 16-byte loads of the warp's rows are issued before the first use
                         Raw8<T> raw[8];
 #pragma unroll
@@ -201,6 +207,7 @@ project_stream_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                         if (rr < rows_left) {
                             float g[8];
                             const T* src = G + (int64_t)(j_base + rr) * cols + c0 + x;
+                            if (!APOLLO_DBG_RANGE(src - G, src - G + count - 1, g_extent, status)) continue;
                             if (vec_ok) load8_aligned(src, g); else load8_guarded(src, count, g);
 #pragma unroll
                             for (int e = 0; e < 8; ++e) { accR[rr] = fmaf(p[e], g[e], accR[rr]); accG[rr] = fmaf(g[e], g[e], accG[rr]); }
@@ -217,7 +224,7 @@ project_stream_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                     g2 += __shfl_xor_sync(0xFFFFFFFFu, g2, off);
                 }
                 const int j = j_base + rr;
-                if (lane == 0 && j < d.rows)
+                if (lane == 0 && j < d.rows && APOLLO_DBG_RANGE(j, j, (int64_t)d.slices * d.n, status))
                     reinterpret_cast<float2*>(d.part)[j] = make_float2(r * d.r_scale, g2);
             }
         }
@@ -236,7 +243,7 @@ constexpr int SIMT_THREADS = 256;
 template <typename T>
 __global__ void __launch_bounds__(SIMT_THREADS)
 project_simt_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix, int n_mat,
-                    int tile_begin, int tile_end, StepParams sp)
+                    int tile_begin, int tile_end, StepParams sp, int32_t* __restrict__ status)
 {
     __shared__ float Ps[SIMT_BK][SIMT_BR + 1];     // [kk][row of R]
     __shared__ float Gs[SIMT_BK][SIMT_BN + 1];     // [kk][channel]
@@ -254,6 +261,8 @@ project_simt_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
         const int cols = d.cols, m = d.m, n = d.n, r = sp.rank;
         const float r_scale = d.r_scale;
         const float* __restrict__ ext_p = d.ext_p;
+        const int64_t g_extent = (int64_t)d.rows * cols, state_extent = state_elements(n, r, false);   // (debug build)
+        (void)g_extent; (void)state_extent; (void)status;
 
         float acc[4][4];
 #pragma unroll
@@ -290,13 +299,15 @@ project_simt_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                 for (int at = tid; at < SIMT_BK * SIMT_BN; at += SIMT_THREADS) {
                     const int kk = at / SIMT_BN, jj = at % SIMT_BN;
                     const int i = i0 + kk, j = j0 + jj;
-                    Gs[kk][jj] = (i < m && j < n) ? load1(G + (int64_t)i * cols + j) : 0.0f;
+                    Gs[kk][jj] = (i < m && j < n && APOLLO_DBG_RANGE((int64_t)i * cols + j, (int64_t)i * cols + j, g_extent, status))
+                                     ? load1(G + (int64_t)i * cols + j) : 0.0f;
                 }
             } else {
                 for (int at = tid; at < SIMT_BK * SIMT_BN; at += SIMT_THREADS) {
                     const int jj = at / SIMT_BK, kk = at % SIMT_BK;
                     const int i = i0 + kk, j = j0 + jj;
-                    Gs[kk][jj] = (i < m && j < n) ? load1(G + (int64_t)j * cols + i) : 0.0f;
+                    Gs[kk][jj] = (i < m && j < n && APOLLO_DBG_RANGE((int64_t)j * cols + i, (int64_t)j * cols + i, g_extent, status))
+                                     ? load1(G + (int64_t)j * cols + i) : 0.0f;
                 }
             }
             __syncthreads();
@@ -324,7 +335,7 @@ project_simt_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
 #pragma unroll
             for (int y = 0; y < 4; ++y) {
                 const int j = j0 + tx * 4 + y;
-                if (k < r && j < n) {
+                if (k < r && j < n && APOLLO_DBG_RANGE((int64_t)k * d.ns + j, (int64_t)k * d.ns + j, state_extent, status)) {
                     const float rv = acc[x][y] * r_scale;
                     const int64_t at = (int64_t)k * d.ns + j;
                     const bool sb = sp.state_bf16 != 0;
@@ -341,7 +352,8 @@ project_simt_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
 #pragma unroll
         for (int y = 0; y < 4; ++y) { red[0][ty][tx * 4 + y] = num[y]; red[1][ty][tx * 4 + y] = den[y]; }
         __syncthreads();
-        if (tid < SIMT_BN && j0 + tid < n) {
+        if (tid < SIMT_BN && j0 + tid < n &&
+            APOLLO_DBG_RANGE((int64_t)tr * n + j0 + tid, (int64_t)tr * n + j0 + tid, (int64_t)d.slices * n, status)) {
             float a = 0.f, b = 0.f;
 #pragma unroll
             for (int w = 0; w < 16; ++w) { a += red[0][w][tid]; b += red[1][w][tid]; }
@@ -359,7 +371,7 @@ project_simt_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
 constexpr int FINALIZE_THREADS = 1024;
 
 __global__ void __launch_bounds__(FINALIZE_THREADS)
-finalize_kernel(const MatDesc* __restrict__ descs, int first, StepParams sp, const int32_t* __restrict__ status)
+finalize_kernel(const MatDesc* __restrict__ descs, int first, StepParams sp, int32_t* __restrict__ status)
 {
     __shared__ double scratch[32];
     if (status && *status != STATUS_OK) return;      // the projection did not complete: leave s, prev and scal alone
@@ -370,6 +382,7 @@ finalize_kernel(const MatDesc* __restrict__ descs, int first, StepParams sp, con
 
     for (int j = threadIdx.x; j < n; j += blockDim.x) {
         float num = 0.f, den = 0.f, g2 = 0.f;
+        if (!APOLLO_DBG_RANGE(j, (int64_t)(d.slices - 1) * n + j, (int64_t)d.slices * n, status)) continue;
         if (d.path == PATH_STREAM) {
             float r = 0.f;
             for (int sl = 0; sl < d.slices; ++sl) {
@@ -446,7 +459,7 @@ __device__ __forceinline__ void store1(__nv_bfloat16* p, float v) { *p = __float
 template <typename T>
 __global__ void __launch_bounds__(UPDATE_THREADS)
 update_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix, int n_mat,
-              int tile_begin, int tile_end, StepParams sp, const int32_t* __restrict__ status)
+              int tile_begin, int tile_end, StepParams sp, int32_t* __restrict__ status)
 {
     if (status && *status != STATUS_OK) return;      // the projection did not complete: leave W alone
     for (int tile = tile_begin + blockIdx.x; tile < tile_end; tile += gridDim.x) {
@@ -479,6 +492,8 @@ update_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix,
             const int r0 = (rb * d.upd_groups + grp) * UPDATE_ROWS;
             if (grp >= d.upd_groups || c >= ecols || r0 >= erows) continue;
             const int nr = min(UPDATE_ROWS, erows - r0);
+            if (!APOLLO_DBG_RANGE((int64_t)r0 * ecols + c, (int64_t)(r0 + nr - 1) * ecols + c + 7, total, status)) continue;
+            if (!sup && !APOLLO_DBG_RANGE(tall ? r0 : (int)c, tall ? r0 + nr - 1 : (int)c + 7, d.n, status)) continue;
             float sa[8];                               // step x scale of this thread's columns (wide)
             if (sup) {
                 uint32_t col = c % cols;               // the same in every super-row
@@ -538,6 +553,7 @@ update_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix,
 
         constexpr int VECS = UPDATE_TILE / (UPDATE_THREADS * 8);   // vectors per thread per tile
         constexpr int BATCH = 4;                                   // vectors whose loads are issued together
+        if (!APOLLO_DBG_RANGE(e0, e0, total, status)) continue;
         if (e0 + UPDATE_TILE <= total) {
             // whole tile inside the matrix: every vector is full; issue a batch of loads first
 #pragma unroll 1
@@ -660,30 +676,30 @@ static int grid_for(int total_tiles, int per_sm, int sm_count)
 }
 
 void launch_project_stream(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int tile_begin, int tile_end,
-                           const StepParams& sp, int sm_count, cudaStream_t stream)
+                           const StepParams& sp, int sm_count, int32_t* d_status, cudaStream_t stream)
 {
     const int total_tiles = tile_end - tile_begin;
     if (total_tiles <= 0) return;
     const int grid = grid_for(total_tiles, 6, sm_count);
     if (dtype == 0)
-        project_stream_kernel<float><<<grid, STREAM_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end, sp);
+        project_stream_kernel<float><<<grid, STREAM_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end, sp, d_status);
     else
-        project_stream_kernel<__nv_bfloat16><<<grid, STREAM_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end, sp);
+        project_stream_kernel<__nv_bfloat16><<<grid, STREAM_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end, sp, d_status);
 }
 
 void launch_project_simt(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int tile_begin, int tile_end,
-                         const StepParams& sp, int sm_count, cudaStream_t stream)
+                         const StepParams& sp, int sm_count, int32_t* d_status, cudaStream_t stream)
 {
     const int total_tiles = tile_end - tile_begin;
     if (total_tiles <= 0) return;
     const int grid = grid_for(total_tiles, 4, sm_count);
     if (dtype == 0)
-        project_simt_kernel<float><<<grid, SIMT_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end, sp);
+        project_simt_kernel<float><<<grid, SIMT_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end, sp, d_status);
     else
-        project_simt_kernel<__nv_bfloat16><<<grid, SIMT_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end, sp);
+        project_simt_kernel<__nv_bfloat16><<<grid, SIMT_THREADS, 0, stream>>>(d_descs, d_prefix, n_mat, tile_begin, tile_end, sp, d_status);
 }
 
-void launch_finalize(const MatDesc* d_descs, int first, int count, const StepParams& sp, const int32_t* d_status,
+void launch_finalize(const MatDesc* d_descs, int first, int count, const StepParams& sp, int32_t* d_status,
                      cudaStream_t stream)
 {
     if (count <= 0) return;
@@ -691,7 +707,7 @@ void launch_finalize(const MatDesc* d_descs, int first, int count, const StepPar
 }
 
 void launch_update(int dtype, const MatDesc* d_descs, const int* d_prefix, int n_mat, int tile_begin, int tile_end,
-                   const StepParams& sp, int sm_count, const int32_t* d_status, cudaStream_t stream)
+                   const StepParams& sp, int sm_count, int32_t* d_status, cudaStream_t stream)
 {
     const int total_tiles = tile_end - tile_begin;
     if (total_tiles <= 0) return;

@@ -573,7 +573,9 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                 float rv[16];
                 ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * r_slice + cchunk * 16), rv);
                 const int j = j0 + b * 128 + ch_in_blk;
-                if (j < n) {
+                if (j < n && APOLLO_DBG_RANGE(state_at(true, 0, sp.rank, r0 + cchunk * 16, j),
+                                              state_at(true, 0, sp.rank, r0 + cchunk * 16 + 15, j),
+                                              state_elements(n, sp.rank, true), status)) {
                     const int64_t at = state_at(true, 0, sp.rank, r0 + cchunk * 16, j);     // channel blocks of 128: rows are 128 elements apart
                     const bool sb = sp.state_bf16 != 0;
                     float mv[16], vv[16];
@@ -600,7 +602,7 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
             const int parts = tall ? 1 : TC_NORM_THREADS / (16 * nblk);
             for (int ch = tid - 64; ch < chan_tile; ch += TC_EPI_THREADS) {
                 const int j = j0 + ch;
-                if (j < n) {
+                if (j < n && APOLLO_DBG_RANGE((int64_t)tr * n + j, (int64_t)tr * n + j, (int64_t)__ldg(&dp->slices) * n, status)) {
                     const float2 a = red[ch], b2 = red[chan_tile + ch], c2 = red[2 * chan_tile + ch];
                     reinterpret_cast<float2*>(part)[(int64_t)tr * n + j] = make_float2(a.x + b2.x + c2.x, a.y + b2.y + c2.y);
                     if (tr == 0) {
@@ -747,6 +749,7 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             uint4* const out = static_cast<uint4*>(gp->pstage);
             // two vectors per pass: four Philox chains in flight per thread
             for (int c = piece * per + lane; c < c_end; c += 64) {
+                if (!APOLLO_DBG_RANGE(c, c, total, status)) break;
                 const int row0 = c / vec_per_row;
                 const uint4 v0 = p_vector(ext_p, gmm, row0, c - row0 * vec_per_row, matrix_id, sp);
                 if (c + 32 < c_end) {
@@ -914,7 +917,9 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                                        (ptx::f32x2_sum(acc2[4 * pass + 2]) + ptx::f32x2_sum(acc2[4 * pass + 3]));
                     const float v = mine + __shfl_xor_sync(0xFFFFFFFFu, mine, 1);
                     const int j = j0 + ((t + pass * 128) >> 1);
-                    if (!stop && tr == 0 && !(lane & 1) && j < n) g2out[j] = v;
+                    if (!stop && tr == 0 && !(lane & 1) && j < n &&
+                        APOLLO_DBG_RANGE(j, j, (int64_t)__ldg(&dp->g2_slices) * n, status))
+                        g2out[j] = v;
                 }
             } else {
                 // lanes l and l + 16 hold two row groups of the same eight channels: one slice per warp
@@ -925,7 +930,9 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                 for (int e = 0; e < 8; ++e) {
                     const float v = acc[e] + __shfl_xor_sync(0xFFFFFFFFu, acc[e], 16);
                     const int j = j0 + cc * 8 + e;
-                    if (!stop && tr == 0 && lane < 16 && j < n) g2out[(int64_t)(warp - 4) * n + j] = v;
+                    if (!stop && tr == 0 && lane < 16 && j < n &&
+                        APOLLO_DBG_RANGE((int64_t)(warp - 4) * n + j, (int64_t)(warp - 4) * n + j, (int64_t)__ldg(&dp->g2_slices) * n, status))
+                        g2out[(int64_t)(warp - 4) * n + j] = v;
                 }
             }
             if (stop) break;
@@ -962,7 +969,9 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                 if (pf && cchunk + 2 * pf_d < chunks) ask(cchunk + 2 * pf_d);
                 float rv[16];
                 ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + buf * (uint32_t)r_slice + (uint32_t)(cchunk * 16), rv);
-                if (j < n) {
+                if (j < n && APOLLO_DBG_RANGE(tile_el + (int64_t)(r0 + cchunk * 16) * 128 + ch,
+                                              tile_el + (int64_t)(r0 + cchunk * 16 + 15) * 128 + ch,
+                                              state_elements(n, sp.rank, true), status)) {
                     const int64_t at = tile_el + (int64_t)(r0 + cchunk * 16) * 128 + ch;
                     const bool sb = sp.state_bf16 != 0;
                     float mv[16], vv[16];
@@ -987,7 +996,8 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0 && acc_ok) ptx::mbar_arrive_remote(ptx::map_to_cta(bar_acc_empty + 8 * buf, 0));
-            if (acc_ok && j < n)
+            if (acc_ok && j < n &&
+                APOLLO_DBG_RANGE((int64_t)(tr * 2 + half) * n + j, (int64_t)(tr * 2 + half) * n + j, (int64_t)__ldg(&dp->slices) * n, status))
                 reinterpret_cast<float2*>(dp->part)[(int64_t)(tr * 2 + half) * n + j] = make_float2(num, den);
             if (__shfl_sync(0xFFFFFFFFu, *abort_flag, 0) != 0) break;
         } else if (__shfl_sync(0xFFFFFFFFu, *abort_flag, 0) != 0) {

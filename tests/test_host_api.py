@@ -24,12 +24,36 @@ def test_library_exports_every_declared_symbol():
     assert declared == set(B.EXPORTS)
     for name in declared:
         assert hasattr(lib, name), name
+    # the bounds-checking build is the same library with checks compiled in
+    from paper_2412_05270_b200.build import build_library
+    import ctypes
+    debug = ctypes.CDLL(str(build_library(debug=True)))
+    for name in declared:
+        assert hasattr(debug, name), name
 
 
 def test_strerror_names_every_code():
-    for code in range(0, -10, -1):
+    for code in range(0, -11, -1):
         assert B.strerror(code) and "unknown" not in B.strerror(code)
     assert "unknown" in B.strerror(-99)
+
+
+def test_tuning_is_validated_and_sizes_the_p_scratch():
+    shapes = [(4096, 4096)] * 40
+    cfg = B.make_config(rank=256, dtype=B.DT_BF16)
+    moments = 40 * 2 * 256 * 4096 * 4
+    per_step = B.workspace_bytes(shapes, cfg)
+    kept = B.workspace_bytes(shapes, B.make_config(rank=256, dtype=B.DT_BF16, flags=B.FLAG_KEEP_P))
+    p_bytes = 256 * 4096 * 2
+    # default: a 32 MB scratch (16 slots of 2 MB); kept: one slot per matrix
+    assert per_step - moments < 48 << 20       # scratch + scales, partial sums, tables
+    assert kept - per_step == (40 - 16) * p_bytes
+    assert B.workspace_bytes(shapes, cfg, B.make_tuning(scratch_mb=8)) == per_step - (16 - 4) * p_bytes
+    for bad in (dict(kernel=2), dict(p_source=3), dict(r_slice=24), dict(r_slice=512), dict(nblk=3),
+                dict(nblk=4, r_slice=256), dict(scratch_mb=-1), dict(epi_prefetch=9), dict(p_generator=2)):
+        with pytest.raises(B.ApolloError) as err:
+            B.workspace_bytes(shapes, cfg, B.make_tuning(**bad))
+        assert err.value.code == B.ERR_INVALID_ARG, bad
 
 
 def test_workspace_grows_with_rank_and_counts_moments():
