@@ -112,7 +112,10 @@ typedef struct {
     int32_t nblk;          /* ring kernel: 128-channel blocks per tile (1, 2 or 4; nblk * r_slice <= 512); 0 = default */
     int32_t epi_prefetch;  /* pair kernel: how many 16-row chunks ahead of its loads an epilogue warp asks L2 for
                               the moments, as distance + 1 (1 = no prefetch ... 9 = eight chunks); 0 = default (one chunk) */
-    int32_t reserved;      /* 0 */
+    int32_t realign;       /* gradients whose rows start on no 16-byte boundary (cols % 8 != 0), which no tensor map
+                              can describe: 0 = default, 1 = wide ones with rows % 8 == 0 are fetched as they lie and
+                              re-aligned in shared memory by the pair kernel (no extra memory), 2 = all of them are
+                              first copied to a padded pitch (rows x round_up(cols, 8) bf16 of workspace per matrix) */
 } apollo_tuning;
 
 /*

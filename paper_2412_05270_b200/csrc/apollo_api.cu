@@ -28,7 +28,7 @@ struct NvtxRange {
 };
 
 struct MatPlan {
-    int32_t rows, cols, m, n, tall, path, slices, g2_slices, tiles_n, tiles_k;
+    int32_t rows, cols, m, n, tall, path, slices, g2_slices, tiles_n, tiles_k, raw;
     int64_t proj_tiles, update_tiles;
     size_t off_M, off_V, off_scal, off_s, off_part, off_g2, off_tmap, off_pstage, off_gpad, gpad_bytes;
 };
@@ -102,6 +102,9 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
             }
         } else if (tensor_path_supports(p.rows, p.cols, r, cfg->dtype) && !(cfg->flags & APOLLO_FLAG_NO_TENSOR_CORES)) {
             p.path = PATH_TENSOR;
+            // rows that start on no 16-byte boundary: re-aligned in shared memory where the pair kernel can, else a padded copy
+            p.raw = tensor_path_raw_ok(p.rows, p.cols, plan.tc) ? 1 : 0;
+            if (p.raw) tensor_path_enable_raw(&plan.tc);
             tensor_path_tiling(p.rows, p.cols, r, plan.tc, &p.tiles_n, &p.tiles_k, &p.slices, &p.g2_slices);
         } else {
             p.path = PATH_SIMT;
@@ -182,7 +185,7 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
     for (int i = 0; i < n_mat; ++i) {
         MatPlan& p = plan.mats[i];
         p.gpad_bytes = 0;
-        if (p.path == PATH_TENSOR && (p.cols % 8) != 0) {
+        if (p.path == PATH_TENSOR && (p.cols % 8) != 0 && !p.raw) {
             p.gpad_bytes = (size_t)p.rows * (size_t)((p.cols + 7) / 8 * 8) * 2;
             plan.any_repitch = true;
         }
@@ -352,6 +355,7 @@ int apollo_create_tuned(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_
         d.m_pad = (p.m + 63) / 64 * 64;
         d.gpad = p.gpad_bytes ? ctx->ws + p.off_gpad : nullptr;
         d.g_pitch = p.gpad_bytes ? (p.cols + 7) / 8 * 8 : p.cols;
+        d.raw = p.raw;
         d.upd_super = update_super_rows(p.rows, p.cols, p.tall != 0) ? 1 : 0;
         if (p.cols % 8 == 0 || d.upd_super) {
             const UpdateTiling ut = update_tiling(d.upd_super ? 8 * p.cols : p.cols);
@@ -679,7 +683,7 @@ int apollo_status(apollo_ctx* ctx, void* cuda_stream)
     if (ctx->first) return APOLLO_OK;   // nothing has run; the status word is not initialised yet
     if (cudaMemcpy(&word, ctx->d_status, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return APOLLO_ERR_CUDA;
     if (word != STATUS_OK) {
-        cudaMemset(ctx->d_status, 0, sizeof(word));
+        cudaMemset(ctx->d_status, 0, 2 * sizeof(word));      // the status word and the record of the wait that gave up
         return word == STATUS_BOUNDS ? APOLLO_ERR_INTERNAL : APOLLO_ERR_TIMEOUT;
     }
     return APOLLO_OK;

@@ -106,6 +106,8 @@ struct MatDesc {
     int32_t tiles_k;  // projection tiles along the other tiled axis (rows of G, or rows of R)
     int32_t m_pad;    // m rounded up to 64: row length of the staged P
     int32_t g_pitch;  // row pitch (elements) of the array the tensor path reads: cols, or cols rounded up to 8
+    int32_t raw;      // 1: wide matrix with cols % 8 != 0 and rows % 8 == 0 on the pair kernel: its G tiles are fetched
+                      //    as they lie in memory and re-aligned in shared memory (no padded copy)
     int32_t upd_chunks, upd_width, upd_groups;   // 2-D tiling of the update pass (update_tiling(cols)); 0 chunks: flat tiles
     int32_t upd_super;   // 1: the 2-D tiles run over super-rows of 8 stored rows (update_super_rows)
     float r_scale;    // factor applied to the contraction: 1/sqrt(r) for generated standard normals, 1 for a supplied P
@@ -143,8 +145,14 @@ struct TcTiling {
     int32_t keep;      // 1: every matrix owns a slot of the scratch, filled once per epoch (APOLLO_FLAG_KEEP_P)
     int32_t gen;       // 1: spare warps of the pair kernel generate P into a ring of `slots` slots, ahead of its use
     int32_t slots;     // gen: slots of the ring (matrix with tensor ordinal q uses slot q % slots)
+    int32_t raw_allowed; // tuning: matrices that qualify are re-aligned in shared memory rather than copied to a padded pitch
+    int32_t raw;       // 1: the list has matrices whose G tiles are re-aligned in shared memory (MatDesc::raw): the
+                       //    G part of a stage is RAW_G_BYTES and the norm warps arrive on the stage's `full` barrier
     int64_t scratch_bytes; // byte budget of the scratch when it is neither kept nor a ring (groups of matrices share it)
 };
+
+constexpr int RAW_BOX_W = 136;                       // elements per fetched row piece: 128 channels + up to 7 of misalignment, whole 16-byte units
+constexpr int RAW_G_BYTES = 64 * RAW_BOX_W * 2;      // 64 rows of a k-block as fetched: 17408 bytes (17 KiB)
 
 // What the generator warps of the pair kernel and the consumers of their output share (TcTiling::gen).
 // The counters are zeroed before every launch.

@@ -35,6 +35,10 @@ bool tensor_path_supports(int rows, int cols, int rank, int dtype);
 // The tiling and mode for a rank, the context's flags and the caller's tuning (may be null):
 // APOLLO_OK, or APOLLO_ERR_INVALID_ARG for a tuning value out of range.
 int tensor_path_configure(int rank, uint32_t flags, const apollo_tuning* tuning, TcTiling* out);
+// Whether the pair kernel re-aligns this matrix's G tiles in shared memory instead of reading a padded copy.
+bool tensor_path_raw_ok(int rows, int cols, const TcTiling& tl);
+// Switches the tiling to the stage layout that such matrices need (fewer, larger stages).
+void tensor_path_enable_raw(TcTiling* tl);
 void tensor_path_tiling(int rows, int cols, int rank, const TcTiling& tl, int32_t* tiles_n, int32_t* tiles_k,
                         int32_t* slices, int32_t* g2_slices);
 // Bytes one matrix's P needs in the scratch (rank x round_up(m, 64) bf16).

@@ -84,7 +84,7 @@ int tensor_path_configure(int rank, uint32_t flags, const apollo_tuning* tuning,
     if (tu.kernel != APOLLO_TC_KERNEL_PAIR && tu.kernel != APOLLO_TC_KERNEL_RING) return APOLLO_ERR_INVALID_ARG;
     if (tu.p_source != APOLLO_P_SCRATCH && tu.p_source != APOLLO_P_SHARED) return APOLLO_ERR_INVALID_ARG;
     if (tu.p_generator != 0 && tu.p_generator != 1) return APOLLO_ERR_INVALID_ARG;
-    if (tu.scratch_mb < 0 || tu.scratch_mb > 65536 || tu.reserved != 0) return APOLLO_ERR_INVALID_ARG;
+    if (tu.scratch_mb < 0 || tu.scratch_mb > 65536 || tu.realign < 0 || tu.realign > 2) return APOLLO_ERR_INVALID_ARG;
     if (tu.epi_prefetch < 0 || tu.epi_prefetch > 9) return APOLLO_ERR_INVALID_ARG;
     t.r_slice = rank <= 256 ? rank : rank / 2;
     if (tu.r_slice != 0) {
@@ -101,6 +101,7 @@ int tensor_path_configure(int rank, uint32_t flags, const apollo_tuning* tuning,
     t.keep = t.staged && (flags & APOLLO_FLAG_KEEP_P) ? 1 : 0;
     t.scratch_bytes = (int64_t)(tu.scratch_mb ? tu.scratch_mb : 32) << 20;
     t.epi_prefetch = tu.epi_prefetch ? tu.epi_prefetch - 1 : 1;
+    t.raw_allowed = tu.realign == 1 ? 1 : 0;      // default: padded copy (the faster of the two as measured)
     // Staged P has two kernels: the pair kernel (default; faster on every list measured) and the single-CTA
     // ring kernel, which is also the one that can generate P in shared memory.
     if (t.staged && tu.kernel == APOLLO_TC_KERNEL_PAIR) {   // (APOLLO_P_SHARED always runs on the ring kernel)
@@ -130,6 +131,21 @@ bool tensor_path_supports(int rows, int cols, int rank, int dtype)
     if (rank > 256 && rank % 32) return false;
     (void)rows; (void)cols;   // a row pitch that is not a multiple of 16 bytes goes through a padded copy
     return true;
+}
+
+bool tensor_path_raw_ok(int rows, int cols, const TcTiling& tl)
+{
+    return tl.pair != 0 && tl.raw_allowed != 0 && rows <= cols && (cols % 8) != 0 && (rows % 8) == 0;
+}
+
+void tensor_path_enable_raw(TcTiling* tl)
+{
+    if (!tl->pair || tl->raw) return;
+    tl->raw = 1;
+    const int stage = RAW_G_BYTES + (tl->r_slice / 2) * 128;
+    tl->stages = (TC_MAX_SMEM - 1536) / stage;
+    if (tl->stages > 8) tl->stages = 8;
+    tl->smem_bytes = tl->stages * stage + 1536;
 }
 
 void tensor_path_tiling(int rows, int cols, int rank, const TcTiling& t, int32_t* tiles_n, int32_t* tiles_k,
@@ -162,10 +178,25 @@ int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, const TcTiling& t
         // wide: 64 channels x 64 rows of G; tall: 64 contraction elements x 128 channels
         const cuuint32_t box[2] = { 64u, d.tall ? 128u : 64u };
         const cuuint32_t elem[2] = { 1u, 1u };
-        const CUresult rc = encode(&maps[2 * i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
-                                   d.gpad ? d.gpad : const_cast<void*>(d.G), dims,
-                                   strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        CUresult rc;
+        if (d.raw) {
+            // Rows of `cols` elements with cols % 8 != 0 start on no 16-byte boundary, which a tensor map cannot
+            // describe.  Eight stored rows together are whole 16-byte units: the map sees rows/8 "super-rows" of
+            // 8 cols elements, and a box is RAW_BOX_W elements of one stored row in each of 8 consecutive
+            // super-rows (rows 8 apart start at the same offset within a 16-byte unit).  No swizzle: the pieces
+            // are re-aligned in shared memory.
+            const cuuint64_t rdims[2] = { (cuuint64_t)d.cols * 8, (cuuint64_t)d.rows / 8 };
+            const cuuint64_t rstrides[1] = { (cuuint64_t)d.cols * 16 };
+            const cuuint32_t rbox[2] = { (cuuint32_t)RAW_BOX_W, 8u };
+            rc = encode(&maps[2 * i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(d.G), rdims, rstrides, rbox,
+                        elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        } else {
+            rc = encode(&maps[2 * i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                        d.gpad ? d.gpad : const_cast<void*>(d.G), dims,
+                        strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        }
         if (rc != CUDA_SUCCESS) return APOLLO_ERR_CUDA;
         if (tl.staged) {
             // staged P: rank rows of m_pad bf16, loaded as 64 x r_slice boxes (K-major UMMA tiles)
@@ -187,20 +218,25 @@ namespace {
 // status word are set; later waits return at once, so the kernel always terminates.
 // Bounded wait on an mbarrier phase.  false = this wait, or an earlier one of this CTA, gave up: the
 // caller stops issuing work and falls through to the barriers and the drain at the end of the kernel.
-__device__ __forceinline__ bool wait_phase(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status)
+// `where` names the wait (role and barrier); the first one of a launch that gives up is kept in the word after
+// the status word, for whoever has to find out what stalled.
+__device__ __forceinline__ bool wait_phase(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
+                                           int where = 0)
 {
     if (ptx::mbar_try_wait(bar, parity)) return true;      // the common case costs one poll and no flag read
     if (*abort_flag) return false;
     for (uint32_t i = 0; i < TC_WAIT_CAP; ++i)
         if (ptx::mbar_try_wait(bar, parity)) return true;
     *abort_flag = 1;
+    atomicCAS(status + 1, 0, where);
     atomicExch(status, STATUS_TIMEOUT);
     return false;
 }
 
 // The same for waits that have slack (an epilogue waiting for its accumulator): sleeps between polls,
 // which costs nothing there and saves issue slots, i.e. power, on a board that runs at its power cap.
-__device__ __forceinline__ bool wait_phase_idle(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status)
+__device__ __forceinline__ bool wait_phase_idle(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
+                                                int where = 0)
 {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
@@ -209,6 +245,7 @@ __device__ __forceinline__ bool wait_phase_idle(uint32_t bar, uint32_t parity, v
         if (ptx::mbar_try_wait(bar, parity)) return true;
     }
     *abort_flag = 1;
+    atomicCAS(status + 1, 0, where);
     atomicExch(status, STATUS_TIMEOUT);
     return false;
 }
@@ -236,7 +273,7 @@ __device__ __forceinline__ void red_release_gpu_add(uint32_t* p, uint32_t v)
 // occupancy query), so the writers run; the bound covers the case that one of them gave up.  A set status
 // word ends the wait at once.  false = gave up (abort flag and status word are set).
 __device__ __forceinline__ bool wait_counter(const uint32_t* counter, uint32_t target, volatile int* abort_flag,
-                                             int32_t* status)
+                                             int32_t* status, int where = 0)
 {
     if (ld_acquire_gpu(counter) >= target) return true;
     if (*abort_flag) return false;
@@ -246,6 +283,7 @@ __device__ __forceinline__ bool wait_counter(const uint32_t* counter, uint32_t t
         if ((i & 63u) == 63u && *reinterpret_cast<volatile int32_t*>(status) != STATUS_OK) break;
     }
     *abort_flag = 1;
+    atomicCAS(status + 1, 0, where);
     atomicExch(status, STATUS_TIMEOUT);
     return false;
 }
@@ -665,6 +703,10 @@ constexpr int P2_MAX_STAGES = 8;
 constexpr int P2_MISC_BYTES = 512 + 1024;          // barriers and flags, alignment slack
 static_assert(P2_MISC_BYTES == 1536, "tensor_path_configure() reserves this many bytes");
 
+// RAW: the list has matrices whose G tiles are re-aligned in shared memory (TcTiling::raw).  The kernel without
+// that code is a separate instantiation, so that lists without such matrices run exactly the code they ran
+// before it existed (with it compiled in, the other roles of the kernel came out 15 % slower).
+template <bool RAW>
 __global__ void __launch_bounds__(P2_THREADS, 1)
 project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix, int n_mat, int tile_begin,
                     int tile_end, StepParams sp, TcTiling tl, GenArgs gen, int32_t* __restrict__ status)
@@ -675,11 +717,15 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
 
     const uint32_t rank = ptx::cluster_ctarank();          // 0: leader, 1: peer
     const int r_slice = tl.r_slice, ns = tl.stages, r_half = r_slice / 2;
-    const uint32_t p_bytes = (uint32_t)r_half * 128u, stage_bytes = (uint32_t)P2_G_BYTES + p_bytes;
+    // the G part of a stage holds 128 channels x 64 rows in the UMMA layout (16 KiB); in a list with matrices
+    // whose rows start on no 16-byte boundary it is large enough for the 64 row pieces as fetched (17 KiB)
+    const uint32_t g_bytes = RAW ? (uint32_t)RAW_G_BYTES : (uint32_t)P2_G_BYTES;
+    const uint32_t p_bytes = (uint32_t)r_half * 128u, stage_bytes = g_bytes + p_bytes;
     const uint32_t misc = (uint32_t)ns * stage_bytes;
     const uint32_t bars = smem_base + misc;
     const uint32_t bar_full = bars, bar_done = bars + 64, bar_empty = bars + 128, bar_acc_full = bars + 192,
-                   bar_acc_empty = bars + 208, bar_drain = bars + 224;
+                   bar_acc_empty = bars + 208, bar_drain = bars + 224, bar_raw = bars + 256, bar_read = bars + 320,
+                   bar_ready = bars + 384;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + misc + 240);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + misc + 244);
 
@@ -690,6 +736,11 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             ptx::mbar_init(bar_full + 8 * s, 1);        // the leader's arrive.expect_tx
             ptx::mbar_init(bar_done + 8 * s, 1);        // the leader's commit
             ptx::mbar_init(bar_empty + 8 * s, 4);       // four norm warps of this CTA
+            // used by re-aligned tiles only; these complete one phase per such k-block, not per turn of the ring,
+            // so whoever waits on them keeps the parity of each stage's next phase in a bit mask of its own
+            ptx::mbar_init(bar_raw + 8 * s, 1);         // this CTA's arrive.expect_tx for the row pieces as fetched
+            ptx::mbar_init(bar_read + 8 * s, 4);        // the four norm warps have the row pieces in registers
+            ptx::mbar_init(bar_ready + 8 * s, 8);       // leader's copy: the norm warps of both CTAs have written the tile
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(bar_acc_full + 8 * b, 1);    // the leader's commit
@@ -714,6 +765,7 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
     // their own instruction count, and a division per k-block is a large part of it
     uint32_t it = 0, tile_iter = 0, stage = 0, phase = 0;
     auto next_stage = [&]() { ++it; if (++stage == (uint32_t)ns) { stage = 0; phase ^= 1; } };
+    uint32_t raw_bits = 0, raw_used = 0;     // bit s: parity of stage s's next re-aligned k-block; stages that had one
 
     // ---------------- generator warps (TcTiling::gen): P of every matrix of the launch, ahead of its use ----------------
     // The spare warps of all CTAs (warp 3 everywhere, warp 1 of the peers, whose MMA role is the leader's) draw
@@ -735,7 +787,7 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             if (q - tl.slots >= gen.q_begin) {
                 const int pm = __ldg(gen.mats + q - tl.slots);
                 const uint32_t need = (uint32_t)(__ldg(&descs[pm].tiles_n) * __ldg(&descs[pm].tiles_k));
-                if (lane == 0) ok = wait_counter(gen.use_done + pm, need, abort_flag, status) ? 1 : 0;
+                if (lane == 0) ok = wait_counter(gen.use_done + pm, need, abort_flag, status, 112) ? 1 : 0;
                 ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
             }
             if (!ok) break;
@@ -780,6 +832,8 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
         const int j0 = tn * 256 + (int)rank * 128, r0 = tr * r_slice;
         const int num_kb = (m + TC_BK - 1) / TC_BK;
         const uint32_t buf = tile_iter & 1, use = tile_iter >> 1;
+        // this matrix's rows start on no 16-byte boundary: its tiles are fetched as they lie and re-aligned by the norm warps
+        const bool raw_tile = RAW && __ldg(&dp->raw) != 0;
 
         if (warp == 0) {
             // ---------------- G producer (one thread in each CTA) ----------------
@@ -793,11 +847,27 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                 // there before the leader's expect_tx (the count is signed), never a phase early,
                 // because the peer's stage is only free once the leader's MMA has consumed it
                 const uint32_t full0 = ptx::map_to_cta(bar_full, 0);
+                const int cols = __ldg(&dp->cols);
                 for (int kb = 0; kb < num_kb; ++kb, next_stage()) {
                     const uint32_t s = stage;
-                    if (!wait_phase(bar_empty + 8 * s, phase ^ 1, abort_flag, status)) break;
+                    // with re-aligned tiles in the list the norm warps free a stage before the MMA has read it
+                    if (RAW && !wait_phase(bar_done + 8 * s, phase ^ 1, abort_flag, status, 101)) break;
+                    if (!wait_phase(bar_empty + 8 * s, phase ^ 1, abort_flag, status, 102)) break;
                     const uint32_t g_s = smem_base + s * stage_bytes, full = full0 + 8 * s;
-                    if (rank == 0) ptx::mbar_arrive_expect_tx(bar_full + 8 * s, 2u * stage_bytes);   // G and P of both CTAs
+                    if (raw_tile) {
+                        // 8 boxes, one per row residue b: RAW_BOX_W elements of rows 8 a + b, a = 8 kb .. 8 kb + 7,
+                        // starting at the 16-byte unit that holds channel j0 of those rows; they land on this CTA's
+                        // own barrier, the leader's `full` barrier expects the P bytes only
+                        ptx::mbar_arrive_expect_tx(bar_raw + 8 * s, (uint32_t)RAW_G_BYTES);
+                        raw_bits ^= 1u << s; raw_used |= 1u << s;
+                        if (rank == 0) ptx::mbar_arrive_expect_tx(bar_full + 8 * s, 2u * p_bytes);
+#pragma unroll
+                        for (int b = 0; b < 8; ++b)
+                            ptx::tma_load_2d_hint(g_s + b * (8 * RAW_BOX_W * 2), tmap, (b * cols + j0) & ~7, kb * 8,
+                                                  bar_raw + 8 * s, pol_g);
+                        continue;
+                    }
+                    if (rank == 0) ptx::mbar_arrive_expect_tx(bar_full + 8 * s, 2u * (P2_G_BYTES + p_bytes));   // G and P of both CTAs
                     if (tall) {
                         ptx::tma_load_2d_pair(g_s, tmap, kb * TC_BK, j0, full, pol_g);
                     } else {
@@ -820,14 +890,18 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                 if (tl.gen != 0 && mat != p_ready_mat) {
                     // every piece of this matrix's P has been written (by generic stores of other SMs): order
                     // them before this thread's loads through the async proxy
-                    p_ok = wait_counter(gen.gen_done + mat, (uint32_t)GEN_CHUNKS, abort_flag, status);
+                    p_ok = wait_counter(gen.gen_done + mat, (uint32_t)GEN_CHUNKS, abort_flag, status, 105);
                     ptx::fence_proxy_async_global();
                     p_ready_mat = mat;
                 }
                 for (int kb = 0; p_ok && kb < num_kb; ++kb, next_stage()) {
                     const uint32_t s = stage;
-                    if (!wait_phase(bar_empty + 8 * s, phase ^ 1, abort_flag, status)) break;
-                    ptx::tma_load_2d_pair(smem_base + s * stage_bytes + P2_G_BYTES, tmap_p, kb * TC_BK, p_row, full0 + 8 * s, pol_p);
+                    // The P part of a stage is read by the MMA alone.  Without re-aligned tiles in the list `empty`
+                    // (the norm warps, who wait for the MMA) says that it is free; with them the norm warps may
+                    // free a stage before this thread has even filled it, and the MMA's own commit is the signal.
+                    if (RAW ? !wait_phase(bar_done + 8 * s, phase ^ 1, abort_flag, status, 103)
+                            : !wait_phase(bar_empty + 8 * s, phase ^ 1, abort_flag, status, 104)) break;
+                    ptx::tma_load_2d_pair(smem_base + s * stage_bytes + g_bytes, tmap_p, kb * TC_BK, p_row, full0 + 8 * s, pol_p);
                 }
             }
             __syncwarp();
@@ -837,18 +911,22 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             if (lane == 0 && rank == 0) {
                 const uint32_t idesc = ptx::instr_desc_bf16((uint32_t)r_slice, !tall, 256u);
                 const uint32_t d_tmem = tmem_base + buf * (uint32_t)r_slice;
-                bool ok = wait_phase(bar_acc_empty + 8 * buf, (use & 1) ^ 1, abort_flag, status);   // epilogue of the tile before last
+                bool ok = wait_phase(bar_acc_empty + 8 * buf, (use & 1) ^ 1, abort_flag, status, 106);   // epilogue of the tile before last
                 ptx::tc_fence_after_sync();
                 // descriptors of stage 0, k-step 0; the start-address field (bits 0..13, address >> 4) is the
                 // only one that moves, and shared-memory addresses stay below 2^18, so it never carries out
                 const uint64_t a_desc0 = tall ? ptx::smem_desc_sw128(smem_base, 16, 1024)
                                               : ptx::smem_desc_sw128(smem_base, P2_G_BYTES / 2, 1024);
-                const uint64_t b_desc0 = ptx::smem_desc_sw128(smem_base + P2_G_BYTES, 16, 1024);
+                const uint64_t b_desc0 = ptx::smem_desc_sw128(smem_base + g_bytes, 16, 1024);
                 const uint32_t a_step = tall ? 32u >> 4 : 2048u >> 4, stage_step = stage_bytes >> 4;
                 int kb = 0;
                 for (; ok && kb < num_kb; ++kb, next_stage()) {
                     const uint32_t s = stage;
-                    if (!wait_phase(bar_full + 8 * s, phase, abort_flag, status)) break;
+                    if (!wait_phase(bar_full + 8 * s, phase, abort_flag, status, 107)) break;
+                    if (raw_tile) {        // the G tile was written by the norm warps of both CTAs
+                        if (!wait_phase(bar_ready + 8 * s, (raw_bits >> s) & 1u, abort_flag, status, 113)) break;
+                        raw_bits ^= 1u << s;
+                    }
                     ptx::tc_fence_after_sync();
                     const uint64_t a_desc = a_desc0 + s * stage_step, b_desc = b_desc0 + s * stage_step;
 #pragma unroll
@@ -869,10 +947,90 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc2[e] = 0ull;
             const int cc = t & 15, part = t >> 4;     // wide: 16 chunk columns x 8 row groups
+            const uint32_t ready_leader = ptx::map_to_cta(bar_ready, 0);
+            const int cols = __ldg(&dp->cols);
             for (int kb = 0; kb < num_kb; ++kb, next_stage()) {
                 const uint32_t s = stage, ph = phase;
-                if (!__all_sync(0xFFFFFFFFu, wait_phase(bar_done + 8 * s, ph, abort_flag, status))) break;   // landed, and the MMA has read it
                 const uint32_t g_s = smem_base + s * stage_bytes;
+                if (raw_tile) {
+                    // ---- re-align the row pieces as fetched into the UMMA layout, in place, before the MMA ----
+                    // The stage holds 8 boxes (row residue b) of 8 rows (a) of RAW_BOX_W elements; row 8 a + b of the
+                    // k-block starts (b cols + j0) mod 8 elements into its piece.  This warp takes the residues
+                    // 2 (warp - 4) and + 1; a lane takes one 16-byte chunk column c of one 64-channel half h for two
+                    // rows a per (b, h): a quarter-warp reads 128 contiguous bytes of one piece and writes the eight
+                    // chunks of one row of the swizzled tile (no bank conflicts either way).  All pieces are read into
+                    // registers (and shifted into place there) before the first write: the tile overwrites them.
+                    const uint32_t rph = (raw_bits >> s) & 1u;
+                    raw_bits ^= 1u << s;
+                    const bool ok = __all_sync(0xFFFFFFFFu, wait_phase(bar_raw + 8 * s, rph, abort_flag, status, 108));
+                    const int c = lane & 7, a_lo = lane >> 3;
+                    uint4 o[8];
+                    if (ok) {
+#pragma unroll
+                        for (int pass = 0; pass < 8; ++pass) {
+                            const int b = 2 * (warp - 4) + (pass >> 2), h = (pass >> 1) & 1, a = a_lo + 4 * (pass & 1);
+                            const uint32_t src = g_s + (uint32_t)((b * 8 + a) * (RAW_BOX_W * 2) + (h * 8 + c) * 16);
+                            const uint4 lo = ld_shared_v4(src), hi = ld_shared_v4(src + 16);
+                            const uint32_t mis = (uint32_t)((b * cols + j0) & 7) * 2u, wsel = mis >> 2, sh = (mis & 2u) * 8u;
+                            const uint32_t w[8] = { lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w };
+                            uint32_t v[4];
+                            switch (wsel) {          // uniform over the warp
+                            case 0:
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) v[k] = __funnelshift_r(w[k], w[k + 1], sh);
+                                break;
+                            case 1:
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) v[k] = __funnelshift_r(w[k + 1], w[k + 2], sh);
+                                break;
+                            case 2:
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) v[k] = __funnelshift_r(w[k + 2], w[k + 3], sh);
+                                break;
+                            default:
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) v[k] = __funnelshift_r(w[k + 3], w[k + 4], sh);
+                                break;
+                            }
+                            // channels at and beyond the end of the row hold the next row's elements: zero them
+                            const int jc = j0 + h * 64 + c * 8;
+                            if (jc + 8 > cols) {
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) {
+                                    if (jc + 2 * k >= cols) v[k] = 0u;
+                                    else if (jc + 2 * k + 1 >= cols) v[k] &= 0xFFFFu;
+                                }
+                            }
+                            o[pass] = make_uint4(v[0], v[1], v[2], v[3]);
+                        }
+                    }
+                    // all four norm warps have read before anyone writes (a bounded wait like every other: a warp
+                    // that gave up does not arrive, and the others give up in turn)
+                    __syncwarp();
+                    if (!ok) break;
+                    if (lane == 0) ptx::mbar_arrive(bar_read + 8 * s);
+                    if (!__all_sync(0xFFFFFFFFu, wait_phase(bar_read + 8 * s, rph, abort_flag, status, 109))) break;
+#pragma unroll
+                    for (int pass = 0; pass < 8; ++pass) {
+                        const int b = 2 * (warp - 4) + (pass >> 2), h = (pass >> 1) & 1, a = a_lo + 4 * (pass & 1);
+                        const int krow = 8 * a + b;      // row of the k-block
+                        st_shared_v4(g_s + (uint32_t)(h * (P2_G_BYTES / 2) + krow * 128 + ((c ^ (krow & 7)) << 4)), o[pass]);
+                        if (tr == 0) {
+                            ptx::fma_sq_f32x2(acc2[h * 4 + 0], ptx::bf16x2_to_f32x2(o[pass].x));
+                            ptx::fma_sq_f32x2(acc2[h * 4 + 1], ptx::bf16x2_to_f32x2(o[pass].y));
+                            ptx::fma_sq_f32x2(acc2[h * 4 + 2], ptx::bf16x2_to_f32x2(o[pass].z));
+                            ptx::fma_sq_f32x2(acc2[h * 4 + 3], ptx::bf16x2_to_f32x2(o[pass].w));
+                        }
+                    }
+                    ptx::fence_proxy_async_smem();      // the tile was written by plain stores; the MMA reads it through the async proxy
+                    __syncwarp();
+                    if (lane == 0) {
+                        ptx::mbar_arrive_remote(ready_leader + 8 * s);
+                        ptx::mbar_arrive(bar_empty + 8 * s);      // the producers also wait for the MMA's commit before refilling
+                    }
+                    continue;
+                }
+                if (!__all_sync(0xFFFFFFFFu, wait_phase(bar_done + 8 * s, ph, abort_flag, status, 110))) break;   // landed, and the MMA has read it
                 if (tr != 0) {
                     // the norms belong to the channel tile, not to the row slice: the first slice has them
                 } else if (tall) {
@@ -909,7 +1067,23 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             // squared norms of this tile's channels -> global slices (only the first row slice writes them)
             const bool stop = __shfl_sync(0xFFFFFFFFu, *abort_flag, 0) != 0;     // one answer per warp
             float* const g2out = dp->g2;
-            if (tall) {
+            if (raw_tile) {
+                // lanes with the same chunk column (lane & 7) hold the rows a = lane >> 3 (+ 4) of the same 16 channels:
+                // 8 of half 0 in acc2[0..3], 8 of half 1 in acc2[4..7]; one slice per warp (its two row residues)
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    float x0, x1;
+                    ptx::f32x2_unpack(acc2[i], x0, x1);
+                    x0 += __shfl_xor_sync(0xFFFFFFFFu, x0, 8);  x1 += __shfl_xor_sync(0xFFFFFFFFu, x1, 8);
+                    x0 += __shfl_xor_sync(0xFFFFFFFFu, x0, 16); x1 += __shfl_xor_sync(0xFFFFFFFFu, x1, 16);
+                    const int j = j0 + (i >> 2) * 64 + (lane & 7) * 8 + 2 * (i & 3);
+                    if (!stop && tr == 0 && lane < 8) {
+                        float* const out = g2out + (int64_t)(warp - 4) * n;
+                        if (j < n && APOLLO_DBG_RANGE((int64_t)(warp - 4) * n + j, (int64_t)(warp - 4) * n + j, (int64_t)__ldg(&dp->g2_slices) * n, status)) out[j] = x0;
+                        if (j + 1 < n && APOLLO_DBG_RANGE((int64_t)(warp - 4) * n + j + 1, (int64_t)(warp - 4) * n + j + 1, (int64_t)__ldg(&dp->g2_slices) * n, status)) out[j + 1] = x1;
+                    }
+                }
+            } else if (tall) {
                 // lanes 2k and 2k+1 hold the two halves of one stored row
 #pragma unroll
                 for (int pass = 0; pass < 2; ++pass) {
@@ -959,7 +1133,7 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             if (pf)
                 for (int a = 0; a < pf_d; ++a)
                     if (half + 2 * a < r_slice / 16) ask(half + 2 * a);
-            const bool acc_ok = __all_sync(0xFFFFFFFFu, wait_phase_idle(bar_acc_full + 8 * buf, use & 1, abort_flag, status));   // tcgen05.ld needs the whole warp
+            const bool acc_ok = __all_sync(0xFFFFFFFFu, wait_phase_idle(bar_acc_full + 8 * buf, use & 1, abort_flag, status, 111));   // tcgen05.ld needs the whole warp
             ptx::tc_fence_after_sync();
             // the MMAs of this tile are done, so both CTAs' last P tiles have been read: one count per pair tile
             if (tl.gen != 0 && rank == 0 && warp == 8 && lane == 0 && acc_ok) red_release_gpu_add(gen.use_done + mat, 1u);
@@ -1007,10 +1181,11 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
 
     // The leader lets the loads of both CTAs (they are counted on its barriers) and its MMAs finish
     // before either CTA gives up shared memory or TMEM; on the normal path these return at once.
-    if (rank == 0 && tid == 0) {
+    if (tid == 0) {
         for (uint32_t s = 0; s < (uint32_t)ns && s < it; ++s) {
             const uint32_t last = s + (it - 1 - s) / ns * ns;
-            drain_phase(bar_full + 8 * s, (last / ns) & 1);
+            if (rank == 0) drain_phase(bar_full + 8 * s, (last / ns) & 1);
+            if ((raw_used >> s) & 1u) drain_phase(bar_raw + 8 * s, ((raw_bits >> s) & 1u) ^ 1u);     // row pieces land on each CTA's own barrier
         }
     }
     if (rank == 0 && tid == 32) {
@@ -1160,7 +1335,8 @@ void launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_ma
     // the shared-memory opt-in is a per-device attribute of the kernels: set once per context
     if (!state.attr_set) {
         cudaFuncSetAttribute(project_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
-        cudaFuncSetAttribute(project_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
+        cudaFuncSetAttribute(project_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
+        cudaFuncSetAttribute(project_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
         state.attr_set = true;
     }
     if (tl.pair) {
@@ -1178,7 +1354,9 @@ void launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_ma
         // (a pair sits in one GPC, so this can be fewer than half the SMs)
         if (state.max_pairs == 0) {
             int clusters = 0;
-            if (cudaOccupancyMaxActiveClusters(&clusters, project_pair_kernel, &cfg) != cudaSuccess || clusters < 1) {
+            const cudaError_t oe = tl.raw ? cudaOccupancyMaxActiveClusters(&clusters, project_pair_kernel<true>, &cfg)
+                                          : cudaOccupancyMaxActiveClusters(&clusters, project_pair_kernel<false>, &cfg);
+            if (oe != cudaSuccess || clusters < 1) {
                 cudaGetLastError();
                 clusters = sm_count / 2;
             }
@@ -1187,7 +1365,10 @@ void launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_ma
         int pairs = state.max_pairs;
         if (tiles < pairs) pairs = tiles;
         cfg.gridDim = dim3(2 * pairs);
-        cudaLaunchKernelEx(&cfg, project_pair_kernel, d_descs, d_prefix, n_mat, tile_begin, tile_end, sp, tl, gen, d_status);
+        if (tl.raw)
+            cudaLaunchKernelEx(&cfg, project_pair_kernel<true>, d_descs, d_prefix, n_mat, tile_begin, tile_end, sp, tl, gen, d_status);
+        else
+            cudaLaunchKernelEx(&cfg, project_pair_kernel<false>, d_descs, d_prefix, n_mat, tile_begin, tile_end, sp, tl, gen, d_status);
         return;
     }
     const int grid = tiles < sm_count ? tiles : sm_count;

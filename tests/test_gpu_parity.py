@@ -66,11 +66,19 @@ def test_streaming_path_spanning_row_blocks_and_column_tiles():
     (256, [(512, 1376), (1376, 512), (512, 512)]),
     (512, [(512, 1376), (1376, 512)]),
     (48, [(96, 200), (200, 96)]),
-    (32, [(200, 333), (336, 203), (64, 77)]),      # row pitch not a multiple of 16 bytes: padded copy
+    # row pitch not a multiple of 16 bytes.  Wide with rows % 8 == 0: tiles fetched as they lie and re-aligned in
+    # shared memory; tall, or rows % 8 != 0: padded copy.  Mixed with aligned matrices in one list.
+    (32, [(200, 333), (336, 203), (64, 77)]),
+    (64, [(264, 1029), (200, 1000), (200, 1001), (204, 333), (1000, 203)]),
+    (256, [(512, 1381), (512, 1376), (256, 257)]),
+    (512, [(512, 1381), (1376, 512), (512, 515)]),  # two row slices per channel tile
 ])
 def test_tensor_core_path(rank, shapes):
     wl = _wl(shapes, rank, dtype="bf16", steps=4, T=2, wd=0.01)
     run_parity(wl, expect_path=B.PATH_TENSOR)
+    if any(c % 8 for _, c in shapes):
+        # the same list with the unaligned wide matrices re-aligned in shared memory instead of copied
+        run_parity(wl, expect_path=B.PATH_TENSOR, tuning=B.make_tuning(realign=1))
 
 
 MODES = [
