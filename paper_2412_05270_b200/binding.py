@@ -65,14 +65,14 @@ class Tuning(ctypes.Structure):
     """apollo_tuning: zero fields select the defaults."""
     _fields_ = [("kernel", ctypes.c_int32), ("p_source", ctypes.c_int32), ("p_generator", ctypes.c_int32),
                 ("scratch_mb", ctypes.c_int32), ("r_slice", ctypes.c_int32), ("nblk", ctypes.c_int32),
-                ("epi_prefetch", ctypes.c_int32), ("realign", ctypes.c_int32)]
+                ("epi_prefetch", ctypes.c_int32), ("realign", ctypes.c_int32), ("repitch_mb", ctypes.c_int32)]
 
 
 def make_tuning(kernel=TC_KERNEL_PAIR, p_source=P_SCRATCH, p_generator=0, scratch_mb=0, r_slice=0, nblk=0,
-                epi_prefetch=None, realign=0) -> Tuning:
+                epi_prefetch=None, realign=0, repitch_mb=0) -> Tuning:
     """epi_prefetch: distance in chunks (0 = no prefetch), None = the default."""
     return Tuning(int(kernel), int(p_source), int(p_generator), int(scratch_mb), int(r_slice), int(nblk),
-                  0 if epi_prefetch is None else int(epi_prefetch) + 1, int(realign))
+                  0 if epi_prefetch is None else int(epi_prefetch) + 1, int(realign), int(repitch_mb))
 
 
 _lib = None

@@ -7,6 +7,7 @@
 #include <cmath>
 #include <cstring>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "apollo_internal.h"
@@ -44,6 +45,7 @@ struct Plan {
     bool any_repitch;
     int64_t tiles[4];   // stream, simt, tensor, update
     std::vector<StageGroup> groups;
+    std::vector<std::pair<int, int>> rp_groups;   // matrix ranges whose padded gradient copies share the repitch buffer
     TcTiling tc;                    // tiling and mode of the tensor-core projection
     std::vector<int32_t> tensor_mats;   // tensor ordinal -> matrix index
     std::vector<int32_t> tq_prefix;     // matrix index -> number of tensor-path matrices before it
@@ -182,14 +184,31 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
     plan.off_stage = off; off = align_up(off + plan.stage_bytes);
     // padded copies of the gradients whose row pitch TMA cannot take (cols not a multiple of 8)
     plan.any_repitch = false;
-    for (int i = 0; i < n_mat; ++i) {
-        MatPlan& p = plan.mats[i];
-        p.gpad_bytes = 0;
-        if (p.path == PATH_TENSOR && (p.cols % 8) != 0 && !p.raw) {
-            p.gpad_bytes = (size_t)p.rows * (size_t)((p.cols + 7) / 8 * 8) * 2;
-            plan.any_repitch = true;
+    plan.rp_groups.clear();
+    {
+        // consecutive matrices share the buffer until their copies would exceed the budget; then the next group
+        // starts again at its beginning (each group is copied and projected before the next one is copied)
+        const size_t budget = plan.tc.repitch_bytes > 0 ? (size_t)plan.tc.repitch_bytes : (size_t)-1;
+        size_t used = 0, largest = 0;
+        int begin = 0;
+        for (int i = 0; i < n_mat; ++i) {
+            MatPlan& p = plan.mats[i];
+            p.gpad_bytes = 0;
+            if (p.path == PATH_TENSOR && (p.cols % 8) != 0 && !p.raw) {
+                p.gpad_bytes = align_up((size_t)p.rows * (size_t)((p.cols + 7) / 8 * 8) * 2);
+                plan.any_repitch = true;
+            }
+            if (used > 0 && p.gpad_bytes > 0 && (used >= budget || p.gpad_bytes > budget - used)) {
+                plan.rp_groups.push_back({ begin, i });
+                begin = i;
+                used = 0;
+            }
+            p.off_gpad = off + used;
+            used += p.gpad_bytes;
+            if (used > largest) largest = used;
         }
-        p.off_gpad = off; off = align_up(off + p.gpad_bytes);
+        plan.rp_groups.push_back({ begin, n_mat });
+        off = align_up(off + largest);
     }
     plan.zero_begin = off;
     for (int i = 0; i < n_mat; ++i) {
@@ -550,10 +569,19 @@ static int step_range(apollo_ctx* ctx, int first, int count, void* const* d_W, c
                             ctx->d_status, stream);
         ++launches;
     }
-    if (tiles_of(PATH_TENSOR, first, last, tb, te)) {
+    // The padded copies of gradients with an unaligned row pitch share one buffer group by group (one group
+    // when there are none): each group's part of the range is copied, then projected, before the next is copied.
+    for (const std::pair<int, int>& rg : plan.rp_groups) {
+        const int ra = rg.first > first ? rg.first : first;
+        const int rb = rg.second < last ? rg.second : last;
+        if (rb <= ra || !tiles_of(PATH_TENSOR, ra, rb, tb, te)) continue;
         if (plan.any_repitch) {
-            launch_repitch(ctx->d_descs, first, count, stream);
-            ++launches;
+            bool any = false;
+            for (int i = ra; i < rb; ++i) any |= ctx->h_descs[i].gpad != nullptr;
+            if (any) {
+                launch_repitch(ctx->d_descs, ra, rb - ra, stream);
+                ++launches;
+            }
         }
         const TcTiling& tc = plan.tc;
         GenArgs gen = {};
@@ -563,7 +591,7 @@ static int step_range(apollo_ctx* ctx, int first, int count, void* const* d_W, c
             uint32_t* counters = reinterpret_cast<uint32_t*>(ctx->ws + plan.off_counters);
             if (cudaMemsetAsync(counters, 0, plan.counter_bytes, stream) != cudaSuccess) return APOLLO_ERR_CUDA;
             gen.mats = reinterpret_cast<const int32_t*>(ctx->ws + plan.off_tmats);
-            gen.q_begin = plan.tq_prefix[first]; gen.q_end = plan.tq_prefix[last];
+            gen.q_begin = plan.tq_prefix[ra]; gen.q_end = plan.tq_prefix[rb];
             gen.ticket = counters; gen.gen_done = counters + 1; gen.use_done = counters + 1 + ctx->n_mat;
             launch_project_tensor(ctx->d_descs, ctx->d_prefix[PATH_TENSOR], ctx->n_mat, tb, te, sp, tc, gen,
                                   ctx->tc_state, ctx->sm_count, ctx->d_status, stream);
@@ -571,8 +599,8 @@ static int step_range(apollo_ctx* ctx, int first, int count, void* const* d_W, c
         } else {
             for (const StageGroup& g : plan.groups) {
                 // the part of this staging group inside the range
-                const int mb = g.mat_begin > first ? g.mat_begin : first;
-                const int me = g.mat_end < last ? g.mat_end : last;
+                const int mb = g.mat_begin > ra ? g.mat_begin : ra;
+                const int me = g.mat_end < rb ? g.mat_end : rb;
                 if (me <= mb || !tiles_of(PATH_TENSOR, mb, me, tb, te)) continue;
                 if (tc.staged) {
                     // P changes only with the epoch (every T steps).  When every matrix keeps its own slot

@@ -148,6 +148,7 @@ struct TcTiling {
     int32_t raw_allowed; // tuning: matrices that qualify are re-aligned in shared memory rather than copied to a padded pitch
     int32_t raw;       // 1: the list has matrices whose G tiles are re-aligned in shared memory (MatDesc::raw): the
                        //    G part of a stage is RAW_G_BYTES and the norm warps arrive on the stage's `full` barrier
+    int64_t repitch_bytes; // byte budget of the padded copies of gradients with an unaligned row pitch (shared group by group)
     int64_t scratch_bytes; // byte budget of the scratch when it is neither kept nor a ring (groups of matrices share it)
 };
 

@@ -85,6 +85,7 @@ int tensor_path_configure(int rank, uint32_t flags, const apollo_tuning* tuning,
     if (tu.p_source != APOLLO_P_SCRATCH && tu.p_source != APOLLO_P_SHARED) return APOLLO_ERR_INVALID_ARG;
     if (tu.p_generator != 0 && tu.p_generator != 1) return APOLLO_ERR_INVALID_ARG;
     if (tu.scratch_mb < 0 || tu.scratch_mb > 65536 || tu.realign < 0 || tu.realign > 2) return APOLLO_ERR_INVALID_ARG;
+    if (tu.repitch_mb < 0 || tu.repitch_mb > 65536) return APOLLO_ERR_INVALID_ARG;
     if (tu.epi_prefetch < 0 || tu.epi_prefetch > 9) return APOLLO_ERR_INVALID_ARG;
     t.r_slice = rank <= 256 ? rank : rank / 2;
     if (tu.r_slice != 0) {
@@ -100,6 +101,7 @@ int tensor_path_configure(int rank, uint32_t flags, const apollo_tuning* tuning,
     t.staged = tu.p_source == APOLLO_P_SCRATCH ? 1 : 0;
     t.keep = t.staged && (flags & APOLLO_FLAG_KEEP_P) ? 1 : 0;
     t.scratch_bytes = (int64_t)(tu.scratch_mb ? tu.scratch_mb : 32) << 20;
+    t.repitch_bytes = (int64_t)tu.repitch_mb << 20;      // 0: no limit, every matrix has its own copy (one projection launch)
     t.epi_prefetch = tu.epi_prefetch ? tu.epi_prefetch - 1 : 1;
     t.raw_allowed = tu.realign == 1 ? 1 : 0;      // default: padded copy (the faster of the two as measured)
     // Staged P has two kernels: the pair kernel (default; faster on every list measured) and the single-CTA

@@ -79,6 +79,9 @@ def test_tensor_core_path(rank, shapes):
     if any(c % 8 for _, c in shapes):
         # the same list with the unaligned wide matrices re-aligned in shared memory instead of copied
         run_parity(wl, expect_path=B.PATH_TENSOR, tuning=B.make_tuning(realign=1))
+        # and with a 1 MB buffer for the padded copies: the matrices share it group by group
+        run_parity(wl, expect_path=B.PATH_TENSOR, tuning=B.make_tuning(repitch_mb=1))
+        run_parity(wl, flags=B.FLAG_KEEP_P, expect_path=B.PATH_TENSOR, tuning=B.make_tuning(repitch_mb=1))
 
 
 MODES = [
