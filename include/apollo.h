@@ -108,7 +108,8 @@ typedef struct {
                               kernel generate the projections a few matrices ahead of their use (default);
                               1 = a separate kernel fills the scratch group by group between projection launches */
     int32_t scratch_mb;    /* size of the P scratch in MB; 0 = default (32) */
-    int32_t r_slice;       /* rows of R per tile: a multiple of 16 that divides the rank, <= 256; 0 = default */
+    int32_t r_slice;       /* rows of R per tile: a multiple of 16, <= 256, that divides the rank rounded up to a
+                              multiple of 16 (32 above 256); 0 = default */
     int32_t nblk;          /* ring kernel: 128-channel blocks per tile (1, 2 or 4; nblk * r_slice <= 512); 0 = default */
     int32_t epi_prefetch;  /* pair kernel: how many 16-row chunks ahead of its loads an epilogue warp asks L2 for
                               the moments, as distance + 1 (1 = no prefetch ... 9 = eight chunks); 0 = default (one chunk) */

@@ -46,6 +46,7 @@ struct Plan {
     int64_t tiles[4];   // stream, simt, tensor, update
     std::vector<StageGroup> groups;
     std::vector<std::pair<int, int>> rp_groups;   // matrix ranges whose padded gradient copies share the repitch buffer
+    int tc_rank;                    // the rank the tensor path works with (rounded up to the MMA's granularity)
     TcTiling tc;                    // tiling and mode of the tensor-core projection
     std::vector<int32_t> tensor_mats;   // tensor ordinal -> matrix index
     std::vector<int32_t> tq_prefix;     // matrix index -> number of tensor-path matrices before it
@@ -74,8 +75,10 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
     int rc = validate_config(cfg);
     if (rc != APOLLO_OK) return rc;
     plan.tc = TcTiling{};
+    plan.tc_rank = cfg->rank;
     if (cfg->rank >= 16) {
-        rc = tensor_path_configure(cfg->rank, cfg->flags, tuning, &plan.tc);
+        plan.tc_rank = tensor_path_padded_rank(cfg->rank);
+        rc = tensor_path_configure(plan.tc_rank, cfg->flags, tuning, &plan.tc);
         if (rc != APOLLO_OK) return rc;
     }
     plan.mats.resize(n_mat);
@@ -107,7 +110,7 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
             // rows that start on no 16-byte boundary: re-aligned in shared memory where the pair kernel can, else a padded copy
             p.raw = tensor_path_raw_ok(p.rows, p.cols, plan.tc) ? 1 : 0;
             if (p.raw) tensor_path_enable_raw(&plan.tc);
-            tensor_path_tiling(p.rows, p.cols, r, plan.tc, &p.tiles_n, &p.tiles_k, &p.slices, &p.g2_slices);
+            tensor_path_tiling(p.rows, p.cols, plan.tc_rank, plan.tc, &p.tiles_n, &p.tiles_k, &p.slices, &p.g2_slices);
         } else {
             p.path = PATH_SIMT;
             p.tiles_n = (p.n + SIMT_BN - 1) / SIMT_BN;
@@ -147,7 +150,7 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
     if (plan.tc.gen && !plan.tensor_mats.empty()) {
         size_t slot = 0;
         for (int i : plan.tensor_mats) {
-            const size_t need = align_up(tensor_path_stage_bytes(plan.mats[i].rows, plan.mats[i].cols, r));
+            const size_t need = align_up(tensor_path_stage_bytes(plan.mats[i].rows, plan.mats[i].cols, plan.tc_rank));
             if (need > slot) slot = need;
         }
         int64_t slots = plan.tc.scratch_bytes / (int64_t)slot;
@@ -166,7 +169,7 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
         for (int i = 0; i < n_mat; ++i) {
             MatPlan& p = plan.mats[i];
             const bool tensor = p.path == PATH_TENSOR;
-            const size_t need = tensor && plan.tc.staged ? align_up(tensor_path_stage_bytes(p.rows, p.cols, r)) : 0;
+            const size_t need = tensor && plan.tc.staged ? align_up(tensor_path_stage_bytes(p.rows, p.cols, plan.tc_rank)) : 0;
             if (used > 0 && (used >= budget || need > budget - used)) {
                 g.mat_end = i; g.tile_end = tile_at;
                 plan.groups.push_back(g);
@@ -213,7 +216,7 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
     plan.zero_begin = off;
     for (int i = 0; i < n_mat; ++i) {
         MatPlan& p = plan.mats[i];
-        const size_t state = ((cfg->flags & APOLLO_FLAG_BF16_STATES) ? 2 : sizeof(float)) * (size_t)state_elements(p.n, r, p.path == PATH_TENSOR);
+        const size_t state = ((cfg->flags & APOLLO_FLAG_BF16_STATES) ? 2 : sizeof(float)) * (size_t)state_elements(p.n, p.path == PATH_TENSOR ? plan.tc_rank : r, p.path == PATH_TENSOR);
         p.off_M = off; off = align_up(off + state);
         p.off_V = off; off = align_up(off + state);
         p.off_scal = off; off += ALIGN;     // scal[4] then prev at float index 8
@@ -506,7 +509,7 @@ static int step_range(apollo_ctx* ctx, int first, int count, void* const* d_W, c
             changed = true;
         }
         if ((g_moved || ctx->first) && d.path == PATH_TENSOR) {
-            const int rc = tensor_path_prepare(&d, 1, cfg.rank, plan.tc, ctx->h_maps.data() + 256 * (size_t)i);
+            const int rc = tensor_path_prepare(&d, 1, plan.tc_rank, plan.tc, ctx->h_maps.data() + 256 * (size_t)i);
             if (rc != APOLLO_OK) return rc;
         }
     }
@@ -539,6 +542,7 @@ static int step_range(apollo_ctx* ctx, int first, int count, void* const* d_W, c
     sp.state_bf16 = (cfg.flags & APOLLO_FLAG_BF16_STATES) ? 1 : 0;
     sp.epoch = (uint32_t)(ctx->t / cfg.T);
     sp.rank = cfg.rank; sp.mode = cfg.mode;
+    sp.rank_pad = plan.tc_rank;
     sp.inv_sqrt_r = (float)(1.0 / std::sqrt((double)cfg.rank));
     sp.lr = lr; sp.wd = wd; sp.alpha = cfg.alpha; sp.gamma = cfg.gamma;
     sp.beta1 = cfg.beta1; sp.beta2 = cfg.beta2; sp.eps = cfg.eps;
@@ -685,8 +689,8 @@ int apollo_get_state(apollo_ctx* ctx, int32_t matrix, float* d_M, float* d_V, vo
     const bool bf16 = (ctx->cfg.flags & APOLLO_FLAG_BF16_STATES) != 0;
     if (bf16 || d.state_tiled) {
         // the caller gets dense fp32 rows whatever the library's layout and storage type
-        launch_state_copy(d.M, d_M, (int)r, d.n, d.ns, d.state_tiled != 0, bf16 ? 2 : 4, 4, true, stream);
-        launch_state_copy(d.V, d_V, (int)r, d.n, d.ns, d.state_tiled != 0, bf16 ? 2 : 4, 4, true, stream);
+        launch_state_copy(d.M, d_M, (int)r, ctx->plan.tc_rank, d.n, d.ns, d.state_tiled != 0, bf16 ? 2 : 4, 4, true, stream);
+        launch_state_copy(d.V, d_V, (int)r, ctx->plan.tc_rank, d.n, d.ns, d.state_tiled != 0, bf16 ? 2 : 4, 4, true, stream);
         return cuda_ok(cudaGetLastError()) ? APOLLO_OK : APOLLO_ERR_CUDA;
     }
     // the library's rows have pitch ns; the caller gets them dense
@@ -744,7 +748,7 @@ static int state_copy(apollo_ctx* ctx, char* d_flat, bool to_flat, cudaStream_t 
         for (int k = 0; k < 2; ++k) {
             if (d.state_tiled) {
                 const int esz = (int)state_elem_bytes(ctx);
-                launch_state_copy(parts[k], d_flat + at, (int)r, d.n, d.ns, true, esz, esz, to_flat, stream);
+                launch_state_copy(parts[k], d_flat + at, (int)r, ctx->plan.tc_rank, d.n, d.ns, true, esz, esz, to_flat, stream);
                 if (!cuda_ok(cudaGetLastError())) return APOLLO_ERR_CUDA;
             } else {
                 const cudaError_t e = to_flat
@@ -773,6 +777,10 @@ int apollo_state_export(apollo_ctx* ctx, void* d_out, void* cuda_stream)
 int apollo_state_import(apollo_ctx* ctx, const void* d_in, int64_t step_count, void* cuda_stream)
 {
     if (!ctx || !d_in || step_count < 0) return APOLLO_ERR_INVALID_ARG;
+    // what the checkpoint does not hold starts at zero: the rows that pad the rank on the tensor path, the pitch padding
+    if (cudaMemsetAsync(ctx->ws + ctx->plan.zero_begin, 0, ctx->plan.zero_end - ctx->plan.zero_begin,
+                        static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return APOLLO_ERR_CUDA;
     const int rc = state_copy(ctx, const_cast<char*>(static_cast<const char*>(d_in)), false,
                               static_cast<cudaStream_t>(cuda_stream));
     if (rc != APOLLO_OK) return rc;

@@ -9,7 +9,7 @@ namespace apollo {
 enum Path : int32_t {
     PATH_STREAM = 0,  // rank 1: streaming matrix-vector pass, moments updated by the finalize kernel
     PATH_SIMT = 1,    // any rank, any dtype, any pitch: CUDA-core tiles
-    PATH_TENSOR = 2,  // bf16, rank a multiple of 16, 16-byte row pitch: TMA + tcgen05 + TMEM
+    PATH_TENSOR = 2,  // bf16, rank >= 16 (worked on rounded up to a multiple of 16): TMA + tcgen05 + TMEM
 };
 
 constexpr int STREAM_ROWS = 512;     // rows of a wide matrix one streaming tile covers
@@ -117,6 +117,8 @@ struct StepParams {
     uint32_t key0, key1;   // Philox key = seed
     uint32_t epoch;        // floor(t / T)
     int32_t rank, mode;
+    int32_t rank_pad;         // tensor path: rank rounded up to the MMA's granularity (16; 32 above 256); the rows of P
+                              // from `rank` on are zero, and M and V are laid out with rank_pad rows
     float inv_sqrt_r;
     float lr, wd, alpha, gamma;
     float beta1, beta2, eps;

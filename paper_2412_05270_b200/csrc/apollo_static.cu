@@ -148,7 +148,7 @@ extern "C" int apollo_mini_step_static(void* d_W, const void* d_G, int64_t rows,
     fill_round_keys(sp);
     sp.state_bf16 = 0;
     sp.epoch = (uint32_t)(t / cfg->T);
-    sp.rank = 1; sp.mode = cfg->mode;
+    sp.rank = 1; sp.rank_pad = 1; sp.mode = cfg->mode;
     sp.inv_sqrt_r = 1.0f;
     sp.lr = lr; sp.wd = wd; sp.alpha = cfg->alpha; sp.gamma = cfg->gamma;
     sp.beta1 = cfg->beta1; sp.beta2 = cfg->beta2; sp.eps = cfg->eps;

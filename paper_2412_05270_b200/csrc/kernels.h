@@ -27,8 +27,11 @@ void launch_update(int dtype, const MatDesc* d_descs, const int* d_prefix, int n
 // Copies a moment between the library's layout (state_at(): row-major with pitch ns, or channel blocks of
 // 128) and dense r x n rows; lib_esz / dense_esz are 2 (bfloat16) or 4 (fp32), a bfloat16 source is
 // widened when the destination is fp32.  to_dense = false copies dense -> library (same element size).
-void launch_state_copy(void* d_lib, void* d_dense, int rank, int n, int ns, bool tiled, int lib_esz, int dense_esz,
-                       bool to_dense, cudaStream_t stream);
+// rank_layout: rows the library's layout was planned with (the padded rank on the tensor path); `rank` rows are copied.
+void launch_state_copy(void* d_lib, void* d_dense, int rank, int rank_layout, int n, int ns, bool tiled, int lib_esz,
+                       int dense_esz, bool to_dense, cudaStream_t stream);
+// The rank the tensor path works with: `rank` rounded up to a multiple of 16 (32 above 256).
+int tensor_path_padded_rank(int rank);
 
 // Tensor-core projection (TMA + tcgen05 + TMEM).
 bool tensor_path_supports(int rows, int cols, int rank, int dtype);

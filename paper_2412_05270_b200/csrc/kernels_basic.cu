@@ -640,13 +640,13 @@ update_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix,
     }
 }
 
-__global__ void state_copy_kernel(void* __restrict__ lib, void* __restrict__ dense, int rank, int n, int ns, bool tiled,
-                                  int lib_esz, int dense_esz, bool to_dense)
+__global__ void state_copy_kernel(void* __restrict__ lib, void* __restrict__ dense, int rank, int rank_layout, int n, int ns,
+                                  bool tiled, int lib_esz, int dense_esz, bool to_dense)
 {
     const int64_t count = (int64_t)rank * n;
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x) {
         const int k = (int)(i / n), j = (int)(i - (int64_t)k * n);
-        const int64_t at = state_at(tiled, ns, rank, k, j);
+        const int64_t at = state_at(tiled, ns, rank_layout, k, j);
         if (to_dense) {
             if (lib_esz == 4) static_cast<float*>(dense)[i] = static_cast<const float*>(lib)[at];
             else if (dense_esz == 4) static_cast<float*>(dense)[i] = bf16_bits_to_float((uint32_t)static_cast<const unsigned short*>(lib)[at]);
@@ -658,12 +658,12 @@ __global__ void state_copy_kernel(void* __restrict__ lib, void* __restrict__ den
     }
 }
 
-void launch_state_copy(void* d_lib, void* d_dense, int rank, int n, int ns, bool tiled, int lib_esz, int dense_esz,
-                       bool to_dense, cudaStream_t stream)
+void launch_state_copy(void* d_lib, void* d_dense, int rank, int rank_layout, int n, int ns, bool tiled, int lib_esz,
+                       int dense_esz, bool to_dense, cudaStream_t stream)
 {
     const int64_t count = (int64_t)rank * n;
     if (count == 0) return;
-    state_copy_kernel<<<blocks_for(count), 256, 0, stream>>>(d_lib, d_dense, rank, n, ns, tiled, lib_esz, dense_esz, to_dense);
+    state_copy_kernel<<<blocks_for(count), 256, 0, stream>>>(d_lib, d_dense, rank, rank_layout, n, ns, tiled, lib_esz, dense_esz, to_dense);
 }
 
 // ----------------------------------------------------------------------------------------

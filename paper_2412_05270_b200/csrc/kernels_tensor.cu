@@ -126,11 +126,16 @@ int tensor_path_configure(int rank, uint32_t flags, const apollo_tuning* tuning,
     return APOLLO_OK;
 }
 
+int tensor_path_padded_rank(int rank)
+{
+    return rank <= 256 ? (rank + 15) / 16 * 16 : (rank + 31) / 32 * 32;
+}
+
 bool tensor_path_supports(int rows, int cols, int rank, int dtype)
 {
     if (dtype != APOLLO_DT_BF16) return false;
-    if (rank < 16 || rank > 512 || rank % 16) return false;
-    if (rank > 256 && rank % 32) return false;
+    // any rank from 16 on: the MMA works on the rank rounded up to its granularity, with zero rows of P
+    if (rank < 16 || rank > 512) return false;
     (void)rows; (void)cols;   // a row pitch that is not a multiple of 16 bytes goes through a padded copy
     return true;
 }
@@ -296,6 +301,7 @@ __device__ __forceinline__ uint4 p_vector(const float* __restrict__ ext_p, int m
                                           const StepParams& sp)
 {
     uint4 v;
+    if (row >= sp.rank) return make_uint4(0u, 0u, 0u, 0u);      // padding rows of a rank that is not a multiple of 16
     if (ext_p) {
         float z[8];
 #pragma unroll
@@ -536,6 +542,9 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                     va.z = pack_bf16x2(a1.x, a1.y); va.w = pack_bf16x2(a1.z, a1.w);
                     vb.x = pack_bf16x2(b0.x, b0.y); vb.y = pack_bf16x2(b0.z, b0.w);
                     vb.z = pack_bf16x2(b1.x, b1.y); vb.w = pack_bf16x2(b1.z, b1.w);
+                    // padding rows of a rank that is not a multiple of 16
+                    if (ka >= (uint32_t)sp.rank) va = make_uint4(0u, 0u, 0u, 0u);
+                    if (kbrow >= (uint32_t)sp.rank) vb = make_uint4(0u, 0u, 0u, 0u);
                     const uint32_t at = p_s + row * 128 + ((chunk ^ (row & 7)) << 4);
                     st_shared_v4(at, va);
                     if (c + TC_GEN_THREADS < total) st_shared_v4(at + 32 * 128, vb);   // row + 32: same swizzle phase
@@ -613,10 +622,10 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
                 float rv[16];
                 ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * r_slice + cchunk * 16), rv);
                 const int j = j0 + b * 128 + ch_in_blk;
-                if (j < n && APOLLO_DBG_RANGE(state_at(true, 0, sp.rank, r0 + cchunk * 16, j),
-                                              state_at(true, 0, sp.rank, r0 + cchunk * 16 + 15, j),
-                                              state_elements(n, sp.rank, true), status)) {
-                    const int64_t at = state_at(true, 0, sp.rank, r0 + cchunk * 16, j);     // channel blocks of 128: rows are 128 elements apart
+                if (j < n && APOLLO_DBG_RANGE(state_at(true, 0, sp.rank_pad, r0 + cchunk * 16, j),
+                                              state_at(true, 0, sp.rank_pad, r0 + cchunk * 16 + 15, j),
+                                              state_elements(n, sp.rank_pad, true), status)) {
+                    const int64_t at = state_at(true, 0, sp.rank_pad, r0 + cchunk * 16, j);     // channel blocks of 128: rows are 128 elements apart
                     const bool sb = sp.state_bf16 != 0;
                     float mv[16], vv[16];
 #pragma unroll
@@ -794,7 +803,7 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             }
             if (!ok) break;
             const MatDesc* gp = descs + gm;
-            const int vec_per_row = __ldg(&gp->m_pad) / 8, total = sp.rank * vec_per_row;
+            const int vec_per_row = __ldg(&gp->m_pad) / 8, total = sp.rank_pad * vec_per_row;
             const int per = (total + GEN_CHUNKS - 1) / GEN_CHUNKS;
             const int c_end = min(total, (piece + 1) * per);
             const uint32_t matrix_id = (uint32_t)__ldg(&gp->matrix_id);
@@ -1124,7 +1133,7 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             // as many bytes of the moments are in flight per SM.  The first chunk is asked for before the
             // wait for the accumulator.
             // M and V are stored in channel blocks of 128 (state_at): this CTA's block, rows 128 elements apart
-            const int64_t tile_el = (int64_t)(j0 >> 7) * sp.rank * 128;
+            const int64_t tile_el = (int64_t)(j0 >> 7) * sp.rank_pad * 128;
             const bool pf = tl.epi_prefetch != 0 && j0 + q * 32 < n;
             const char* const pf_base = reinterpret_cast<const char*>(lane < 16 ? Mbase : Vbase);
             const int64_t pf_esz = sp.state_bf16 != 0 ? 2 : 4;
@@ -1147,7 +1156,7 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                 ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + buf * (uint32_t)r_slice + (uint32_t)(cchunk * 16), rv);
                 if (j < n && APOLLO_DBG_RANGE(tile_el + (int64_t)(r0 + cchunk * 16) * 128 + ch,
                                               tile_el + (int64_t)(r0 + cchunk * 16 + 15) * 128 + ch,
-                                              state_elements(n, sp.rank, true), status)) {
+                                              state_elements(n, sp.rank_pad, true), status)) {
                     const int64_t at = tile_el + (int64_t)(r0 + cchunk * 16) * 128 + ch;
                     const bool sb = sp.state_bf16 != 0;
                     float mv[16], vv[16];
@@ -1212,7 +1221,7 @@ __global__ void generate_p_kernel(const MatDesc* __restrict__ descs, int mat_beg
     const uint32_t matrix_id = (uint32_t)__ldg(&dp->matrix_id);
     uint4* out = static_cast<uint4*>(dp->pstage);
     const int chunks_per_row = m_pad / 8;
-    const int total = sp.rank * chunks_per_row;
+    const int total = sp.rank_pad * chunks_per_row;
     const float* __restrict__ ext_p = dp->ext_p;
     const int m = __ldg(&dp->m);
     for (int c = blockIdx.x * blockDim.x + threadIdx.x; c < total; c += gridDim.x * blockDim.x) {

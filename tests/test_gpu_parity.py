@@ -72,6 +72,10 @@ def test_streaming_path_spanning_row_blocks_and_column_tiles():
     (64, [(264, 1029), (200, 1000), (200, 1001), (204, 333), (1000, 203)]),
     (256, [(512, 1381), (512, 1376), (256, 257)]),
     (512, [(512, 1381), (1376, 512), (512, 515)]),  # two row slices per channel tile
+    # ranks that are not multiples of 16: the MMA works on the rank rounded up, with zero rows of P
+    (17, [(64, 72), (72, 64), (17, 520)]),
+    (130, [(300, 1032), (1032, 304), (130, 130)]),
+    (300, [(512, 1376), (1376, 512)]),              # above 256: rounded up to 320, two row slices of 160
 ])
 def test_tensor_core_path(rank, shapes):
     wl = _wl(shapes, rank, dtype="bf16", steps=4, T=2, wd=0.01)
@@ -208,7 +212,8 @@ def test_misaligned_and_null_pointers_are_rejected_before_any_launch():
     opt.close()
 
 
-@pytest.mark.parametrize("rank,mode,flags", [(32, "channel", 0), (1, "tensor", 0), (5, "channel", B.FLAG_NO_TENSOR_CORES)])
+@pytest.mark.parametrize("rank,mode,flags", [(32, "channel", 0), (1, "tensor", 0), (5, "channel", B.FLAG_NO_TENSOR_CORES),
+                                             (40, "channel", 0)])      # 40: kept with 48 rows on the tensor path
 def test_checkpoint_and_resume_continue_bit_for_bit(rank, mode, flags):
     wl = _wl([(200, 336), (336, 200), (64, 64)], rank, mode=mode, dtype="bf16", T=2, steps=6, wd=0.01)
     dev = torch.device("cuda")
@@ -243,13 +248,14 @@ def test_checkpoint_and_resume_continue_bit_for_bit(rank, mode, flags):
         fresh.state_export()                       # nothing has run yet
 
 
+@pytest.mark.parametrize("rank", [32, 40])
 @pytest.mark.parametrize("flags", [0, B.FLAG_BF16_STATES])
-def test_checkpoint_is_dense_whatever_layout_the_kernels_keep(flags):
+def test_checkpoint_is_dense_whatever_layout_the_kernels_keep(flags, rank):
     """The tensor path keeps its moments in channel blocks, the CUDA-core path row by row with a padded
     pitch; the checkpoint and apollo_get_state are dense in both, so a state written by one is read by
     the other, entry for entry."""
     shapes = [(200, 336), (336, 203), (64, 64), (128, 520)]     # n = 336, 336, 64, 520: ragged last blocks
-    wl = _wl(shapes, 32, dtype="bf16", T=2, steps=3, wd=0.01)
+    wl = _wl(shapes, rank, dtype="bf16", T=2, steps=3, wd=0.01)
     dev = torch.device("cuda")
     tensor = B.Apollo(wl.shapes, B.config_for(wl, flags))
     assert all(tensor.path(i) == B.PATH_TENSOR for i in range(len(shapes)))
