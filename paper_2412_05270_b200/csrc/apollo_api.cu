@@ -29,7 +29,7 @@ struct NvtxRange {
 };
 
 struct MatPlan {
-    int32_t rows, cols, m, n, tall, path, slices, g2_slices, tiles_n, tiles_k, raw;
+    int32_t rows, cols, m, n, tall, path, slices, g2_slices, tiles_n, tiles_k, raw, split, g_pitch;
     int64_t proj_tiles, update_tiles;
     size_t off_M, off_V, off_scal, off_s, off_part, off_g2, off_tmap, off_pstage, off_gpad, gpad_bytes;
 };
@@ -80,6 +80,8 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
         plan.tc_rank = tensor_path_padded_rank(cfg->rank);
         rc = tensor_path_configure(plan.tc_rank, cfg->flags, tuning, &plan.tc);
         if (rc != APOLLO_OK) return rc;
+        // fp32 gradients reach the tensor cores as bfloat16 high and low parts (pair kernel with a P scratch)
+        plan.tc.split = cfg->dtype == APOLLO_DT_F32 && plan.tc.pair && plan.tc.staged ? 1 : 0;
     }
     plan.mats.resize(n_mat);
     for (int t = 0; t < 4; ++t) plan.tiles[t] = 0;
@@ -105,10 +107,11 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
                 p.tiles_k = 1;
                 p.slices = 1;
             }
-        } else if (tensor_path_supports(p.rows, p.cols, r, cfg->dtype) && !(cfg->flags & APOLLO_FLAG_NO_TENSOR_CORES)) {
+        } else if (tensor_path_supports(p.rows, p.cols, r, cfg->dtype, plan.tc) && !(cfg->flags & APOLLO_FLAG_NO_TENSOR_CORES)) {
             p.path = PATH_TENSOR;
             // rows that start on no 16-byte boundary: re-aligned in shared memory where the pair kernel can, else a padded copy
-            p.raw = tensor_path_raw_ok(p.rows, p.cols, plan.tc) ? 1 : 0;
+            p.split = plan.tc.split;
+            p.raw = !p.split && tensor_path_raw_ok(p.rows, p.cols, plan.tc) ? 1 : 0;
             if (p.raw) tensor_path_enable_raw(&plan.tc);
             tensor_path_tiling(p.rows, p.cols, plan.tc_rank, plan.tc, &p.tiles_n, &p.tiles_k, &p.slices, &p.g2_slices);
         } else {
@@ -150,7 +153,7 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
     if (plan.tc.gen && !plan.tensor_mats.empty()) {
         size_t slot = 0;
         for (int i : plan.tensor_mats) {
-            const size_t need = align_up(tensor_path_stage_bytes(plan.mats[i].rows, plan.mats[i].cols, plan.tc_rank));
+            const size_t need = align_up(tensor_path_stage_bytes(plan.mats[i].rows, plan.mats[i].cols, plan.tc_rank, plan.mats[i].split != 0));
             if (need > slot) slot = need;
         }
         int64_t slots = plan.tc.scratch_bytes / (int64_t)slot;
@@ -169,7 +172,7 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
         for (int i = 0; i < n_mat; ++i) {
             MatPlan& p = plan.mats[i];
             const bool tensor = p.path == PATH_TENSOR;
-            const size_t need = tensor && plan.tc.staged ? align_up(tensor_path_stage_bytes(p.rows, p.cols, plan.tc_rank)) : 0;
+            const size_t need = tensor && plan.tc.staged ? align_up(tensor_path_stage_bytes(p.rows, p.cols, plan.tc_rank, p.split != 0)) : 0;
             if (used > 0 && (used >= budget || need > budget - used)) {
                 g.mat_end = i; g.tile_end = tile_at;
                 plan.groups.push_back(g);
@@ -197,8 +200,15 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
         for (int i = 0; i < n_mat; ++i) {
             MatPlan& p = plan.mats[i];
             p.gpad_bytes = 0;
-            if (p.path == PATH_TENSOR && (p.cols % 8) != 0 && !p.raw) {
-                p.gpad_bytes = align_up((size_t)p.rows * (size_t)((p.cols + 7) / 8 * 8) * 2);
+            p.g_pitch = p.cols;
+            if (p.path == PATH_TENSOR && p.split) {
+                int pitch = 0;
+                p.gpad_bytes = align_up(tensor_path_split_bytes(p.rows, p.cols, &pitch));
+                p.g_pitch = pitch;
+                plan.any_repitch = true;
+            } else if (p.path == PATH_TENSOR && (p.cols % 8) != 0 && !p.raw) {
+                p.g_pitch = (p.cols + 7) / 8 * 8;
+                p.gpad_bytes = align_up((size_t)p.rows * (size_t)p.g_pitch * 2);
                 plan.any_repitch = true;
             }
             if (used > 0 && p.gpad_bytes > 0 && (used >= budget || p.gpad_bytes > budget - used)) {
@@ -376,8 +386,10 @@ int apollo_create_tuned(apollo_ctx** out_ctx, const apollo_shape* shapes, int32_
         d.pstage = ctx->ws + ctx->plan.off_stage + p.off_pstage;
         d.m_pad = (p.m + 63) / 64 * 64;
         d.gpad = p.gpad_bytes ? ctx->ws + p.off_gpad : nullptr;
-        d.g_pitch = p.gpad_bytes ? (p.cols + 7) / 8 * 8 : p.cols;
+        d.g_pitch = p.g_pitch;
         d.raw = p.raw;
+        d.split = p.split;
+        d.p_width = (p.split ? 2 : 1) * d.m_pad;
         d.upd_super = update_super_rows(p.rows, p.cols, p.tall != 0) ? 1 : 0;
         if (p.cols % 8 == 0 || d.upd_super) {
             const UpdateTiling ut = update_tiling(d.upd_super ? 8 * p.cols : p.cols);
@@ -583,7 +595,8 @@ static int step_range(apollo_ctx* ctx, int first, int count, void* const* d_W, c
             bool any = false;
             for (int i = ra; i < rb; ++i) any |= ctx->h_descs[i].gpad != nullptr;
             if (any) {
-                launch_repitch(ctx->d_descs, ra, rb - ra, stream);
+                if (plan.tc.split) launch_split(ctx->d_descs, ra, rb - ra, stream);
+                else launch_repitch(ctx->d_descs, ra, rb - ra, stream);
                 ++launches;
             }
         }

@@ -106,6 +106,10 @@ struct MatDesc {
     int32_t tiles_k;  // projection tiles along the other tiled axis (rows of G, or rows of R)
     int32_t m_pad;    // m rounded up to 64: row length of the staged P
     int32_t g_pitch;  // row pitch (elements) of the array the tensor path reads: cols, or cols rounded up to 8
+    int32_t split;    // 1: fp32 gradient on the tensor path: `gpad` holds its bfloat16 high and low parts ([hi; lo] along the
+                      //    projected side, m_pad apart), the P slot holds [P_hi | P_lo], and a tile's contraction runs over
+                      //    three segments (P_hi G_hi, P_lo G_hi, P_hi G_lo)
+    int32_t p_width;  // elements per row of the P slot: m_pad, or 2 m_pad for a split matrix
     int32_t raw;      // 1: wide matrix with cols % 8 != 0 and rows % 8 == 0 on the pair kernel: its G tiles are fetched
                       //    as they lie in memory and re-aligned in shared memory (no padded copy)
     int32_t upd_chunks, upd_width, upd_groups;   // 2-D tiling of the update pass (update_tiling(cols)); 0 chunks: flat tiles
@@ -147,6 +151,7 @@ struct TcTiling {
     int32_t keep;      // 1: every matrix owns a slot of the scratch, filled once per epoch (APOLLO_FLAG_KEEP_P)
     int32_t gen;       // 1: spare warps of the pair kernel generate P into a ring of `slots` slots, ahead of its use
     int32_t slots;     // gen: slots of the ring (matrix with tensor ordinal q uses slot q % slots)
+    int32_t split;     // 1: the gradients are fp32 and go through the bfloat16 high/low split (MatDesc::split)
     int32_t raw_allowed; // tuning: matrices that qualify are re-aligned in shared memory rather than copied to a padded pitch
     int32_t raw;       // 1: the list has matrices whose G tiles are re-aligned in shared memory (MatDesc::raw): the
                        //    G part of a stage is RAW_G_BYTES and the norm warps arrive on the stage's `full` barrier

@@ -34,7 +34,7 @@ void launch_state_copy(void* d_lib, void* d_dense, int rank, int rank_layout, in
 int tensor_path_padded_rank(int rank);
 
 // Tensor-core projection (TMA + tcgen05 + TMEM).
-bool tensor_path_supports(int rows, int cols, int rank, int dtype);
+bool tensor_path_supports(int rows, int cols, int rank, int dtype, const TcTiling& tl);
 // The tiling and mode for a rank, the context's flags and the caller's tuning (may be null):
 // APOLLO_OK, or APOLLO_ERR_INVALID_ARG for a tuning value out of range.
 int tensor_path_configure(int rank, uint32_t flags, const apollo_tuning* tuning, TcTiling* out);
@@ -45,7 +45,11 @@ void tensor_path_enable_raw(TcTiling* tl);
 void tensor_path_tiling(int rows, int cols, int rank, const TcTiling& tl, int32_t* tiles_n, int32_t* tiles_k,
                         int32_t* slices, int32_t* g2_slices);
 // Bytes one matrix's P needs in the scratch (rank x round_up(m, 64) bf16).
-size_t tensor_path_stage_bytes(int rows, int cols, int rank);
+size_t tensor_path_stage_bytes(int rows, int cols, int rank, bool split);
+// Bytes of the bfloat16 high/low copy of an fp32 gradient, and its row pitch in elements.
+size_t tensor_path_split_bytes(int rows, int cols, int* pitch);
+// Writes those copies for matrices [first, first + count) and the squared column norms of the gradients.
+void launch_split(const MatDesc* d_descs, int first, int count, cudaStream_t stream);
 // Encodes the tensor maps of the matrices on the tensor path (G at +0, staged P at +128 of
 // each 256-byte slot) into h_maps (2 x n_mat maps of 128 bytes, host).  Returns an APOLLO_* code.
 int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, const TcTiling& tl, void* h_maps);

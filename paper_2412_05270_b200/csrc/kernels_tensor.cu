@@ -70,10 +70,22 @@ EncodeTiledFn encode_fn()
 }  // namespace
 
 // Bytes one matrix's P takes in the scratch: rank rows of round_up(m, 64) bfloat16 standard normals.
-size_t tensor_path_stage_bytes(int rows, int cols, int rank)
+// A split matrix (fp32 gradient) keeps the high and the low bfloat16 part of every normal: twice the width.
+size_t tensor_path_stage_bytes(int rows, int cols, int rank, bool split)
 {
     const int m = rows > cols ? cols : rows;
-    return (size_t)rank * (size_t)((m + 63) / 64 * 64) * 2;
+    return (size_t)rank * (size_t)((m + 63) / 64 * 64) * 2 * (split ? 2 : 1);
+}
+
+// The bfloat16 high/low copy of an fp32 gradient: [hi; lo] along the projected side, each part m_pad =
+// round_up(m, 64) long (zero beyond m).  Wide: 2 m_pad rows of round_up(cols, 8) elements; tall: rows of 2 m_pad.
+size_t tensor_path_split_bytes(int rows, int cols, int* pitch)
+{
+    const bool tall = rows > cols;
+    const int m_pad = ((tall ? cols : rows) + 63) / 64 * 64;
+    const int p = tall ? 2 * m_pad : (cols + 7) / 8 * 8;
+    if (pitch) *pitch = p;
+    return (size_t)(tall ? rows : 2 * m_pad) * (size_t)p * 2;
 }
 
 int tensor_path_configure(int rank, uint32_t flags, const apollo_tuning* tuning, TcTiling* out)
@@ -131,9 +143,10 @@ int tensor_path_padded_rank(int rank)
     return rank <= 256 ? (rank + 15) / 16 * 16 : (rank + 31) / 32 * 32;
 }
 
-bool tensor_path_supports(int rows, int cols, int rank, int dtype)
+bool tensor_path_supports(int rows, int cols, int rank, int dtype, const TcTiling& tl)
 {
-    if (dtype != APOLLO_DT_BF16) return false;
+    // fp32 gradients go through a bfloat16 high/low split that only the pair kernel with a P scratch reads
+    if (dtype != APOLLO_DT_BF16 && !(tl.pair && tl.staged)) return false;
     // any rank from 16 on: the MMA works on the rank rounded up to its granularity, with zero rows of P
     if (rank < 16 || rank > 512) return false;
     (void)rows; (void)cols;   // a row pitch that is not a multiple of 16 bytes goes through a padded copy
@@ -180,7 +193,9 @@ int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, const TcTiling& t
         const MatDesc& d = h_descs[i];
         if (d.path != PATH_TENSOR) continue;
         // dimension 0 is the contiguous one (the stored columns)
-        const cuuint64_t dims[2] = { (cuuint64_t)d.cols, (cuuint64_t)d.rows };
+        // (a split matrix is read from its high/low copy: the projected side is 2 m_pad long there)
+        const cuuint64_t dims[2] = { (cuuint64_t)(d.split && d.tall ? 2 * d.m_pad : d.cols),
+                                     (cuuint64_t)(d.split && !d.tall ? 2 * d.m_pad : d.rows) };
         const cuuint64_t strides[1] = { (cuuint64_t)d.g_pitch * 2 };
         // wide: 64 channels x 64 rows of G; tall: 64 contraction elements x 128 channels
         const cuuint32_t box[2] = { 64u, d.tall ? 128u : 64u };
@@ -207,8 +222,8 @@ int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, const TcTiling& t
         if (rc != CUDA_SUCCESS) return APOLLO_ERR_CUDA;
         if (tl.staged) {
             // staged P: rank rows of m_pad bf16, loaded as 64 x r_slice boxes (K-major UMMA tiles)
-            const cuuint64_t pdims[2] = { (cuuint64_t)d.m_pad, (cuuint64_t)rank };
-            const cuuint64_t pstrides[1] = { (cuuint64_t)d.m_pad * 2 };
+            const cuuint64_t pdims[2] = { (cuuint64_t)d.p_width, (cuuint64_t)rank };
+            const cuuint64_t pstrides[1] = { (cuuint64_t)d.p_width * 2 };
             const cuuint32_t pbox[2] = { 64u, (cuuint32_t)(tl.pair ? tl.r_slice / 2 : tl.r_slice) };
             const CUresult rp = encode(&maps[2 * i + 1], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, d.pstage, pdims, pstrides,
                                        pbox, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -297,11 +312,34 @@ __device__ __forceinline__ bool wait_counter(const uint32_t* counter, uint32_t t
 
 // Eight standard normals of row `row`, columns 8 ch .. 8 ch + 7 of a matrix's P as bfloat16 (one 16-byte
 // store of the scratch), from the generator or from a projection supplied by the caller.
+// SPLIT (fp32 gradients): a row of the slot is [P_hi | P_lo], each half_vpr vectors long: the normals in fp32
+// (the precise transform), their bfloat16 rounding and the bfloat16 rounding of what the first rounding left.
+template <bool SPLIT>
 __device__ __forceinline__ uint4 p_vector(const float* __restrict__ ext_p, int m, int row, int ch, uint32_t matrix_id,
-                                          const StepParams& sp)
+                                          const StepParams& sp, int half_vpr = 0)
 {
     uint4 v;
     if (row >= sp.rank) return make_uint4(0u, 0u, 0u, 0u);      // padding rows of a rank that is not a multiple of 16
+    if (SPLIT) {
+        const bool low = ch >= half_vpr;
+        const int c = low ? ch - half_vpr : ch;
+        float z[8];
+        if (ext_p) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) z[e] = 8 * c + e < m ? __ldg(ext_p + (int64_t)row * m + 8 * c + e) : 0.f;
+        } else {
+            const float4 a0 = normal_quad((uint32_t)(2 * c), (uint32_t)row, matrix_id, sp.epoch, sp.key0, sp.key1);
+            const float4 a1 = normal_quad((uint32_t)(2 * c + 1), (uint32_t)row, matrix_id, sp.epoch, sp.key0, sp.key1);
+            z[0] = a0.x; z[1] = a0.y; z[2] = a0.z; z[3] = a0.w; z[4] = a1.x; z[5] = a1.y; z[6] = a1.z; z[7] = a1.w;
+        }
+        if (low) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) z[e] -= round_to_bf16(z[e]);
+        }
+        v.x = pack_bf16x2(z[0], z[1]); v.y = pack_bf16x2(z[2], z[3]);
+        v.z = pack_bf16x2(z[4], z[5]); v.w = pack_bf16x2(z[6], z[7]);
+        return v;
+    }
     if (ext_p) {
         float z[8];
 #pragma unroll
@@ -717,7 +755,11 @@ static_assert(P2_MISC_BYTES == 1536, "tensor_path_configure() reserves this many
 // RAW: the list has matrices whose G tiles are re-aligned in shared memory (TcTiling::raw).  The kernel without
 // that code is a separate instantiation, so that lists without such matrices run exactly the code they ran
 // before it existed (with it compiled in, the other roles of the kernel came out 15 % slower).
-template <bool RAW>
+// SPLIT: the gradients are fp32 (TcTiling::split).  A tile's contraction then runs over three segments of the
+// bfloat16 high/low copies, P_hi G_hi + P_lo G_hi + P_hi G_lo (what is dropped, P_lo G_lo, is 2^-16 of a
+// term), and the column norms come from the kernel that made the copies.  A third instantiation, for the
+// same reason as the second.
+template <bool RAW, bool SPLIT>
 __global__ void __launch_bounds__(P2_THREADS, 1)
 project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix, int n_mat, int tile_begin,
                     int tile_end, StepParams sp, TcTiling tl, GenArgs gen, int32_t* __restrict__ status)
@@ -803,7 +845,8 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             }
             if (!ok) break;
             const MatDesc* gp = descs + gm;
-            const int vec_per_row = __ldg(&gp->m_pad) / 8, total = sp.rank_pad * vec_per_row;
+            const int half_vpr = __ldg(&gp->m_pad) / 8;
+            const int vec_per_row = SPLIT ? 2 * half_vpr : half_vpr, total = sp.rank_pad * vec_per_row;
             const int per = (total + GEN_CHUNKS - 1) / GEN_CHUNKS;
             const int c_end = min(total, (piece + 1) * per);
             const uint32_t matrix_id = (uint32_t)__ldg(&gp->matrix_id);
@@ -814,10 +857,10 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             for (int c = piece * per + lane; c < c_end; c += 64) {
                 if (!APOLLO_DBG_RANGE(c, c, total, status)) break;
                 const int row0 = c / vec_per_row;
-                const uint4 v0 = p_vector(ext_p, gmm, row0, c - row0 * vec_per_row, matrix_id, sp);
+                const uint4 v0 = p_vector<SPLIT>(ext_p, gmm, row0, c - row0 * vec_per_row, matrix_id, sp, half_vpr);
                 if (c + 32 < c_end) {
                     const int row1 = (c + 32) / vec_per_row;
-                    out[c + 32] = p_vector(ext_p, gmm, row1, c + 32 - row1 * vec_per_row, matrix_id, sp);
+                    out[c + 32] = p_vector<SPLIT>(ext_p, gmm, row1, c + 32 - row1 * vec_per_row, matrix_id, sp, half_vpr);
                 }
                 out[c] = v0;
             }
@@ -841,7 +884,13 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
         const int local = tile - __ldg(prefix + mat);
         const int tr = local % tiles_k, tn = local / tiles_k;
         const int j0 = tn * 256 + (int)rank * 128, r0 = tr * r_slice;
-        const int num_kb = (m + TC_BK - 1) / TC_BK;
+        const int nkb1 = (m + TC_BK - 1) / TC_BK;
+        const int num_kb = SPLIT ? 3 * nkb1 : nkb1;
+        // SPLIT: where k-block kb starts along the projected side of the G copy ([hi; lo], m_pad apart) and of the
+        // P slot ([P_hi | P_lo]): segments hi x hi, lo x hi, hi x lo (P x G)
+        const int m_pad_s = SPLIT ? __ldg(&dp->m_pad) : 0;
+        auto g_at = [&](int kb) { return SPLIT ? (kb >= 2 * nkb1 ? m_pad_s + (kb - 2 * nkb1) * TC_BK : (kb >= nkb1 ? kb - nkb1 : kb) * TC_BK) : kb * TC_BK; };
+        auto p_at = [&](int kb) { return SPLIT ? (kb >= 2 * nkb1 ? (kb - 2 * nkb1) * TC_BK : (kb >= nkb1 ? m_pad_s + (kb - nkb1) * TC_BK : kb * TC_BK)) : kb * TC_BK; };
         const uint32_t buf = tile_iter & 1, use = tile_iter >> 1;
         // this matrix's rows start on no 16-byte boundary: its tiles are fetched as they lie and re-aligned by the norm warps
         const bool raw_tile = RAW && __ldg(&dp->raw) != 0;
@@ -880,10 +929,10 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                     }
                     if (rank == 0) ptx::mbar_arrive_expect_tx(bar_full + 8 * s, 2u * (P2_G_BYTES + p_bytes));   // G and P of both CTAs
                     if (tall) {
-                        ptx::tma_load_2d_pair(g_s, tmap, kb * TC_BK, j0, full, pol_g);
+                        ptx::tma_load_2d_pair(g_s, tmap, g_at(kb), j0, full, pol_g);
                     } else {
-                        ptx::tma_load_2d_pair(g_s, tmap, j0, kb * TC_BK, full, pol_g);
-                        ptx::tma_load_2d_pair(g_s + P2_G_BYTES / 2, tmap, j0 + 64, kb * TC_BK, full, pol_g);
+                        ptx::tma_load_2d_pair(g_s, tmap, j0, g_at(kb), full, pol_g);
+                        ptx::tma_load_2d_pair(g_s + P2_G_BYTES / 2, tmap, j0 + 64, g_at(kb), full, pol_g);
                     }
                 }
             }
@@ -912,7 +961,7 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                     // free a stage before this thread has even filled it, and the MMA's own commit is the signal.
                     if (RAW ? !wait_phase(bar_done + 8 * s, phase ^ 1, abort_flag, status, 103)
                             : !wait_phase(bar_empty + 8 * s, phase ^ 1, abort_flag, status, 104)) break;
-                    ptx::tma_load_2d_pair(smem_base + s * stage_bytes + g_bytes, tmap_p, kb * TC_BK, p_row, full0 + 8 * s, pol_p);
+                    ptx::tma_load_2d_pair(smem_base + s * stage_bytes + g_bytes, tmap_p, p_at(kb), p_row, full0 + 8 * s, pol_p);
                 }
             }
             __syncwarp();
@@ -1042,8 +1091,9 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                     continue;
                 }
                 if (!__all_sync(0xFFFFFFFFu, wait_phase(bar_done + 8 * s, ph, abort_flag, status, 110))) break;   // landed, and the MMA has read it
-                if (tr != 0) {
+                if (tr != 0 || SPLIT) {
                     // the norms belong to the channel tile, not to the row slice: the first slice has them
+                    // (and those of an fp32 gradient come from the kernel that split it)
                 } else if (tall) {
                     // units (row, half): 256 units over 128 threads; the order of the chunks is free
 #pragma unroll
@@ -1088,7 +1138,7 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                     x0 += __shfl_xor_sync(0xFFFFFFFFu, x0, 8);  x1 += __shfl_xor_sync(0xFFFFFFFFu, x1, 8);
                     x0 += __shfl_xor_sync(0xFFFFFFFFu, x0, 16); x1 += __shfl_xor_sync(0xFFFFFFFFu, x1, 16);
                     const int j = j0 + (i >> 2) * 64 + (lane & 7) * 8 + 2 * (i & 3);
-                    if (!stop && tr == 0 && lane < 8) {
+                    if (!stop && !SPLIT && tr == 0 && lane < 8) {
                         float* const out = g2out + (int64_t)(warp - 4) * n;
                         if (j < n && APOLLO_DBG_RANGE((int64_t)(warp - 4) * n + j, (int64_t)(warp - 4) * n + j, (int64_t)__ldg(&dp->g2_slices) * n, status)) out[j] = x0;
                         if (j + 1 < n && APOLLO_DBG_RANGE((int64_t)(warp - 4) * n + j + 1, (int64_t)(warp - 4) * n + j + 1, (int64_t)__ldg(&dp->g2_slices) * n, status)) out[j + 1] = x1;
@@ -1102,7 +1152,7 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                                        (ptx::f32x2_sum(acc2[4 * pass + 2]) + ptx::f32x2_sum(acc2[4 * pass + 3]));
                     const float v = mine + __shfl_xor_sync(0xFFFFFFFFu, mine, 1);
                     const int j = j0 + ((t + pass * 128) >> 1);
-                    if (!stop && tr == 0 && !(lane & 1) && j < n &&
+                    if (!stop && !SPLIT && tr == 0 && !(lane & 1) && j < n &&
                         APOLLO_DBG_RANGE(j, j, (int64_t)__ldg(&dp->g2_slices) * n, status))
                         g2out[j] = v;
                 }
@@ -1115,7 +1165,7 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                 for (int e = 0; e < 8; ++e) {
                     const float v = acc[e] + __shfl_xor_sync(0xFFFFFFFFu, acc[e], 16);
                     const int j = j0 + cc * 8 + e;
-                    if (!stop && tr == 0 && lane < 16 && j < n &&
+                    if (!stop && !SPLIT && tr == 0 && lane < 16 && j < n &&
                         APOLLO_DBG_RANGE((int64_t)(warp - 4) * n + j, (int64_t)(warp - 4) * n + j, (int64_t)__ldg(&dp->g2_slices) * n, status))
                         g2out[(int64_t)(warp - 4) * n + j] = v;
                 }
@@ -1220,13 +1270,15 @@ __global__ void generate_p_kernel(const MatDesc* __restrict__ descs, int mat_beg
     const int m_pad = __ldg(&dp->m_pad);
     const uint32_t matrix_id = (uint32_t)__ldg(&dp->matrix_id);
     uint4* out = static_cast<uint4*>(dp->pstage);
-    const int chunks_per_row = m_pad / 8;
+    const bool split = __ldg(&dp->split) != 0;
+    const int chunks_per_row = (split ? 2 : 1) * (m_pad / 8);
     const int total = sp.rank_pad * chunks_per_row;
     const float* __restrict__ ext_p = dp->ext_p;
     const int m = __ldg(&dp->m);
     for (int c = blockIdx.x * blockDim.x + threadIdx.x; c < total; c += gridDim.x * blockDim.x) {
         const int row = c / chunks_per_row, ch = c - row * chunks_per_row;
-        out[c] = p_vector(ext_p, m, row, ch, matrix_id, sp);
+        out[c] = split ? p_vector<true>(ext_p, m, row, ch, matrix_id, sp, m_pad / 8)
+                       : p_vector<false>(ext_p, m, row, ch, matrix_id, sp);
     }
 }
 
@@ -1297,6 +1349,61 @@ __global__ void repitch_kernel(const MatDesc* __restrict__ descs, int first)
     }
 }
 
+// fp32 gradient -> its bfloat16 high and low parts, [hi; lo] along the projected side, each part m_pad long
+// (zero beyond m), for the three-segment contraction of the pair kernel; and the squared column norms of the
+// gradient in fp32, which the tiles of the two parts cannot give (the cross term is missing there).
+//   wide: a thread owns a column of one of four row slabs (coalesced over the 256 columns of a block); one
+//         slice of norms per slab, summed by finalize_kernel.  tall: a warp owns a stored row (= channel).
+__global__ void __launch_bounds__(256) split_kernel(const MatDesc* __restrict__ descs, int first)
+{
+    const MatDesc* dp = descs + first + blockIdx.y;
+    if (__ldg(&dp->split) == 0) return;
+    const float* __restrict__ G = static_cast<const float*>(dp->G);
+    __nv_bfloat16* __restrict__ out = static_cast<__nv_bfloat16*>(dp->gpad);
+    float* __restrict__ g2 = dp->g2;
+    const int rows = __ldg(&dp->rows), cols = __ldg(&dp->cols), n = __ldg(&dp->n);
+    const int m_pad = __ldg(&dp->m_pad);
+    const int64_t pitch = __ldg(&dp->g_pitch);
+    if (__ldg(&dp->tall) == 0) {
+        const int ctiles = (cols + 255) / 256, rows_per = m_pad / 4;
+        for (int u = blockIdx.x; u < 4 * ctiles; u += gridDim.x) {
+            const int ct = u % ctiles, slab = u / ctiles, j = ct * 256 + (int)threadIdx.x;
+            if (j >= cols) continue;
+            float acc = 0.f;
+            for (int i = slab * rows_per; i < (slab + 1) * rows_per; ++i) {
+                const float g = i < rows ? __ldg(G + (int64_t)i * cols + j) : 0.f;
+                const __nv_bfloat16 hi = __float2bfloat16_rn(g);
+                out[(int64_t)i * pitch + j] = hi;
+                out[(int64_t)(m_pad + i) * pitch + j] = __float2bfloat16_rn(g - __bfloat162float(hi));
+                acc = fmaf(g, g, acc);
+            }
+            g2[(int64_t)slab * n + j] = acc;
+        }
+    } else {
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        for (int row = blockIdx.x * 8 + warp; row < rows; row += gridDim.x * 8) {
+            float acc = 0.f;
+            for (int c = lane; c < m_pad; c += 32) {
+                const float g = c < cols ? __ldg(G + (int64_t)row * cols + c) : 0.f;
+                const __nv_bfloat16 hi = __float2bfloat16_rn(g);
+                out[(int64_t)row * pitch + c] = hi;
+                out[(int64_t)row * pitch + m_pad + c] = __float2bfloat16_rn(g - __bfloat162float(hi));
+                acc = fmaf(g, g, acc);
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
+            if (lane == 0) g2[row] = acc;
+        }
+    }
+}
+
+void launch_split(const MatDesc* d_descs, int first, int count, cudaStream_t stream)
+{
+    if (count <= 0) return;
+    const dim3 grid(592, (unsigned)count);
+    split_kernel<<<grid, 256, 0, stream>>>(d_descs, first);
+}
+
 void launch_repitch(const MatDesc* d_descs, int first, int count, cudaStream_t stream)
 {
     if (count <= 0) return;
@@ -1346,8 +1453,9 @@ void launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_ma
     // the shared-memory opt-in is a per-device attribute of the kernels: set once per context
     if (!state.attr_set) {
         cudaFuncSetAttribute(project_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
-        cudaFuncSetAttribute(project_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
-        cudaFuncSetAttribute(project_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
+        cudaFuncSetAttribute(project_pair_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
+        cudaFuncSetAttribute(project_pair_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
+        cudaFuncSetAttribute(project_pair_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
         state.attr_set = true;
     }
     if (tl.pair) {
@@ -1365,8 +1473,9 @@ void launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_ma
         // (a pair sits in one GPC, so this can be fewer than half the SMs)
         if (state.max_pairs == 0) {
             int clusters = 0;
-            const cudaError_t oe = tl.raw ? cudaOccupancyMaxActiveClusters(&clusters, project_pair_kernel<true>, &cfg)
-                                          : cudaOccupancyMaxActiveClusters(&clusters, project_pair_kernel<false>, &cfg);
+            const cudaError_t oe = tl.split ? cudaOccupancyMaxActiveClusters(&clusters, project_pair_kernel<false, true>, &cfg)
+                                   : tl.raw ? cudaOccupancyMaxActiveClusters(&clusters, project_pair_kernel<true, false>, &cfg)
+                                            : cudaOccupancyMaxActiveClusters(&clusters, project_pair_kernel<false, false>, &cfg);
             if (oe != cudaSuccess || clusters < 1) {
                 cudaGetLastError();
                 clusters = sm_count / 2;
@@ -1376,10 +1485,12 @@ void launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_ma
         int pairs = state.max_pairs;
         if (tiles < pairs) pairs = tiles;
         cfg.gridDim = dim3(2 * pairs);
-        if (tl.raw)
-            cudaLaunchKernelEx(&cfg, project_pair_kernel<true>, d_descs, d_prefix, n_mat, tile_begin, tile_end, sp, tl, gen, d_status);
+        if (tl.split)
+            cudaLaunchKernelEx(&cfg, project_pair_kernel<false, true>, d_descs, d_prefix, n_mat, tile_begin, tile_end, sp, tl, gen, d_status);
+        else if (tl.raw)
+            cudaLaunchKernelEx(&cfg, project_pair_kernel<true, false>, d_descs, d_prefix, n_mat, tile_begin, tile_end, sp, tl, gen, d_status);
         else
-            cudaLaunchKernelEx(&cfg, project_pair_kernel<false>, d_descs, d_prefix, n_mat, tile_begin, tile_end, sp, tl, gen, d_status);
+            cudaLaunchKernelEx(&cfg, project_pair_kernel<false, false>, d_descs, d_prefix, n_mat, tile_begin, tile_end, sp, tl, gen, d_status);
         return;
     }
     const int grid = tiles < sm_count ? tiles : sm_count;

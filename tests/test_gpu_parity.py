@@ -156,7 +156,28 @@ def test_limiter_engages_on_growing_gradients():
 
 
 def test_config_single_matrix_fp32_rank128():
-    run_parity(WL.workload("single"))
+    """fp32 gradients run on the tensor cores too, as bfloat16 high and low parts (three contraction segments);
+    the oracle's P and G are not rounded."""
+    worst = run_parity(WL.workload("single"), expect_path=B.PATH_TENSOR)
+    assert worst["dw"] <= 1.0 and worst["exempt"] == 0.0
+    run_parity(WL.workload("single"), flags=B.FLAG_NO_TENSOR_CORES, expect_path=B.PATH_SIMT)
+
+
+@pytest.mark.parametrize("rank,shapes", [
+    (16, [(64, 72), (72, 64), (128, 128), (16, 520)]),
+    (64, [(200, 1000), (1000, 200), (520, 264), (200, 333), (336, 203)]),   # ragged tiles, odd pitches
+    (130, [(300, 1032), (1032, 304)]),                                      # rank padded to 144
+    (512, [(512, 1376), (1376, 512)]),
+])
+def test_tensor_core_path_fp32_gradients(rank, shapes):
+    wl = _wl(shapes, rank, dtype="f32", steps=4, T=2, wd=0.01)
+    worst = run_parity(wl, expect_path=B.PATH_TENSOR)
+    assert worst["exempt"] == 0.0
+    run_parity(wl, flags=B.FLAG_KEEP_P, expect_path=B.PATH_TENSOR, tuning=B.make_tuning(repitch_mb=1))
+    # the ring kernel does not read the split copies: fp32 gradients stay on the CUDA cores there
+    opt = B.Apollo(wl.shapes, B.config_for(wl), tuning=B.make_tuning(kernel=B.TC_KERNEL_RING))
+    assert opt.path(0) == B.PATH_SIMT
+    opt.close()
 
 
 def test_config_llama60m_mini_all_matrices():
