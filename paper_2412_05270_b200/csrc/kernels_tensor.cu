@@ -319,7 +319,9 @@ __device__ __forceinline__ uint4 p_vector(const float* __restrict__ ext_p, int m
                                           const StepParams& sp, int half_vpr = 0)
 {
     uint4 v;
-    if (row >= sp.rank) return make_uint4(0u, 0u, 0u, 0u);      // padding rows of a rank that is not a multiple of 16
+    // rows from `rank` on pad a rank that is not a multiple of 16: zero (selected at the end, without a branch, so that
+    // the Philox chains of two calls still interleave)
+    const bool pad_row = row >= sp.rank;
     if (SPLIT) {
         const bool low = ch >= half_vpr;
         const int c = low ? ch - half_vpr : ch;
@@ -338,7 +340,7 @@ __device__ __forceinline__ uint4 p_vector(const float* __restrict__ ext_p, int m
         }
         v.x = pack_bf16x2(z[0], z[1]); v.y = pack_bf16x2(z[2], z[3]);
         v.z = pack_bf16x2(z[4], z[5]); v.w = pack_bf16x2(z[6], z[7]);
-        return v;
+        return pad_row ? make_uint4(0u, 0u, 0u, 0u) : v;
     }
     if (ext_p) {
         float z[8];
@@ -346,13 +348,13 @@ __device__ __forceinline__ uint4 p_vector(const float* __restrict__ ext_p, int m
         for (int e = 0; e < 8; ++e) z[e] = 8 * ch + e < m ? __ldg(ext_p + (int64_t)row * m + 8 * ch + e) : 0.f;
         v.x = pack_bf16x2(z[0], z[1]); v.y = pack_bf16x2(z[2], z[3]);
         v.z = pack_bf16x2(z[4], z[5]); v.w = pack_bf16x2(z[6], z[7]);
-        return v;
+        return pad_row ? make_uint4(0u, 0u, 0u, 0u) : v;
     }
     const float4 a0 = normal_quad_fast((uint32_t)(2 * ch), (uint32_t)row, matrix_id, sp.epoch, sp.round_key);
     const float4 a1 = normal_quad_fast((uint32_t)(2 * ch + 1), (uint32_t)row, matrix_id, sp.epoch, sp.round_key);
     v.x = pack_bf16x2(a0.x, a0.y); v.y = pack_bf16x2(a0.z, a0.w);
     v.z = pack_bf16x2(a1.x, a1.y); v.w = pack_bf16x2(a1.z, a1.w);
-    return v;
+    return pad_row ? make_uint4(0u, 0u, 0u, 0u) : v;
 }
 
 __device__ __forceinline__ float sum_sq_bf16x8(const uint4& v)
