@@ -107,7 +107,9 @@ typedef struct {
     int32_t p_generator;   /* with APOLLO_P_SCRATCH and without APOLLO_FLAG_KEEP_P: 0 = spare warps of the pair
                               kernel generate the projections a few matrices ahead of their use (default);
                               1 = a separate kernel fills the scratch group by group between projection launches */
-    int32_t scratch_mb;    /* size of the P scratch in MB; 0 = default (32) */
+    int32_t scratch_mb;    /* most the P scratch may take, in MB; 0 = default (128).  A list whose projections all
+                              fit is regenerated into it by one launch of the generator kernel per step; a larger
+                              list goes through a ring of at most 32 MB of it (see p_generator) */
     int32_t r_slice;       /* rows of R per tile: a multiple of 16, <= 256, that divides the rank rounded up to a
                               multiple of 16 (32 above 256); 0 = default */
     int32_t nblk;          /* ring kernel: 128-channel blocks per tile (1, 2 or 4; nblk * r_slice <= 512); 0 = default */
@@ -126,8 +128,8 @@ typedef struct {
 /*
  * Bytes of DEVICE workspace a context over `shapes[0..n_matrices)` needs: moments, scales,
  * partial sums, descriptor tables, tensor maps, and for the tensor-core path a scratch for the
- * random projections.  By default that scratch holds a few matrices' projections (32 MB) and
- * is refilled from the seed in every step (Algorithm 1 "P_t <- N_seed(0, 1/r)": only the seed is
+ * random projections.  By default that scratch holds a few matrices' projections (32 MB; all of
+ * them when they fit in 128 MB) and is refilled from the seed in every step (Algorithm 1 "P_t <- N_seed(0, 1/r)": only the seed is
  * kept).  With APOLLO_FLAG_KEEP_P every matrix has its own r x m slot, filled in the step that
  * opens an epoch (every T steps, Algorithm 1 "if t mod T = 0") and read again by the following
  * steps of the epoch; the steps of such a context must reach the GPU in order, whatever streams

@@ -150,13 +150,23 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
     // Otherwise staging groups: consecutive matrices whose P fit the scratch together, filled group by group.
     plan.groups.clear();
     plan.stage_bytes = 0;
+    if (plan.tc.gen) {
+        // A list whose projections all fit the scratch is served better by the separate generator kernel, once
+        // per step and with the whole chip (44 M normals of the 350M list: 40 us), than by the spare warps of
+        // the pair kernel, which then sit on the critical path (such lists have few tiles per matrix).
+        size_t all = 0;
+        for (int i : plan.tensor_mats)
+            all += align_up(tensor_path_stage_bytes(plan.mats[i].rows, plan.mats[i].cols, plan.tc_rank, plan.mats[i].split != 0));
+        if (all <= (size_t)plan.tc.scratch_bytes) plan.tc.gen = 0;
+    }
     if (plan.tc.gen && !plan.tensor_mats.empty()) {
         size_t slot = 0;
         for (int i : plan.tensor_mats) {
             const size_t need = align_up(tensor_path_stage_bytes(plan.mats[i].rows, plan.mats[i].cols, plan.tc_rank, plan.mats[i].split != 0));
             if (need > slot) slot = need;
         }
-        int64_t slots = plan.tc.scratch_bytes / (int64_t)slot;
+        const int64_t ring_bytes = plan.tc.scratch_bytes < ((int64_t)32 << 20) ? plan.tc.scratch_bytes : ((int64_t)32 << 20);
+        int64_t slots = ring_bytes / (int64_t)slot;      // a deeper ring gains nothing (32, 64 and 256 MB measured equal)
         if (slots < 2) slots = 2;
         if (slots > (int64_t)plan.tensor_mats.size()) slots = (int64_t)plan.tensor_mats.size();
         plan.tc.slots = (int32_t)slots;

@@ -112,7 +112,7 @@ int tensor_path_configure(int rank, uint32_t flags, const apollo_tuning* tuning,
     }
     t.staged = tu.p_source == APOLLO_P_SCRATCH ? 1 : 0;
     t.keep = t.staged && (flags & APOLLO_FLAG_KEEP_P) ? 1 : 0;
-    t.scratch_bytes = (int64_t)(tu.scratch_mb ? tu.scratch_mb : 32) << 20;
+    t.scratch_bytes = (int64_t)(tu.scratch_mb ? tu.scratch_mb : 128) << 20;
     t.repitch_bytes = (int64_t)tu.repitch_mb << 20;      // 0: no limit, every matrix has its own copy (one projection launch)
     t.epi_prefetch = tu.epi_prefetch ? tu.epi_prefetch - 1 : 1;
     t.raw_allowed = tu.realign == 1 ? 1 : 0;      // default: padded copy (the faster of the two as measured)

@@ -39,16 +39,19 @@ def test_strerror_names_every_code():
 
 
 def test_tuning_is_validated_and_sizes_the_p_scratch():
-    shapes = [(4096, 4096)] * 40
+    shapes = [(4096, 4096)] * 100
     cfg = B.make_config(rank=256, dtype=B.DT_BF16)
-    moments = 40 * 2 * 256 * 4096 * 4
+    moments = 100 * 2 * 256 * 4096 * 4
     per_step = B.workspace_bytes(shapes, cfg)
     kept = B.workspace_bytes(shapes, B.make_config(rank=256, dtype=B.DT_BF16, flags=B.FLAG_KEEP_P))
     p_bytes = 256 * 4096 * 2
-    # default: a 32 MB scratch (16 slots of 2 MB); kept: one slot per matrix
-    assert per_step - moments < 48 << 20       # scratch + scales, partial sums, tables
-    assert kept - per_step == (40 - 16) * p_bytes
+    # 200 MB of projections do not fit the 128 MB scratch: a ring of 32 MB (16 slots of 2 MB); kept: one slot per matrix
+    assert per_step - moments < 56 << 20       # ring + scales, partial sums, tables
+    assert kept - per_step == (100 - 16) * p_bytes
     assert B.workspace_bytes(shapes, cfg, B.make_tuning(scratch_mb=8)) == per_step - (16 - 4) * p_bytes
+    # 80 MB of projections fit: all of them are regenerated into the scratch by the generator kernel every step
+    few = [(4096, 4096)] * 40
+    assert B.workspace_bytes(few, B.make_config(rank=256, dtype=B.DT_BF16, flags=B.FLAG_KEEP_P)) == B.workspace_bytes(few, cfg)
     for bad in (dict(kernel=2), dict(p_source=3), dict(r_slice=24), dict(r_slice=512), dict(nblk=3),
                 dict(nblk=4, r_slice=256), dict(scratch_mb=-1), dict(epi_prefetch=9), dict(p_generator=2), dict(realign=3), dict(repitch_mb=-1)):
         with pytest.raises(B.ApolloError) as err:
