@@ -34,7 +34,7 @@ struct MatPlan {
     size_t off_M, off_V, off_scal, off_s, off_part, off_g2, off_tmap, off_pstage, off_gpad, gpad_bytes;
 };
 
-struct StageGroup {   // matrices whose staged P share one filling of the staging buffer
+struct StageGroup {   // matrices whose P share one filling of the P scratch by generate_p_kernel
     int mat_begin, mat_end, tile_begin, tile_end;
 };
 
@@ -277,7 +277,7 @@ struct apollo_ctx {
     int32_t n_mat;
     Plan plan;
     TcLaunchState tc_state;
-    std::vector<char> h_maps;        // 2 x n_mat tensor maps of 128 bytes (G, staged P)
+    std::vector<char> h_maps;        // 2 x n_mat tensor maps of 128 bytes (G, the matrix's P slot)
     UploadSlot upload[2];
     int upload_next;
     std::vector<MatDesc> h_descs;

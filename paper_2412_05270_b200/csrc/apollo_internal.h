@@ -89,8 +89,8 @@ struct MatDesc {
     float* scal;      // {norm after limiting, c, norm before limiting, tensor-wise s}
     float* prev;      // previous limited norm (one float)
     const void* tmap; // 128-byte TMA tensor map of G in device memory (tensor path only)
-    const void* tmap_p; // tensor map of the staged P (tensor path with L2 staging)
-    void* pstage;     // this matrix's r x m_pad bf16 standard normals in the staging buffer
+    const void* tmap_p; // tensor map of this matrix's slot of the P scratch
+    void* pstage;     // this matrix's slot of the P scratch: rank_pad x p_width bf16 standard normals
     const float* ext_p; // caller-supplied projection (r x m fp32, row-major) used instead of the generator, or nullptr
     void* gpad;       // copy of G with a 16-byte row pitch when cols % 8 != 0 (tensor path), else nullptr
     int32_t rows, cols;
@@ -104,7 +104,7 @@ struct MatDesc {
     int32_t matrix_id;
     int32_t tiles_n;  // projection tiles along the channels
     int32_t tiles_k;  // projection tiles along the other tiled axis (rows of G, or rows of R)
-    int32_t m_pad;    // m rounded up to 64: row length of the staged P
+    int32_t m_pad;    // m rounded up to 64: row length of P in its slot (twice that for a split matrix)
     int32_t g_pitch;  // row pitch (elements) of the array the tensor path reads: cols, or cols rounded up to 8
     int32_t split;    // 1: fp32 gradient on the tensor path: `gpad` holds its bfloat16 high and low parts ([hi; lo] along the
                       //    projected side, m_pad apart), the P slot holds [P_hi | P_lo], and a tile's contraction runs over

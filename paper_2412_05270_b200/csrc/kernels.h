@@ -50,14 +50,14 @@ size_t tensor_path_stage_bytes(int rows, int cols, int rank, bool split);
 size_t tensor_path_split_bytes(int rows, int cols, int* pitch);
 // Writes those copies for matrices [first, first + count) and the squared column norms of the gradients.
 void launch_split(const MatDesc* d_descs, int first, int count, cudaStream_t stream);
-// Encodes the tensor maps of the matrices on the tensor path (G at +0, staged P at +128 of
+// Encodes the tensor maps of the matrices on the tensor path (G at +0, the P slot at +128 of
 // each 256-byte slot) into h_maps (2 x n_mat maps of 128 bytes, host).  Returns an APOLLO_* code.
 int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, const TcTiling& tl, void* h_maps);
 // Copies the gradients whose row pitch is not a multiple of 16 bytes into their padded buffers.
 void launch_repitch(const MatDesc* d_descs, int first, int count, cudaStream_t stream);
-// Fills the staging buffer with the standard normals of matrices [mat_begin, mat_end).
 // Test hook: a bounded wait that is left to run out (sets STATUS_TIMEOUT in *d_status).
 void launch_bounded_wait_selftest(int32_t* d_status, cudaStream_t stream);
+// Fills the P slots of matrices [mat_begin, mat_end) with their standard normals (generate_p_kernel).
 void launch_generate_p(const MatDesc* d_descs, int mat_begin, int mat_end, const StepParams& sp, cudaStream_t stream);
 // Projection over tiles [tile_begin, tile_end) of the tensor-path prefix table.
 void launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_mat, int tile_begin, int tile_end,

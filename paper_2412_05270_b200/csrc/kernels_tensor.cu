@@ -9,9 +9,9 @@
 // above its definition) and project_tensor_kernel, the single-CTA ring kernel described here.
 //
 // Roles of the 14 warps of a ring-kernel CTA (one CTA per SM, persistent over tiles of 256 channels):
-//   warp 0      TMA producer: G tiles (and staged P tiles) into a shared-memory ring, 128-byte swizzle
+//   warp 0      TMA producer: G tiles (and P tiles from the scratch) into a shared-memory ring, 128-byte swizzle
 //   warp 1      MMA issuer (one thread) and owner of the 512 TMEM columns
-//   warps 2-9   staged P: L2 prefetch of the G lines the producer will ask for next;
+//   warps 2-9   P from the scratch: L2 prefetch of the G lines the producer will ask for next;
 //               otherwise generators: Philox -> Box-Muller -> bf16 P tile in the UMMA K-major layout
 //   warps 10-13 column norms of G from the landed tiles
 //   warps 2-13  epilogue: tcgen05.ld of R, read-modify-write of M and V, partial sums
@@ -221,7 +221,7 @@ int tensor_path_prepare(MatDesc* h_descs, int n_mat, int rank, const TcTiling& t
         }
         if (rc != CUDA_SUCCESS) return APOLLO_ERR_CUDA;
         if (tl.staged) {
-            // staged P: rank rows of m_pad bf16, loaded as 64 x r_slice boxes (K-major UMMA tiles)
+            // the P slot: rank rows of p_width bf16, loaded as 64 x r_slice boxes (K-major UMMA tiles)
             const cuuint64_t pdims[2] = { (cuuint64_t)d.p_width, (cuuint64_t)rank };
             const cuuint64_t pstrides[1] = { (cuuint64_t)d.p_width * 2 };
             const cuuint32_t pbox[2] = { 64u, (cuuint32_t)(tl.pair ? tl.r_slice / 2 : tl.r_slice) };
@@ -517,7 +517,7 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
             // ---------------- generators: P tile for every k-block ----------------
             const int g = tid - 64;
             if (staged) {
-                // P arrives by TMA from the staging buffer.  These warps instead ask L2 for the lines of G
+                // P arrives by TMA from the scratch.  These warps instead ask L2 for the lines of G
                 // TC_PREFETCH k-blocks ahead of the producer (into the next tile at the end of this one), so
                 // that the loads into the shared-memory ring find them there.
                 struct Ahead { const char* base; size_t pitch; int m, n, j0, nkb; bool tall; };
@@ -732,7 +732,7 @@ project_tensor_kernel(const MatDesc* __restrict__ descs, const int* __restrict__
 }
 
 // ----------------------------------------------------------------------------------------
-// Pair kernel (default for staged P): two CTAs of a cluster share every MMA (cta_group::2,
+// Pair kernel (default): two CTAs of a cluster share every MMA (cta_group::2,
 // M = 256).  A pair tile is 256 channels x r_slice rows of R.  Each CTA loads the G tile of its own
 // 128 channels and half of the rows of the P tile (so a k-block costs 32 KB of shared-memory fill per
 // CTA instead of 48 KB for the same work), and keeps r_slice accumulator columns per buffer, double
@@ -1264,7 +1264,7 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
     if (warp == 1) ptx::tmem_dealloc_pair(tmem_base, 512);
 }
 
-// Standard normals of the staged P: one 16-byte store (8 bf16) per thread and pass.
+// Standard normals of the matrices' P slots: one 16-byte store (8 bf16) per thread and pass.
 __global__ void generate_p_kernel(const MatDesc* __restrict__ descs, int mat_begin, StepParams sp)
 {
     const MatDesc* dp = descs + mat_begin + blockIdx.y;
