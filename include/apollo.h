@@ -104,9 +104,11 @@ typedef struct {
 typedef struct {
     int32_t kernel;        /* APOLLO_TC_KERNEL_* */
     int32_t p_source;      /* APOLLO_P_* */
-    int32_t p_generator;   /* with APOLLO_P_SCRATCH and without APOLLO_FLAG_KEEP_P: 0 = spare warps of the pair
-                              kernel generate the projections a few matrices ahead of their use (default);
-                              1 = a separate kernel fills the scratch group by group between projection launches */
+    int32_t p_generator;   /* with APOLLO_P_SCRATCH and without APOLLO_FLAG_KEEP_P: 0 = default: a list whose projections
+                              all fit the scratch is refilled by one launch of the generator kernel per step, a
+                              larger one by spare warps of the pair kernel, a few matrices ahead of their use,
+                              through a ring of slots; 1 = always the generator kernel, group by group between
+                              projection launches; 2 = always the spare warps */
     int32_t scratch_mb;    /* most the P scratch may take, in MB; 0 = default (128).  A list whose projections all
                               fit is regenerated into it by one launch of the generator kernel per step; a larger
                               list goes through a ring of at most 32 MB of it (see p_generator) */

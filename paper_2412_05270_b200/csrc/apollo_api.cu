@@ -157,7 +157,7 @@ int make_plan(const apollo_shape* shapes, int32_t n_mat, const apollo_config* cf
         size_t all = 0;
         for (int i : plan.tensor_mats)
             all += align_up(tensor_path_stage_bytes(plan.mats[i].rows, plan.mats[i].cols, plan.tc_rank, plan.mats[i].split != 0));
-        if (all <= (size_t)plan.tc.scratch_bytes) plan.tc.gen = 0;
+        if (plan.tc.gen == 1 && all <= (size_t)plan.tc.scratch_bytes) plan.tc.gen = 0;
     }
     if (plan.tc.gen && !plan.tensor_mats.empty()) {
         size_t slot = 0;

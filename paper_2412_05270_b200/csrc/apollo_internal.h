@@ -149,7 +149,7 @@ struct TcTiling {
     int32_t pair;      // 1: the pair kernel (CTA pairs, cta_group::2); staged only
     int32_t epi_prefetch; // pair kernel: the epilogue warps ask L2 for the moments this many chunks ahead of their loads
     int32_t keep;      // 1: every matrix owns a slot of the scratch, filled once per epoch (APOLLO_FLAG_KEEP_P)
-    int32_t gen;       // 1: spare warps of the pair kernel generate P into a ring of `slots` slots, ahead of its use
+    int32_t gen;       // != 0: spare warps of the pair kernel generate P into a ring of `slots` slots, ahead of its use
     int32_t slots;     // gen: slots of the ring (matrix with tensor ordinal q uses slot q % slots)
     int32_t split;     // 1: the gradients are fp32 and go through the bfloat16 high/low split (MatDesc::split)
     int32_t raw_allowed; // tuning: matrices that qualify are re-aligned in shared memory rather than copied to a padded pitch

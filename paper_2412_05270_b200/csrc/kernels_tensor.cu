@@ -95,7 +95,7 @@ int tensor_path_configure(int rank, uint32_t flags, const apollo_tuning* tuning,
     TcTiling t = {};
     if (tu.kernel != APOLLO_TC_KERNEL_PAIR && tu.kernel != APOLLO_TC_KERNEL_RING) return APOLLO_ERR_INVALID_ARG;
     if (tu.p_source != APOLLO_P_SCRATCH && tu.p_source != APOLLO_P_SHARED) return APOLLO_ERR_INVALID_ARG;
-    if (tu.p_generator != 0 && tu.p_generator != 1) return APOLLO_ERR_INVALID_ARG;
+    if (tu.p_generator < 0 || tu.p_generator > 2) return APOLLO_ERR_INVALID_ARG;
     if (tu.scratch_mb < 0 || tu.scratch_mb > 65536 || tu.realign < 0 || tu.realign > 2) return APOLLO_ERR_INVALID_ARG;
     if (tu.repitch_mb < 0 || tu.repitch_mb > 65536) return APOLLO_ERR_INVALID_ARG;
     if (tu.epi_prefetch < 0 || tu.epi_prefetch > 9) return APOLLO_ERR_INVALID_ARG;
@@ -122,7 +122,7 @@ int tensor_path_configure(int rank, uint32_t flags, const apollo_tuning* tuning,
         // pair tile: 256 channels (128 per CTA) x r_slice rows, accumulator double buffered
         t.pair = 1;
         t.nblk = 2;
-        t.gen = !t.keep && tu.p_generator == 0 ? 1 : 0;
+        t.gen = !t.keep && tu.p_generator != 1 ? (tu.p_generator == 2 ? 2 : 1) : 0;      // 2: also for lists that would fit the scratch
         const int stage = 128 * TC_BK * 2 + (t.r_slice / 2) * 128;
         t.stages = (TC_MAX_SMEM - 1536) / stage;
         if (t.stages > 8) t.stages = 8;

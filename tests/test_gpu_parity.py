@@ -300,14 +300,21 @@ def test_checkpoint_is_dense_whatever_layout_the_kernels_keep(flags, rank):
         assert torch.equal(Ma, Mb) and torch.equal(Va, Vb)
 
 
-@pytest.mark.parametrize("rank,mode,flags", [(32, "channel", 0), (1, "tensor", 0), (5, "channel", B.FLAG_NO_TENSOR_CORES)])
-def test_layer_wise_range_steps_equal_the_whole_list_step(rank, mode, flags):
+@pytest.mark.parametrize("rank,mode,flags,tuning", [
+    (32, "channel", 0, {}), (1, "tensor", 0, {}), (5, "channel", B.FLAG_NO_TENSOR_CORES, {}),
+    # P generated by the pair kernel's spare warps through a ring of two slots: a range starts in the middle of the ring
+    (256, "channel", 0, {"p_generator": 2, "scratch_mb": 1}),
+])
+def test_layer_wise_range_steps_equal_the_whole_list_step(rank, mode, flags, tuning):
     shapes = [(200, 336), (336, 200), (64, 64), (128, 520), (96, 203), (72, 64), (64, 72)]
+    if rank == 256:
+        shapes = [(512, 1376), (1376, 512), (512, 512), (300, 1032), (1376, 1400), (520, 264), (264, 520)]
     wl = _wl(shapes, rank, mode=mode, dtype="bf16", T=2, steps=4, wd=0.01)
     dev = torch.device("cuda")
     cfg = B.config_for(wl, flags)
     n = len(shapes)
-    whole, ranged = B.Apollo(wl.shapes, cfg), B.Apollo(wl.shapes, cfg)
+    whole = B.Apollo(wl.shapes, cfg, tuning=B.make_tuning(**tuning))
+    ranged = B.Apollo(wl.shapes, cfg, tuning=B.make_tuning(**tuning))
     Wa = [WL.make_weight(wl, i).to(dev) for i in range(n)]
     Wb = [w.clone() for w in Wa]
     layers = [(4, 7), (2, 4), (0, 2)]          # visited in backward order
@@ -326,11 +333,14 @@ def test_layer_wise_range_steps_equal_the_whole_list_step(rank, mode, flags):
         ranged.step_range(5, Wb[5:8] + [Wb[0]], G[5:8] + [G[0]], wl.lr)     # runs past the end of the list
 
 
-@pytest.mark.parametrize("rank,dtype,flags,path", [
-    (16, "bf16", 0, B.PATH_TENSOR), (4, "f32", 0, B.PATH_SIMT), (6, "bf16", B.FLAG_NO_TENSOR_CORES, B.PATH_SIMT),
-    (1, "bf16", 0, B.PATH_STREAM),
+@pytest.mark.parametrize("rank,dtype,flags,path,tuning", [
+    (16, "bf16", 0, B.PATH_TENSOR, {}), (4, "f32", 0, B.PATH_SIMT, {}), (6, "bf16", B.FLAG_NO_TENSOR_CORES, B.PATH_SIMT, {}),
+    (1, "bf16", 0, B.PATH_STREAM, {}),
+    (16, "bf16", 0, B.PATH_TENSOR, {"p_generator": 2}),      # converted by the pair kernel's spare warps
+    (16, "bf16", B.FLAG_KEEP_P, B.PATH_TENSOR, {}),
+    (24, "f32", 0, B.PATH_TENSOR, {}),                       # fp32 gradients: the supplied P is split into high and low parts
 ])
-def test_caller_supplied_projection_from_an_svd(rank, dtype, flags, path):
+def test_caller_supplied_projection_from_an_svd(rank, dtype, flags, path, tuning):
     """The "APOLLO w. SVD" variant: P = top-r left singular vectors of the first gradient (computed here
     with torch on the CPU), handed to the library and to the oracle alike."""
     import numpy as np
@@ -340,7 +350,7 @@ def test_caller_supplied_projection_from_an_svd(rank, dtype, flags, path):
     wl = _wl(shapes, rank, mode="tensor" if rank == 1 else "channel", dtype=dtype, T=100, steps=3, wd=0.01,
              alpha=1.0)
     dev = torch.device("cuda")
-    opt = B.Apollo(wl.shapes, B.config_for(wl, flags))
+    opt = B.Apollo(wl.shapes, B.config_for(wl, flags), tuning=B.make_tuning(**tuning))
     Ps, orc = [], []
     for i, (rows, cols) in enumerate(shapes):
         assert opt.path(i) == path

@@ -53,7 +53,7 @@ def test_tuning_is_validated_and_sizes_the_p_scratch():
     few = [(4096, 4096)] * 40
     assert B.workspace_bytes(few, B.make_config(rank=256, dtype=B.DT_BF16, flags=B.FLAG_KEEP_P)) == B.workspace_bytes(few, cfg)
     for bad in (dict(kernel=2), dict(p_source=3), dict(r_slice=24), dict(r_slice=512), dict(nblk=3),
-                dict(nblk=4, r_slice=256), dict(scratch_mb=-1), dict(epi_prefetch=9), dict(p_generator=2), dict(realign=3), dict(repitch_mb=-1)):
+                dict(nblk=4, r_slice=256), dict(scratch_mb=-1), dict(epi_prefetch=9), dict(p_generator=3), dict(realign=3), dict(repitch_mb=-1)):
         with pytest.raises(B.ApolloError) as err:
             B.workspace_bytes(shapes, cfg, B.make_tuning(**bad))
         assert err.value.code == B.ERR_INVALID_ARG, bad
