@@ -213,23 +213,41 @@ def run_reference(args, wl, rank, world):
     print(json.dumps(line), flush=True)
 
 
+RANGE_SIZE = 0      # --range-size: step the list in ranges of this many matrices (apollo_step_range), 0 = apollo_step
+
+
+def one_step(opt, Ws, Gs, wl):
+    """One optimizer step: apollo_step over the whole list, or range by range (projection, finalize and update of
+    a few matrices back to back, as a layer-wise update during the backward pass would issue them)."""
+    if RANGE_SIZE <= 0:
+        opt.step(Ws, Gs, wl.lr, wl.wd, check=False)
+        return opt.last_launches()
+    n, launches = len(Ws), 0
+    for a in range(0, n, RANGE_SIZE):
+        b = min(a + RANGE_SIZE, n)
+        opt.step_range(a, Ws[a:b], Gs[a:b], wl.lr, wl.wd, close_step=(b == n))
+        launches += opt.last_launches()
+    return launches
+
+
 def time_steps(opt, Ws, Gs, wl, steps, warmup, stream, barrier, clocks):
     """`warmup` untimed steps, then `steps` timed ones between two CUDA events on `stream`.  Returns the
     total milliseconds, the kernel launches inside the timed region, the per-phase means and the clocks
     sampled during the region."""
     for _ in range(warmup):
-        opt.step(Ws, Gs, wl.lr, wl.wd, check=False)
+        one_step(opt, Ws, Gs, wl)
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     t0 = time.monotonic()
     start.record(stream)
     launches = 0
     for _ in range(steps):
-        opt.step(Ws, Gs, wl.lr, wl.wd, check=False)
-        launches += opt.last_launches()
+        launches += one_step(opt, Ws, Gs, wl)
     stop.record(stream)
     barrier()
     t1 = time.monotonic()
+    if RANGE_SIZE > 0:          # the per-phase events are recorded by whole-list steps only
+        return start.elapsed_time(stop), launches, {"projection": 0.0, "finalize": 0.0, "update": 1e-9}, clocks.summary(t0, t1)
     phases = [opt.timing(k) for k in range(min(steps, 64))]
     phase_ms = {name: sum(p[k] for p in phases) / len(phases) for k, name in enumerate(("projection", "finalize", "update"))}
     return start.elapsed_time(stop), launches, phase_ms, clocks.summary(t0, t1)
@@ -410,7 +428,7 @@ def run_ours(args, wl, rank, world, local_rank):
         "config": {"workload": wl.name, "matrices": n, "params": wl.params, "rank": wl.rank, "mode": wl.mode,
                    "T": wl.T, "lr": wl.lr, "wd": wl.wd, "states": "bf16" if args.bf16_states else "f32", "replicas": world,
                    "p_storage": "kept" if args.keep_p else "per_step", "workspace_bytes": workspace,
-                   "tuning": args.tuning or "default",
+                   "tuning": args.tuning or "default", "range_size": RANGE_SIZE,
                    "l2": "inputs (W, G: %.1f GB) exceed L2, no flush" % (2 * wl.params * 2 / 1e9)},
         "roofline": {"bound": "hbm", "kernel": "update_kernel", "achieved": upd_gbs, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": upd_gbs / peaks["hbm_gbs"], "traffic": traffic,
@@ -475,6 +493,8 @@ def main():
     ap.add_argument("--bf16-states", action="store_true", help="keep M and V in bfloat16 (a variant, not the headline)")
     ap.add_argument("--keep-p", action="store_true",
                     help="keep every matrix's projection for its epoch (APOLLO_FLAG_KEEP_P) instead of regenerating it every step")
+    ap.add_argument("--range-size", type=int, default=0,
+                    help="step the list in ranges of this many matrices with apollo_step_range (measurement aid; 0: apollo_step)")
     ap.add_argument("--tuning", default="", help="apollo_tuning fields, e.g. p_generator=1,scratch_mb=64 (measurement aid)")
     ap.add_argument("--also", default="llama1b,llama7b_mini,llama350m", help="other lists timed in the same run")
     ap.add_argument("--no-also", action="store_true")
@@ -487,6 +507,11 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    global RANGE_SIZE
+    RANGE_SIZE = args.range_size
+    if RANGE_SIZE > 0:
+        args.no_e2e = args.no_moved = args.no_also = True
+        args.sustain_s = 0.0
     wl = WL.workload(args.workload)
     if args.layers > 0:
         wl.shapes = wl.shapes[:7 * args.layers]
