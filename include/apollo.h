@@ -12,10 +12,12 @@
  * (m = the shorter stored side; on a tie the rows are the projected side):
  *   1. P (r x m), entries N(0, 1/r), is regenerated from a counter-based Philox4x32-10
  *      stream keyed by the seed, with counter (column quad, row, matrix index,
- *      epoch = floor(t / T)); it is never stored (Algorithm 1, "P_t <- N_seed(0, 1/r)";
+ *      epoch = floor(t / T)); it is regenerated in every step and not kept from one step
+ *      to the next unless APOLLO_FLAG_KEEP_P asks for it (Algorithm 1, "P_t <- N_seed(0, 1/r)";
  *      Section "Generating random projection matrix").  P has the precision of the
  *      projection's operands: its standard normals are rounded to bfloat16 for bf16
- *      gradients at rank > 1, and kept in fp32 for fp32 gradients and at rank 1.
+ *      gradients at rank > 1; for fp32 gradients and at rank 1 they are fp32 (on the tensor
+ *      cores: a bfloat16 high part plus a bfloat16 low part, 16 mantissa bits, like G).
  *   2. R = P G  (r x n)                                        (Algorithm 1, step 1).
  *   3. M <- beta1 M + (1-beta1) R,  V <- beta2 V + (1-beta2) R^2,
  *      R~ = M / (sqrt(V) + eps)                                (Algorithm 1, step 2).
