@@ -115,7 +115,7 @@ int tensor_path_configure(int rank, uint32_t flags, const apollo_tuning* tuning,
     t.scratch_bytes = (int64_t)(tu.scratch_mb ? tu.scratch_mb : 128) << 20;
     t.repitch_bytes = (int64_t)tu.repitch_mb << 20;      // 0: no limit, every matrix has its own copy (one projection launch)
     t.epi_prefetch = tu.epi_prefetch ? tu.epi_prefetch - 1 : 1;
-    t.raw_allowed = tu.realign == 1 ? 1 : 0;      // default: padded copy (the faster of the two as measured)
+    t.raw_allowed = tu.realign == 1 ? 1 : 0;      // default: padded copy (5 % faster on the 1B list, at 1.07 GB of workspace)
     // Staged P has two kernels: the pair kernel (default; faster on every list measured) and the single-CTA
     // ring kernel, which is also the one that can generate P in shared memory.
     if (t.staged && tu.kernel == APOLLO_TC_KERNEL_PAIR) {   // (APOLLO_P_SHARED always runs on the ring kernel)
@@ -1028,42 +1028,45 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                     const int c = lane & 7, a_lo = lane >> 3;
                     uint4 o[8];
                     if (ok) {
+                        // one row residue (four passes) at a time: its eight 16-byte loads are issued together, and the
+                        // shift is done without a branch (the word part of the offset by selects, the half-word part by
+                        // the funnel shift), so that nothing keeps the loads of the second residue from overlapping it
 #pragma unroll
-                        for (int pass = 0; pass < 8; ++pass) {
-                            const int b = 2 * (warp - 4) + (pass >> 2), h = (pass >> 1) & 1, a = a_lo + 4 * (pass & 1);
-                            const uint32_t src = g_s + (uint32_t)((b * 8 + a) * (RAW_BOX_W * 2) + (h * 8 + c) * 16);
-                            const uint4 lo = ld_shared_v4(src), hi = ld_shared_v4(src + 16);
-                            const uint32_t mis = (uint32_t)((b * cols + j0) & 7) * 2u, wsel = mis >> 2, sh = (mis & 2u) * 8u;
-                            const uint32_t w[8] = { lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w };
-                            uint32_t v[4];
-                            switch (wsel) {          // uniform over the warp
-                            case 0:
+                        for (int bsel = 0; bsel < 2; ++bsel) {
+                            const int b = 2 * (warp - 4) + bsel;
+                            uint4 lo[4], hi[4];
 #pragma unroll
-                                for (int k = 0; k < 4; ++k) v[k] = __funnelshift_r(w[k], w[k + 1], sh);
-                                break;
-                            case 1:
-#pragma unroll
-                                for (int k = 0; k < 4; ++k) v[k] = __funnelshift_r(w[k + 1], w[k + 2], sh);
-                                break;
-                            case 2:
-#pragma unroll
-                                for (int k = 0; k < 4; ++k) v[k] = __funnelshift_r(w[k + 2], w[k + 3], sh);
-                                break;
-                            default:
-#pragma unroll
-                                for (int k = 0; k < 4; ++k) v[k] = __funnelshift_r(w[k + 3], w[k + 4], sh);
-                                break;
+                            for (int p4 = 0; p4 < 4; ++p4) {
+                                const int h = p4 >> 1, a = a_lo + 4 * (p4 & 1);
+                                const uint32_t src = g_s + (uint32_t)((b * 8 + a) * (RAW_BOX_W * 2) + (h * 8 + c) * 16);
+                                lo[p4] = ld_shared_v4(src);
+                                hi[p4] = ld_shared_v4(src + 16);
                             }
-                            // channels at and beyond the end of the row hold the next row's elements: zero them
-                            const int jc = j0 + h * 64 + c * 8;
-                            if (jc + 8 > cols) {
+                            const uint32_t mis = (uint32_t)((b * cols + j0) & 7) * 2u, wsel = mis >> 2, sh = (mis & 2u) * 8u;
+                            const bool s1 = wsel >= 1u, s2 = wsel >= 2u, s3 = wsel >= 3u;
+#pragma unroll
+                            for (int p4 = 0; p4 < 4; ++p4) {
+                                const uint32_t w[8] = { lo[p4].x, lo[p4].y, lo[p4].z, lo[p4].w, hi[p4].x, hi[p4].y, hi[p4].z, hi[p4].w };
+                                uint32_t u[5];       // words wsel .. wsel + 4 of the piece
+#pragma unroll
+                                for (int k = 0; k < 5; ++k) u[k] = s2 ? (s3 ? w[k + 3] : w[k + 2]) : (s1 ? w[k + 1] : w[k]);
+                                o[4 * bsel + p4] = make_uint4(__funnelshift_r(u[0], u[1], sh), __funnelshift_r(u[1], u[2], sh),
+                                                              __funnelshift_r(u[2], u[3], sh), __funnelshift_r(u[3], u[4], sh));
+                            }
+                        }
+                        // channels at and beyond the end of the row hold the next row's elements: zero them (last channel tile only)
+                        if (j0 + 128 > cols) {
+#pragma unroll
+                            for (int pass = 0; pass < 8; ++pass) {
+                                const int jc = j0 + ((pass >> 1) & 1) * 64 + c * 8;
+                                uint32_t v[4] = { o[pass].x, o[pass].y, o[pass].z, o[pass].w };
 #pragma unroll
                                 for (int k = 0; k < 4; ++k) {
                                     if (jc + 2 * k >= cols) v[k] = 0u;
                                     else if (jc + 2 * k + 1 >= cols) v[k] &= 0xFFFFu;
                                 }
+                                o[pass] = make_uint4(v[0], v[1], v[2], v[3]);
                             }
-                            o[pass] = make_uint4(v[0], v[1], v[2], v[3]);
                         }
                     }
                     // all four norm warps have read before anyone writes (a bounded wait like every other: a warp
@@ -1071,18 +1074,23 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                     __syncwarp();
                     if (!ok) break;
                     if (lane == 0) ptx::mbar_arrive(bar_read + 8 * s);
+                    // the column norms need only the registers: they fill the wait for the other three warps
+                    if (tr == 0) {
+#pragma unroll
+                        for (int pass = 0; pass < 8; ++pass) {
+                            const int h = (pass >> 1) & 1;
+                            ptx::fma_sq_f32x2(acc2[h * 4 + 0], ptx::bf16x2_to_f32x2(o[pass].x));
+                            ptx::fma_sq_f32x2(acc2[h * 4 + 1], ptx::bf16x2_to_f32x2(o[pass].y));
+                            ptx::fma_sq_f32x2(acc2[h * 4 + 2], ptx::bf16x2_to_f32x2(o[pass].z));
+                            ptx::fma_sq_f32x2(acc2[h * 4 + 3], ptx::bf16x2_to_f32x2(o[pass].w));
+                        }
+                    }
                     if (!__all_sync(0xFFFFFFFFu, wait_phase(bar_read + 8 * s, rph, abort_flag, status, 109))) break;
 #pragma unroll
                     for (int pass = 0; pass < 8; ++pass) {
                         const int b = 2 * (warp - 4) + (pass >> 2), h = (pass >> 1) & 1, a = a_lo + 4 * (pass & 1);
                         const int krow = 8 * a + b;      // row of the k-block
                         st_shared_v4(g_s + (uint32_t)(h * (P2_G_BYTES / 2) + krow * 128 + ((c ^ (krow & 7)) << 4)), o[pass]);
-                        if (tr == 0) {
-                            ptx::fma_sq_f32x2(acc2[h * 4 + 0], ptx::bf16x2_to_f32x2(o[pass].x));
-                            ptx::fma_sq_f32x2(acc2[h * 4 + 1], ptx::bf16x2_to_f32x2(o[pass].y));
-                            ptx::fma_sq_f32x2(acc2[h * 4 + 2], ptx::bf16x2_to_f32x2(o[pass].z));
-                            ptx::fma_sq_f32x2(acc2[h * 4 + 3], ptx::bf16x2_to_f32x2(o[pass].w));
-                        }
                     }
                     ptx::fence_proxy_async_smem();      // the tile was written by plain stores; the MMA reads it through the async proxy
                     __syncwarp();

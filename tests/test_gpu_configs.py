@@ -43,6 +43,15 @@ def test_llama1b_rank512_ten_steps_across_a_refresh():
     assert worst["dw"] <= 1.0 and worst["exempt"] == 0.0
 
 
+def test_llama1b_realigned_in_the_kernel():
+    """The same list with the 2048 x 5461 gradients fetched as they lie and re-aligned in shared memory
+    (apollo_tuning.realign = 1: no padded copies): six steps across a refresh, the two kinds of MLP matrices."""
+    wl = WL.workload("llama1b")
+    wl.T = 3
+    worst = run_parity(wl, steps=6, check_mats=[4, 6], gen_device="cuda", tuning=B.make_tuning(realign=1))
+    assert worst["dw"] <= 1.0 and worst["exempt"] == 0.0
+
+
 def test_llama7b_mini_full_list_ten_steps_across_a_refresh():
     """All 224 matrices at rank 1 with the tensor-wise scale, ten consecutive steps with the
     projection refreshed at step 5; four matrices of every kind on the oracle in full."""
