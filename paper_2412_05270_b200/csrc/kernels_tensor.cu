@@ -761,7 +761,9 @@ static_assert(P2_MISC_BYTES == 1536, "tensor_path_configure() reserves this many
 // bfloat16 high/low copies, P_hi G_hi + P_lo G_hi + P_hi G_lo (what is dropped, P_lo G_lo, is 2^-16 of a
 // term), and the column norms come from the kernel that made the copies.  A third instantiation, for the
 // same reason as the second.
-template <bool RAW, bool SPLIT>
+// SB16: M and V are stored as bfloat16 (StepParams::state_bf16) -- a compile-time fact of the epilogue: as a run-time
+// flag on every load and store it cost the fp32 lists up to 4 % of the pass.
+template <bool RAW, bool SPLIT, bool SB16>
 __global__ void __launch_bounds__(P2_THREADS, 1)
 project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ prefix, int n_mat, int tile_begin,
                     int tile_end, StepParams sp, TcTiling tl, GenArgs gen, int32_t* __restrict__ status)
@@ -1196,7 +1198,7 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
             const int64_t tile_el = (int64_t)(j0 >> 7) * sp.rank_pad * 128;
             const bool pf = tl.epi_prefetch != 0 && j0 + q * 32 < n;
             const char* const pf_base = reinterpret_cast<const char*>(lane < 16 ? Mbase : Vbase);
-            const int64_t pf_esz = sp.state_bf16 != 0 ? 2 : 4;
+            const int64_t pf_esz = SB16 ? 2 : 4;
             auto ask = [&](int chunk) {
                 ptx::prefetch_l2(pf_base + (tile_el + (int64_t)(r0 + chunk * 16 + (lane & 15)) * 128 + q * 32) * pf_esz);
             };
@@ -1218,7 +1220,7 @@ project_pair_kernel(const MatDesc* __restrict__ descs, const int* __restrict__ p
                                               tile_el + (int64_t)(r0 + cchunk * 16 + 15) * 128 + ch,
                                               state_elements(n, sp.rank_pad, true), status)) {
                     const int64_t at = tile_el + (int64_t)(r0 + cchunk * 16) * 128 + ch;
-                    const bool sb = sp.state_bf16 != 0;
+                    constexpr bool sb = SB16;
                     float mv[16], vv[16];
 #pragma unroll
                     for (int k = 0; k < 16; ++k) {
@@ -1461,11 +1463,17 @@ void launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_ma
     const int tiles = tile_end - tile_begin;
     if (tiles <= 0) return;
     // the shared-memory opt-in is a per-device attribute of the kernels: set once per context
+    // the instantiation of the pair kernel for this context: re-aligned tiles, fp32 split, bfloat16 moments
+    typedef void (*PairKernel)(const MatDesc*, const int*, int, int, int, StepParams, TcTiling, GenArgs, int32_t*);
+    static const PairKernel pair_kernels[3][2] = {
+        { project_pair_kernel<false, false, false>, project_pair_kernel<false, false, true> },
+        { project_pair_kernel<true, false, false>, project_pair_kernel<true, false, true> },
+        { project_pair_kernel<false, true, false>, project_pair_kernel<false, true, true> },
+    };
+    const PairKernel pair_kernel = pair_kernels[tl.split ? 2 : (tl.raw ? 1 : 0)][sp.state_bf16 ? 1 : 0];
     if (!state.attr_set) {
         cudaFuncSetAttribute(project_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
-        cudaFuncSetAttribute(project_pair_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
-        cudaFuncSetAttribute(project_pair_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
-        cudaFuncSetAttribute(project_pair_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
+        cudaFuncSetAttribute(pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_MAX_SMEM);
         state.attr_set = true;
     }
     if (tl.pair) {
@@ -1483,10 +1491,7 @@ void launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_ma
         // (a pair sits in one GPC, so this can be fewer than half the SMs)
         if (state.max_pairs == 0) {
             int clusters = 0;
-            const cudaError_t oe = tl.split ? cudaOccupancyMaxActiveClusters(&clusters, project_pair_kernel<false, true>, &cfg)
-                                   : tl.raw ? cudaOccupancyMaxActiveClusters(&clusters, project_pair_kernel<true, false>, &cfg)
-                                            : cudaOccupancyMaxActiveClusters(&clusters, project_pair_kernel<false, false>, &cfg);
-            if (oe != cudaSuccess || clusters < 1) {
+            if (cudaOccupancyMaxActiveClusters(&clusters, pair_kernel, &cfg) != cudaSuccess || clusters < 1) {
                 cudaGetLastError();
                 clusters = sm_count / 2;
             }
@@ -1495,12 +1500,7 @@ void launch_project_tensor(const MatDesc* d_descs, const int* d_prefix, int n_ma
         int pairs = state.max_pairs;
         if (tiles < pairs) pairs = tiles;
         cfg.gridDim = dim3(2 * pairs);
-        if (tl.split)
-            cudaLaunchKernelEx(&cfg, project_pair_kernel<false, true>, d_descs, d_prefix, n_mat, tile_begin, tile_end, sp, tl, gen, d_status);
-        else if (tl.raw)
-            cudaLaunchKernelEx(&cfg, project_pair_kernel<true, false>, d_descs, d_prefix, n_mat, tile_begin, tile_end, sp, tl, gen, d_status);
-        else
-            cudaLaunchKernelEx(&cfg, project_pair_kernel<false, false>, d_descs, d_prefix, n_mat, tile_begin, tile_end, sp, tl, gen, d_status);
+        cudaLaunchKernelEx(&cfg, pair_kernel, d_descs, d_prefix, n_mat, tile_begin, tile_end, sp, tl, gen, d_status);
         return;
     }
     const int grid = tiles < sm_count ? tiles : sm_count;
